@@ -1,0 +1,168 @@
+/*
+ * mava_rollout.h -- C ABI of the fused multi-agent rollout + GAE library (CUDA, sm_100a).
+ *
+ * The library runs, entirely on one GPU, the data-parallel "roll out experience from
+ * vectorised environment copies" stage of the Anakin training loop described in the Mava
+ * technical report (Section 2, "Strong baseline algorithms and training architectures",
+ * and Figure 2), followed by advantage estimation for the multi-agent PPO systems the
+ * report names (IPPO with per-agent critics, MAPPO with a centralised critic).
+ *
+ * E level-based-foraging gridworlds (the report's LBF tasks, Section 4) with N agents
+ * each are stepped T times.  One step, per environment:
+ *     observe -> actor/critic MLP forward -> categorical sample (Philox4x32-10,
+ *     inverse CDF) -> environment transition -> auto-reset when the episode ended.
+ *
+ * General rules
+ *   - Every function returns MAVA_OK (0) or a negative MAVA_ERR_* code; nothing throws,
+ *     aborts or exits.  mava_strerror() names a code.
+ *   - "device pointer" = memory of the CUDA device that was current at create time;
+ *     "host pointer" = ordinary (preferably pinned) host memory.
+ *   - Work is enqueued on the stream given at create time and the call returns without
+ *     waiting, unless stated otherwise.  Problems found by a kernel (a bounded wait that
+ *     ran out) are recorded in a device status word that mava_rollout_status() reads.
+ *   - The caller owns the trajectory buffers and the parameters; the library owns only
+ *     the handle and its small internal device state (environment states, re-laid-out
+ *     weights, status word), allocated at create and freed at destroy.
+ *   - The library has no CPU fallback: without a CUDA device create fails.
+ */
+#ifndef MAVA_ROLLOUT_H
+#define MAVA_ROLLOUT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MAVA_OK 0
+#define MAVA_ERR_INVALID_ARG (-1)    /* null pointer, non-positive size, value out of range      */
+#define MAVA_ERR_UNSUPPORTED (-2)    /* shape outside the compiled table, or not an sm_100 GPU   */
+#define MAVA_ERR_CUDA (-3)           /* a CUDA runtime call failed                               */
+#define MAVA_ERR_DEVICE_TIMEOUT (-4) /* a bounded device-side wait gave up (see status)          */
+#define MAVA_ERR_CAPACITY (-5)       /* T larger than max_T, or a size beyond a stated maximum   */
+
+#define MAVA_N_ACTIONS 6 /* 0 noop, 1 up (r-1), 2 down (r+1), 3 left (c-1), 4 right (c+1), 5 load */
+
+#define MAVA_NET_SHARED_TORSO 0 /* one torso, a 6-logit actor head and a value head (IPPO-style)   */
+#define MAVA_NET_CENTRAL_CRITIC 1 /* actor net per agent + critic on the joint observation (MAPPO) */
+
+#define MAVA_PRECISION_FP32 0 /* fp32 SIMT arithmetic (validation path)                            */
+#define MAVA_PRECISION_BF16 1 /* bf16 operands, fp32 accumulation on the tcgen05 tensor cores      */
+
+#define MAVA_FLAG_WRITE_LOGITS 1 /* also write the six logits of every row to buffers.logits       */
+
+typedef struct mava_rollout mava_rollout_t; /* opaque, owned by the library */
+
+/* Plain data, copied at create.  The observation width is D = 3*(2*view_radius+1)^2 + 2 + n_agents. */
+typedef struct {
+  int32_t grid;            /* G: playable area is G x G cells; everything outside is wall         */
+  int32_t n_agents;        /* N agents per environment                                            */
+  int32_t n_food;          /* F food items per environment                                        */
+  int32_t max_agent_level; /* agent levels are uniform in 1..max_agent_level (at most 3)          */
+  int32_t view_radius;     /* egocentric window radius; only 2 is compiled                        */
+  int32_t episode_cap;     /* an episode ends when its step count reaches this                    */
+  int32_t n_envs;          /* E                                                                   */
+  int32_t max_T;           /* capacity, in steps, of the caller's trajectory buffers              */
+  int32_t hidden;          /* H, width of both hidden layers                                      */
+  int32_t net_kind;        /* MAVA_NET_*                                                          */
+  int32_t precision;       /* MAVA_PRECISION_*                                                    */
+  int32_t flags;           /* MAVA_FLAG_* bits                                                    */
+  int32_t first_env;       /* global index of this handle's environment 0 (keys Philox), so that
+                              shards of one large batch reproduce the unsharded run; usually 0    */
+  int32_t reserved;        /* must be 0                                                           */
+  uint64_t seed;           /* keys every Philox stream                                            */
+} mava_config_t;
+
+/* Device pointers to caller-owned, time-major trajectory buffers (M = E*N agent rows per step).
+ * adv/ret may be NULL if mava_gae is never called; logits may be NULL unless
+ * MAVA_FLAG_WRITE_LOGITS is set.  All must stay valid until destroy.  obs must be 16-byte
+ * aligned. */
+typedef struct {
+  float *obs;       /* [max_T][E][N][D]  observation each agent acted on                       */
+  int32_t *actions; /* [max_T][E][N]     action taken                                          */
+  float *logp;      /* [max_T][E][N]     log-probability of that action                        */
+  float *values;    /* [max_T+1][E][N]   critic value of the row; row T = bootstrap            */
+  float *rewards;   /* [max_T][E][N]     shared reward, replicated over the env's agents       */
+  uint8_t *dones;   /* [max_T][E]        1 when the step ended the episode                     */
+  float *adv;       /* [max_T][E][N]     GAE advantages                                        */
+  float *ret;       /* [max_T][E][N]     returns = advantages + values                         */
+  float *logits;    /* [max_T][E][N][6]  optional                                              */
+} mava_buffers_t;
+
+/* The same arrays in host memory, for mava_rollout_collect_host (any pointer may be NULL to
+ * skip that array). */
+typedef mava_buffers_t mava_host_buffers_t;
+
+/* Number of floats in the flat parameter array.  Layout: dense layers as weight[out][in]
+ * (y = x W^T + b) followed by bias[out], in this order
+ *   MAVA_NET_SHARED_TORSO:   W1[H][D] b1  W2[H][H] b2  Wa[6][H] ba  Wv[1][H] bv
+ *   MAVA_NET_CENTRAL_CRITIC: W1[H][D] b1  W2[H][H] b2  Wa[6][H] ba  (actor, per agent)
+ *                            C1[H][N*D] c1  C2[H][H] c2  Cv[1][H] cv (critic; its input is the
+ *                            observations of agents 0..N-1 concatenated)
+ * ReLU follows both hidden layers; heads are linear.  Returns 0 for an invalid config. */
+size_t mava_params_count(const mava_config_t *cfg);
+
+/* Validates cfg, allocates the handle and its device state on the current device, places every
+ * environment at the start of episode 0 (positions and levels from Philox keyed by
+ * (seed, env, episode)) and stores the handle in *out.  `cuda_stream` is a cudaStream_t (NULL =
+ * default stream).  Synchronous.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int mava_rollout_create(const mava_config_t *cfg, const mava_buffers_t *buffers, void *cuda_stream,
+                        mava_rollout_t **out);
+
+/* The fused rollout (Figure 2: "rolls out independent experience from N copies of the
+ * environment").  Continues from the handle's environment states for T steps (1 <= T <= max_T),
+ * writing rows 0..T-1 of obs, actions, logp, values, rewards, dones (and logits when flagged) and
+ * the bootstrap row values[T].  params_dev: device pointer to mava_params_count floats, read
+ * during the call's kernels (must stay valid until they finish).  With the central critic the one
+ * value of an environment is written to all its N slots.  Asynchronous.
+ * Errors: INVALID_ARG, CAPACITY, CUDA. */
+int mava_rollout_run(mava_rollout_t *h, const float *params_dev, int32_t T);
+
+/* Same, but every action is taken from actions_dev ([T][E][N] int32, device pointer, values 0..5)
+ * instead of being sampled ("teacher forcing"); the given actions are copied to buffers.actions
+ * and logp is that of the forced action. */
+int mava_rollout_run_forced(mava_rollout_t *h, const float *params_dev, int32_t T,
+                            const int32_t *actions_dev);
+
+/* Generalised advantage estimation over the rows of the last run (multi-agent PPO, Section 2):
+ *   delta_t = r_t + gamma V_{t+1} (1-d_t) - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1},
+ *   A_T = 0;  Ret_t = A_t + V_t.
+ * Reads values, rewards, dones; writes adv and ret.  Asynchronous.
+ * Errors: INVALID_ARG (no run yet, adv/ret NULL), CUDA. */
+int mava_gae(mava_rollout_t *h, float gamma, float lambda);
+
+/* Back to episode 0 and global step 0 under a new seed.  Asynchronous. */
+int mava_rollout_reset(mava_rollout_t *h, uint64_t seed);
+
+/* Waits for the stream, then returns MAVA_OK, MAVA_ERR_DEVICE_TIMEOUT if a kernel's bounded wait
+ * gave up since the last call (the status word is cleared), or MAVA_ERR_CUDA. */
+int mava_rollout_status(mava_rollout_t *h);
+
+/* Environment states as int32 records of mava_state_record_len(cfg) words per environment:
+ * N x (row, col, level), F x (row, col, level; level 0 = collected), step, episode,
+ * total food level at reset.  Host pointers; both calls wait for the stream.  set validates
+ * ranges (INVALID_ARG) and leaves the global step counter unchanged. */
+int32_t mava_state_record_len(const mava_config_t *cfg);
+int mava_rollout_get_state(mava_rollout_t *h, int32_t *records_host);
+int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host);
+
+/* End-to-end convenience with HOST buffers: copies params_host to the device, runs T steps and
+ * GAE, copies every non-NULL array of `out` back to the host (rows 0..T-1; T+1 rows of values)
+ * and waits.  The caller's device buffers given at create are used as staging.  Synchronous.
+ * Errors: as run and gae. */
+int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32_t T, float gamma,
+                              float lambda, const mava_host_buffers_t *out);
+
+/* Number of kernels this handle has launched so far (for launch accounting). */
+int64_t mava_rollout_launch_count(const mava_rollout_t *h);
+
+/* Frees the handle and its device state after waiting for the stream.  NULL is allowed. */
+void mava_rollout_destroy(mava_rollout_t *h);
+
+const char *mava_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAVA_ROLLOUT_H */

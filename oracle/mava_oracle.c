@@ -398,7 +398,8 @@ int orc_rollout(const orc_config_t *cfg, uint64_t seed, const float *params, int
     orc_env_state_t *s = &states[i];
     for (int t = 0; t <= T; ++t) {
       const size_t row0 = ((size_t)t * E_arr + p) * N; /* first agent row of (t, env) */
-      for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
+      if (obs || compute_mlp)
+        for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
       if (t < T && obs) memcpy(obs + row0 * D, o, sizeof(float) * (size_t)N * D);
       if (compute_mlp) {
         orc_mlp_forward_env(cfg, params, o, emulate_bf16, lg, val);

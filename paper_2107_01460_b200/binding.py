@@ -1,0 +1,192 @@
+"""Thin ctypes binding of libmava_rollout.so: same entry-point names as the C header, argument
+marshalling only.  PyTorch is used for device memory and streams; every step of the rollout and
+of GAE runs inside the library's CUDA kernels.  There is no fallback: if the shared library has
+not been built (``python -m paper_2107_01460_b200.build``) loading raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmava_rollout.so")
+
+MAVA_OK = 0
+MAVA_ERR_INVALID_ARG = -1
+MAVA_ERR_UNSUPPORTED = -2
+MAVA_ERR_CUDA = -3
+MAVA_ERR_DEVICE_TIMEOUT = -4
+MAVA_ERR_CAPACITY = -5
+MAVA_NET_SHARED_TORSO = 0
+MAVA_NET_CENTRAL_CRITIC = 1
+MAVA_PRECISION_FP32 = 0
+MAVA_PRECISION_BF16 = 1
+MAVA_FLAG_WRITE_LOGITS = 1
+N_ACTIONS = 6
+
+EXPORTS = [
+    "mava_params_count", "mava_rollout_create", "mava_rollout_run", "mava_rollout_run_forced", "mava_gae",
+    "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
+    "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
+    "mava_strerror",
+]
+
+
+class mava_config_t(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "grid", "n_agents", "n_food", "max_agent_level", "view_radius", "episode_cap", "n_envs", "max_T", "hidden",
+        "net_kind", "precision", "flags", "first_env", "reserved")] + [("seed", C.c_uint64)]
+
+
+class mava_buffers_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "obs", "actions", "logp", "values", "rewards", "dones", "adv", "ret", "logits")]
+
+
+class MavaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library (raises FileNotFoundError / OSError if it was not built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2107_01460_b200.build` (there is no fallback)")
+        L = C.CDLL(LIB_PATH)
+        cfgp, bufp, vp = C.POINTER(mava_config_t), C.POINTER(mava_buffers_t), C.c_void_p
+        L.mava_params_count.argtypes = [cfgp]; L.mava_params_count.restype = C.c_size_t
+        L.mava_state_record_len.argtypes = [cfgp]; L.mava_state_record_len.restype = C.c_int32
+        L.mava_rollout_create.argtypes = [cfgp, bufp, vp, C.POINTER(vp)]; L.mava_rollout_create.restype = C.c_int
+        L.mava_rollout_run.argtypes = [vp, vp, C.c_int32]; L.mava_rollout_run.restype = C.c_int
+        L.mava_rollout_run_forced.argtypes = [vp, vp, C.c_int32, vp]; L.mava_rollout_run_forced.restype = C.c_int
+        L.mava_gae.argtypes = [vp, C.c_float, C.c_float]; L.mava_gae.restype = C.c_int
+        L.mava_rollout_reset.argtypes = [vp, C.c_uint64]; L.mava_rollout_reset.restype = C.c_int
+        L.mava_rollout_status.argtypes = [vp]; L.mava_rollout_status.restype = C.c_int
+        L.mava_rollout_get_state.argtypes = [vp, vp]; L.mava_rollout_get_state.restype = C.c_int
+        L.mava_rollout_set_state.argtypes = [vp, vp]; L.mava_rollout_set_state.restype = C.c_int
+        L.mava_rollout_collect_host.argtypes = [vp, vp, C.c_int32, C.c_float, C.c_float, bufp]
+        L.mava_rollout_collect_host.restype = C.c_int
+        L.mava_rollout_launch_count.argtypes = [vp]; L.mava_rollout_launch_count.restype = C.c_int64
+        L.mava_rollout_destroy.argtypes = [vp]; L.mava_rollout_destroy.restype = None
+        L.mava_strerror.argtypes = [C.c_int]; L.mava_strerror.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().mava_strerror(code).decode()
+
+
+def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: int | None = None,
+                n_envs: int | None = None, seed: int | None = None, first_env: int = 0) -> mava_config_t:
+    """mava_config_t from a workload description (see ``workloads.WORKLOADS``)."""
+    if precision is None:
+        precision = MAVA_PRECISION_BF16 if w.get("precision") == "bf16" else MAVA_PRECISION_FP32
+    return mava_config_t(
+        grid=w["grid"], n_agents=w["n_agents"], n_food=w["n_food"], max_agent_level=w["max_agent_level"],
+        view_radius=w["view_radius"], episode_cap=w["episode_cap"], n_envs=w["n_envs"] if n_envs is None else n_envs,
+        max_T=w["T"] if max_T is None else max_T, hidden=w["hidden"], net_kind=w["net_kind"], precision=precision,
+        flags=flags, first_env=first_env, reserved=0, seed=w["seed"] if seed is None else seed)
+
+
+def _check(code: int, where: str):
+    if code != MAVA_OK:
+        raise MavaError(code, where)
+
+
+class Rollout:
+    """Owns the torch device tensors of one handle and forwards to the C entry points."""
+
+    def __init__(self, cfg: mava_config_t, device="cuda:0", stream=None, with_gae: bool = True):
+        import torch
+
+        self.torch = torch
+        self.cfg = cfg
+        self.device = torch.device(device)
+        E, N, T = cfg.n_envs, cfg.n_agents, cfg.max_T
+        self.D = 77 + N
+        self.n_params = int(lib().mava_params_count(C.byref(cfg)))
+        if self.n_params == 0:
+            raise MavaError(MAVA_ERR_INVALID_ARG, "mava_params_count")
+        dev = self.device
+        f32, i32, u8 = torch.float32, torch.int32, torch.uint8
+        self.obs = torch.empty((T, E, N, self.D), dtype=f32, device=dev)
+        self.actions = torch.empty((T, E, N), dtype=i32, device=dev)
+        self.logp = torch.empty((T, E, N), dtype=f32, device=dev)
+        self.values = torch.empty((T + 1, E, N), dtype=f32, device=dev)
+        self.rewards = torch.empty((T, E, N), dtype=f32, device=dev)
+        self.dones = torch.empty((T, E), dtype=u8, device=dev)
+        self.adv = torch.empty((T, E, N), dtype=f32, device=dev) if with_gae else None
+        self.ret = torch.empty((T, E, N), dtype=f32, device=dev) if with_gae else None
+        self.logits = (torch.empty((T, E, N, N_ACTIONS), dtype=f32, device=dev)
+                       if cfg.flags & MAVA_FLAG_WRITE_LOGITS else None)
+        ptr = lambda t: None if t is None else t.data_ptr()  # noqa: E731
+        self.buffers = mava_buffers_t(ptr(self.obs), ptr(self.actions), ptr(self.logp), ptr(self.values),
+                                      ptr(self.rewards), ptr(self.dones), ptr(self.adv), ptr(self.ret),
+                                      ptr(self.logits))
+        self.stream = stream if stream is not None else torch.cuda.current_stream(dev)
+        self.handle = C.c_void_p()
+        with torch.cuda.device(dev):
+            _check(lib().mava_rollout_create(C.byref(cfg), C.byref(self.buffers), C.c_void_p(self.stream.cuda_stream),
+                                             C.byref(self.handle)), "mava_rollout_create")
+
+    # -- one method per C entry point ---------------------------------------------------------
+    def run(self, params, T: int):
+        assert params.is_cuda and params.dtype == self.torch.float32 and params.numel() == self.n_params
+        _check(lib().mava_rollout_run(self.handle, params.data_ptr(), T), "mava_rollout_run")
+
+    def run_forced(self, params, T: int, actions):
+        assert actions.is_cuda and actions.dtype == self.torch.int32 and actions.is_contiguous()
+        assert params.is_cuda and params.numel() == self.n_params
+        _check(lib().mava_rollout_run_forced(self.handle, params.data_ptr(), T, actions.data_ptr()),
+               "mava_rollout_run_forced")
+
+    def gae(self, gamma: float, lam: float):
+        _check(lib().mava_gae(self.handle, gamma, lam), "mava_gae")
+
+    def reset(self, seed: int):
+        _check(lib().mava_rollout_reset(self.handle, seed), "mava_rollout_reset")
+
+    def status(self) -> int:
+        return int(lib().mava_rollout_status(self.handle))
+
+    def launch_count(self) -> int:
+        return int(lib().mava_rollout_launch_count(self.handle))
+
+    def get_state(self):
+        import numpy as np
+
+        n = int(lib().mava_state_record_len(C.byref(self.cfg)))
+        out = np.empty((self.cfg.n_envs, n), dtype=np.int32)
+        _check(lib().mava_rollout_get_state(self.handle, out.ctypes.data), "mava_rollout_get_state")
+        return out
+
+    def set_state(self, records):
+        import numpy as np
+
+        rec = np.ascontiguousarray(records, dtype=np.int32)
+        assert rec.shape == (self.cfg.n_envs, int(lib().mava_state_record_len(C.byref(self.cfg))))
+        _check(lib().mava_rollout_set_state(self.handle, rec.ctypes.data), "mava_rollout_set_state")
+
+    def collect_host(self, params_host, T: int, gamma: float, lam: float, out: dict):
+        """`out`: dict name -> pinned CPU tensor (any subset of the buffer names)."""
+        hb = mava_buffers_t(*[(out[n].data_ptr() if n in out else None) for n, _ in mava_buffers_t._fields_])
+        _check(lib().mava_rollout_collect_host(self.handle, params_host.data_ptr(), T, gamma, lam, C.byref(hb)),
+               "mava_rollout_collect_host")
+
+    def close(self):
+        if self.handle:
+            lib().mava_rollout_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

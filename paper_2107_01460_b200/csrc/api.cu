@@ -1,0 +1,283 @@
+// C ABI of libmava_rollout.so: argument checks, handle life cycle and kernel enqueueing.
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "layout.h"
+
+using namespace mava;
+
+namespace {
+
+int obs_dim(const mava_config_t &c) { return kObsFixed + c.n_agents; }
+
+bool config_ok(const mava_config_t &c) {
+  return c.grid >= 3 && c.grid <= 64 && c.n_agents >= 1 && c.n_agents <= kMaxAgents && c.n_food >= 1 &&
+         c.n_food <= kMaxFood && c.max_agent_level >= 1 && c.max_agent_level <= 3 &&
+         c.n_agents + c.n_food <= c.grid * c.grid && c.episode_cap >= 1 && c.n_envs >= 1 && c.max_T >= 1 &&
+         c.hidden >= 1 && c.first_env >= 0 && c.reserved == 0 && (c.net_kind == MAVA_NET_SHARED_TORSO || c.net_kind == MAVA_NET_CENTRAL_CRITIC) &&
+         (c.precision == MAVA_PRECISION_FP32 || c.precision == MAVA_PRECISION_BF16);
+}
+
+EnvParams env_params(const mava_rollout *h) {
+  return EnvParams{h->cfg.grid, h->cfg.max_agent_level, h->cfg.episode_cap, h->cfg.n_envs, h->cfg.first_env,
+                   static_cast<uint32_t>(h->cfg.seed), static_cast<uint32_t>(h->cfg.seed >> 32)};
+}
+
+struct DeviceGuard {  // makes the handle's device current for the duration of a call
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    ok = cudaGetDevice(&prev) == cudaSuccess && (prev == dev || cudaSetDevice(dev) == cudaSuccess);
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_t *forced) {
+  if (!h || !params_dev) return MAVA_ERR_INVALID_ARG;
+  if (T < 1) return MAVA_ERR_INVALID_ARG;
+  if (T > h->cfg.max_T) return MAVA_ERR_CAPACITY;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  RolloutArgs args{};
+  args.env = env_params(h);
+  args.buf = h->buf;
+  args.state = h->d_state;
+  args.forced = forced;
+  args.T = T;
+  args.t_global0 = h->t_global;
+  args.write_logits = (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) ? 1 : 0;
+  args.status = h->d_status;
+  cudaError_t err;
+  if (h->cfg.precision == MAVA_PRECISION_BF16) {
+    err = launch_prep_tc(h, params_dev);
+    if (err == cudaSuccess) err = launch_rollout_tc(h, args);
+  } else {
+    err = launch_prep_simt(h, params_dev);
+    if (err == cudaSuccess) err = launch_rollout_simt(h, args);
+  }
+  if (err != cudaSuccess) return MAVA_ERR_CUDA;
+  h->t_global += static_cast<uint32_t>(T);
+  h->last_T = T;
+  return MAVA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mava_params_count(const mava_config_t *cfg) {
+  if (!cfg || !config_ok(*cfg)) return 0;
+  return param_layout(*cfg, obs_dim(*cfg), 1).total;
+}
+
+int32_t mava_state_record_len(const mava_config_t *cfg) {
+  if (!cfg || !config_ok(*cfg)) return 0;
+  return 3 * (cfg->n_agents + cfg->n_food) + 3;
+}
+
+int mava_rollout_create(const mava_config_t *cfg, const mava_buffers_t *buffers, void *cuda_stream,
+                        mava_rollout_t **out) {
+  if (!cfg || !buffers || !out) return MAVA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(*cfg)) return MAVA_ERR_INVALID_ARG;
+  if (cfg->view_radius != kViewRadius) return MAVA_ERR_UNSUPPORTED;
+  if (cfg->n_agents * cfg->max_agent_level > 31) return MAVA_ERR_UNSUPPORTED;
+  const mava_buffers_t &b = *buffers;
+  if (!b.obs || !b.actions || !b.logp || !b.values || !b.rewards || !b.dones) return MAVA_ERR_INVALID_ARG;
+  if ((cfg->flags & MAVA_FLAG_WRITE_LOGITS) && !b.logits) return MAVA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(b.obs) % 16 != 0) return MAVA_ERR_INVALID_ARG;
+  const int variant = find_variant(*cfg);
+  if (variant < 0) return MAVA_ERR_UNSUPPORTED;
+  if (cfg->precision == MAVA_PRECISION_BF16 && !tc_supported(*cfg)) return MAVA_ERR_UNSUPPORTED;
+
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) return MAVA_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MAVA_ERR_CUDA;
+  if (prop.major != 10) return MAVA_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+
+  mava_rollout *h = new (std::nothrow) mava_rollout();
+  if (!h) return MAVA_ERR_CUDA;
+  h->cfg = *cfg;
+  h->buf = b;
+  h->stream = static_cast<cudaStream_t>(cuda_stream);
+  h->device = device;
+  h->D = obs_dim(*cfg);
+  h->variant = variant;
+  const size_t np = param_layout(*cfg, h->D, 1).total;
+  bool ok = cudaMalloc(&h->d_state, sizeof(EnvRec) * static_cast<size_t>(cfg->n_envs)) == cudaSuccess &&
+            cudaMalloc(&h->d_status, sizeof(int)) == cudaSuccess &&
+            cudaMalloc(&h->d_wsimt, sizeof(float) * simt_weight_floats(*cfg, h->D)) == cudaSuccess &&
+            cudaMalloc(&h->d_params_stage, sizeof(float) * np) == cudaSuccess;
+  if (ok && cfg->precision == MAVA_PRECISION_BF16)
+    ok = cudaMalloc(&h->d_wtc, tc_weight_bytes(*cfg, h->D)) == cudaSuccess;
+  if (ok) ok = cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream) == cudaSuccess;
+  if (ok) ok = launch_env_init(h) == cudaSuccess;
+  if (ok) ok = cudaStreamSynchronize(h->stream) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    mava_rollout_destroy(h);
+    return MAVA_ERR_CUDA;
+  }
+  *out = h;
+  return MAVA_OK;
+}
+
+int mava_rollout_run(mava_rollout_t *h, const float *params_dev, int32_t T) {
+  return run_common(h, params_dev, T, nullptr);
+}
+
+int mava_rollout_run_forced(mava_rollout_t *h, const float *params_dev, int32_t T, const int32_t *actions_dev) {
+  if (!actions_dev) return MAVA_ERR_INVALID_ARG;
+  return run_common(h, params_dev, T, actions_dev);
+}
+
+int mava_gae(mava_rollout_t *h, float gamma, float lambda) {
+  if (!h || h->last_T < 1 || !h->buf.adv || !h->buf.ret) return MAVA_ERR_INVALID_ARG;
+  if (!(gamma >= 0.0f && gamma <= 1.0f && lambda >= 0.0f && lambda <= 1.0f)) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  return launch_gae(h, gamma, lambda) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+}
+
+int mava_rollout_reset(mava_rollout_t *h, uint64_t seed) {
+  if (!h) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  h->cfg.seed = seed;
+  h->t_global = 0;
+  h->last_T = 0;
+  return launch_env_init(h) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+}
+
+int mava_rollout_status(mava_rollout_t *h) {
+  if (!h) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  int status = 0;
+  if (cudaMemcpyAsync(&status, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return MAVA_ERR_CUDA;
+  if (status != 0) {
+    cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream);
+    return MAVA_ERR_DEVICE_TIMEOUT;
+  }
+  return MAVA_OK;
+}
+
+int mava_rollout_get_state(mava_rollout_t *h, int32_t *records_host) {
+  if (!h || !records_host) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  const int E = h->cfg.n_envs, N = h->cfg.n_agents, F = h->cfg.n_food;
+  std::vector<EnvRec> recs(static_cast<size_t>(E));
+  if (cudaMemcpyAsync(recs.data(), h->d_state, sizeof(EnvRec) * recs.size(), cudaMemcpyDeviceToHost, h->stream) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return MAVA_ERR_CUDA;
+  const int len = 3 * (N + F) + 3;
+  for (int e = 0; e < E; ++e) {
+    int32_t *o = records_host + static_cast<size_t>(e) * len;
+    const EnvRec &s = recs[static_cast<size_t>(e)];
+    for (int n = 0; n < N; ++n) { *o++ = s.ar[n]; *o++ = s.ac[n]; *o++ = s.al[n]; }
+    for (int f = 0; f < F; ++f) { *o++ = s.fr[f]; *o++ = s.fc[f]; *o++ = s.fl[f]; }
+    *o++ = s.step; *o++ = s.episode; *o++ = s.total;
+  }
+  return MAVA_OK;
+}
+
+int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host) {
+  if (!h || !records_host) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  const int E = h->cfg.n_envs, N = h->cfg.n_agents, F = h->cfg.n_food, G = h->cfg.grid;
+  const int len = 3 * (N + F) + 3;
+  std::vector<EnvRec> recs(static_cast<size_t>(E));
+  for (int e = 0; e < E; ++e) {
+    const int32_t *in = records_host + static_cast<size_t>(e) * len;
+    EnvRec s{};
+    for (int n = 0; n < N; ++n) {
+      const int r = *in++, c = *in++, l = *in++;
+      if (r < 0 || r >= G || c < 0 || c >= G || l < 1 || l > 3) return MAVA_ERR_INVALID_ARG;
+      s.ar[n] = static_cast<uint8_t>(r); s.ac[n] = static_cast<uint8_t>(c); s.al[n] = static_cast<uint8_t>(l);
+    }
+    for (int f = 0; f < F; ++f) {
+      const int r = *in++, c = *in++, l = *in++;
+      if (r < 0 || r >= G || c < 0 || c >= G || l < 0 || l > 31) return MAVA_ERR_INVALID_ARG;
+      s.fr[f] = static_cast<uint8_t>(r); s.fc[f] = static_cast<uint8_t>(c); s.fl[f] = static_cast<uint8_t>(l);
+    }
+    s.step = *in++; s.episode = *in++; s.total = *in++;
+    if (s.step < 0 || s.step >= h->cfg.episode_cap || s.episode < 0 || s.total < 1) return MAVA_ERR_INVALID_ARG;
+    recs[static_cast<size_t>(e)] = s;
+  }
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess ||
+      cudaMemcpy(h->d_state, recs.data(), sizeof(EnvRec) * recs.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+    return MAVA_ERR_CUDA;
+  return MAVA_OK;
+}
+
+int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32_t T, float gamma, float lambda,
+                              const mava_host_buffers_t *out) {
+  if (!h || !params_host || !out) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  const size_t np = param_layout(h->cfg, h->D, 1).total;
+  if (cudaMemcpyAsync(h->d_params_stage, params_host, np * sizeof(float), cudaMemcpyHostToDevice, h->stream) !=
+      cudaSuccess)
+    return MAVA_ERR_CUDA;
+  int rc = run_common(h, h->d_params_stage, T, nullptr);
+  if (rc != MAVA_OK) return rc;
+  if (h->buf.adv && h->buf.ret) {
+    rc = mava_gae(h, gamma, lambda);
+    if (rc != MAVA_OK) return rc;
+  }
+  const size_t E = static_cast<size_t>(h->cfg.n_envs), M = E * h->cfg.n_agents, rows = M * T;
+  bool ok = true;
+  auto back = [&](void *dst, const void *src, size_t bytes) {
+    if (dst && src && ok)
+      ok = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, h->stream) == cudaSuccess;
+  };
+  back(out->obs, h->buf.obs, rows * h->D * sizeof(float));
+  back(out->actions, h->buf.actions, rows * sizeof(int32_t));
+  back(out->logp, h->buf.logp, rows * sizeof(float));
+  back(out->values, h->buf.values, (rows + M) * sizeof(float));
+  back(out->rewards, h->buf.rewards, rows * sizeof(float));
+  back(out->dones, h->buf.dones, E * T);
+  back(out->adv, h->buf.adv, rows * sizeof(float));
+  back(out->ret, h->buf.ret, rows * sizeof(float));
+  if (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) back(out->logits, h->buf.logits, rows * kActions * sizeof(float));
+  if (!ok || cudaStreamSynchronize(h->stream) != cudaSuccess) return MAVA_ERR_CUDA;
+  return MAVA_OK;
+}
+
+int64_t mava_rollout_launch_count(const mava_rollout_t *h) { return h ? h->launches : 0; }
+
+void mava_rollout_destroy(mava_rollout_t *h) {
+  if (!h) return;
+  DeviceGuard guard(h->device);
+  cudaStreamSynchronize(h->stream);
+  cudaFree(h->d_state);
+  cudaFree(h->d_status);
+  cudaFree(h->d_wsimt);
+  cudaFree(h->d_wtc);
+  cudaFree(h->d_params_stage);
+  delete h;
+}
+
+const char *mava_strerror(int code) {
+  switch (code) {
+    case MAVA_OK: return "ok";
+    case MAVA_ERR_INVALID_ARG: return "invalid argument";
+    case MAVA_ERR_UNSUPPORTED: return "unsupported configuration or device";
+    case MAVA_ERR_CUDA: return "CUDA runtime error";
+    case MAVA_ERR_DEVICE_TIMEOUT: return "a device-side bounded wait gave up";
+    case MAVA_ERR_CAPACITY: return "size beyond the stated capacity";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,94 @@
+// Internal declarations shared by the translation units of libmava_rollout.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mava_rollout.h"
+
+namespace mava {
+
+constexpr int kMaxAgents = 8;
+constexpr int kMaxFood = 8;
+constexpr int kActions = MAVA_N_ACTIONS;
+constexpr int kViewRadius = 2;
+constexpr int kWindow = 2 * kViewRadius + 1;       // 5
+constexpr int kPlane = kWindow * kWindow;          // 25
+constexpr int kObsFixed = 3 * kPlane + 2;          // 77: three planes, own level, step/cap
+
+constexpr uint32_t kDomainReset = 0x52534554u;     // key tweak of the placement stream
+constexpr uint32_t kDomainAction = 0x41435431u;    // key tweak of the action-uniform stream
+
+// Device status word values (0 = fine).
+constexpr int kStatusTimeout = 1;
+
+// Compact per-environment state.  Coordinates and levels fit a byte (G <= 64, levels <= 31).
+struct __align__(4) EnvRec {
+  uint8_t ar[kMaxAgents], ac[kMaxAgents], al[kMaxAgents];
+  uint8_t fr[kMaxFood], fc[kMaxFood], fl[kMaxFood];  // fl == 0: collected
+  int32_t step, episode, total;
+};
+static_assert(sizeof(EnvRec) == 60, "EnvRec layout");
+
+// Runtime scalars every kernel needs.
+struct EnvParams {
+  int32_t grid, max_level, cap, n_envs;
+  int32_t first_env;        // global index of local environment 0 (Philox is keyed on global indices)
+  uint32_t key_lo, key_hi;  // seed halves (domain tweak applied on use)
+};
+
+// Everything a rollout launch needs.
+struct RolloutArgs {
+  EnvParams env;
+  mava_buffers_t buf;
+  EnvRec *state;
+  const int32_t *forced;  // [T][E][N] or nullptr
+  int32_t T;
+  uint32_t t_global0;
+  int32_t write_logits;
+  int *status;
+};
+
+// Re-laid-out fp32 weights of the SIMT path: every dense layer transposed to [in][out].
+struct SimtWeights {
+  const float *W1t, *b1, *W2t, *b2, *Wa, *ba, *Wv, *bv;  // Wa [6][H], Wv [H] stay row-major
+  const float *C1t, *c1, *C2t, *c2, *Cv, *cv;            // central critic (or nullptr)
+};
+
+}  // namespace mava
+
+struct mava_rollout {
+  mava_config_t cfg;
+  mava_buffers_t buf;
+  cudaStream_t stream;
+  int device;
+  int D;            // observation width
+  int variant;      // index in the compiled shape table
+  mava::EnvRec *d_state;
+  int *d_status;
+  float *d_wsimt;   // transposed fp32 weights (SIMT path)
+  void *d_wtc;      // bf16 weights in tensor-core layout (bf16 path)
+  float *d_params_stage;  // device copy of host params (collect_host)
+  uint32_t t_global;
+  int32_t last_T;
+  int64_t launches;
+};
+
+namespace mava {
+
+// Shape table: the (N, F, H, net_kind) combinations kernels are compiled for.
+int find_variant(const mava_config_t &cfg);  // -1 if not compiled
+
+// Launchers (each returns a cudaError_t; all asynchronous on h->stream).
+cudaError_t launch_env_init(mava_rollout *h);
+cudaError_t launch_prep_simt(mava_rollout *h, const float *params_dev);
+cudaError_t launch_rollout_simt(mava_rollout *h, const RolloutArgs &args);
+cudaError_t launch_gae(mava_rollout *h, float gamma, float lambda);
+size_t simt_weight_floats(const mava_config_t &cfg, int D);
+
+// bf16 tensor-core path.
+size_t tc_weight_bytes(const mava_config_t &cfg, int D);
+cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev);
+cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args);
+bool tc_supported(const mava_config_t &cfg);
+
+}  // namespace mava

@@ -1,0 +1,109 @@
+"""GPU-vs-oracle comparison used by the gpu tests (the oracle replays the GPU's recorded actions)."""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle
+from paper_2107_01460_b200 import binding, workloads as wl
+
+TOL = {binding.MAVA_PRECISION_FP32: 1e-4, binding.MAVA_PRECISION_BF16: 2e-2}
+GAE_TOL = 1e-5
+
+
+def close(x, ref, tol):
+    """|x - ref| <= tol * (1 + |ref|), elementwise; returns the worst ratio to the bound."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.max(np.abs(x - ref) / (tol * (1.0 + np.abs(ref))))) if x.size else 0.0
+
+
+def run_gpu(w, precision, T, n_envs=None, params=None, seed=None, flags=binding.MAVA_FLAG_WRITE_LOGITS):
+    import torch
+
+    cfg = binding.make_config(w, precision=precision, flags=flags, max_T=T, n_envs=n_envs, seed=seed)
+    ro = binding.Rollout(cfg)
+    if params is None:
+        params = wl.make_params(w)
+    p_dev = torch.from_numpy(params).cuda()
+    ro.run(p_dev, T)
+    ro.gae(np.float32(wl.GAMMA), np.float32(wl.LAMBDA))
+    assert ro.status() == binding.MAVA_OK
+    return ro, p_dev
+
+
+def check_against_oracle(w, ro, params, T, precision, mlp_env_ids, obs_env_ids=None, t_global0=0, states0=None,
+                         seed=None):
+    """Full comparison of one finished GPU run; returns a dict of worst-case ratios and counts."""
+    E, N = ro.cfg.n_envs, ro.cfg.n_agents
+    seed = w["seed"] if seed is None else seed
+    ocfg = oracle.make_config(w)
+    tol = TOL[precision]
+    g = {k: getattr(ro, k)[:T].cpu().numpy() for k in ("actions", "logp", "rewards", "dones", "adv", "ret")}
+    g["values"] = ro.values[:T + 1].cpu().numpy()
+    g["logits"] = ro.logits[:T].cpu().numpy()
+    assert g["actions"].min() >= 0 and g["actions"].max() < 6
+
+    # 1. environment: bit-exact under the GPU's own actions, all environments
+    all_ids = np.arange(E, dtype=np.int32)
+    small = obs_env_ids is None
+    env = oracle.rollout(ocfg, seed, None, T, all_ids, forced_actions=g["actions"], compute_mlp=False,
+                         want_obs=small, t_global0=t_global0, states=states0)
+    assert np.array_equal(env.rewards.view(np.uint32), g["rewards"].view(np.uint32)), "rewards differ"
+    assert np.array_equal(env.dones, g["dones"]), "dones differ"
+    if small:
+        assert np.array_equal(env.obs.view(np.uint32), ro.obs[:T].cpu().numpy().view(np.uint32)), "obs differ"
+    else:
+        import torch
+
+        idx = torch.from_numpy(np.asarray(obs_env_ids, dtype=np.int64)).cuda()
+        g_obs = ro.obs[:T].index_select(1, idx).cpu().numpy()
+        sub_states = None if states0 is None else [states0[i] for i in obs_env_ids]
+        sub = oracle.rollout(ocfg, seed, None, T, obs_env_ids, forced_actions=g["actions"][:, obs_env_ids],
+                             compute_mlp=False, t_global0=t_global0, states=sub_states)
+        assert np.array_equal(sub.obs.view(np.uint32), g_obs.view(np.uint32)), "obs differ (sampled envs)"
+    # final states
+    rec = ro.get_state()
+    want = np.array([[*sum(([s.agent_r[n], s.agent_c[n], s.agent_level[n]] for n in range(N)), []),
+                      *sum(([s.food_r[f], s.food_c[f], s.food_level[f]] for f in range(ro.cfg.n_food)), []),
+                      s.step, s.episode, s.total_food_level] for s in env.states], dtype=np.int32)
+    assert np.array_equal(rec, want), "final environment states differ"
+
+    # 2. network + sampler on a subset of environments
+    ids = np.asarray(mlp_env_ids, dtype=np.int32)
+    sub_states = None if states0 is None else [states0[i] for i in ids]
+    ref = oracle.rollout(ocfg, seed, params, T, ids, forced_actions=g["actions"][:, ids], want_obs=False,
+                         t_global0=t_global0, states=sub_states)
+    out = {}
+    out["logits"] = close(g["logits"][:, ids], ref.logits, tol)
+    out["values"] = close(g["values"][:, ids], ref.values, tol)
+    out["logp"] = close(g["logp"][:, ids], ref.logp, tol)
+    assert out["logits"] <= 1.0 and out["values"] <= 1.0 and out["logp"] <= 1.0, out
+    # sampled actions: equal unless u*S sits within the propagated logit tolerance of a CDF boundary
+    max_abs_logit = np.max(np.abs(ref.logits), axis=-1)
+    eps = 4.0 * tol * (1.0 + max_abs_logit)
+    differ = g["actions"][:, ids] != ref.own_actions
+    assert not np.any(differ & (ref.margin > eps)), "an action differs away from a CDF boundary"
+    out["excused_actions"] = int(differ.sum())
+    out["rows"] = int(differ.size)
+    assert out["excused_actions"] <= max(2, int(10 * tol * differ.size)), out
+
+    # 3. the sampler itself, exactly: re-sample in double from the GPU's own logits
+    lg = g["logits"][:, ids].astype(np.float64)
+    bad = 0
+    for t in range(T):
+        for i, e in enumerate(ids):
+            for n in range(N):
+                u = oracle.lib().orc_action_uniform(seed, t_global0 + t, int(e), n)
+                a, lp, m = oracle.sample(lg[t, i, n], u)
+                if a != g["actions"][t, e, n]:
+                    assert m < 1e-5, ("sampler disagrees with its own logits", t, e, n, m)
+                    bad += 1
+                assert abs(lp[g["actions"][t, e, n]] - g["logp"][t, e, n]) <= 1e-5 * (1 + abs(lp[a]))
+    out["sampler_boundary_cases"] = bad
+
+    # 4. GAE over the GPU's own values / rewards / dones, every element
+    adv, ret = oracle.gae(g["values"], g["rewards"], g["dones"], float(np.float32(wl.GAMMA)), float(np.float32(wl.LAMBDA)))
+    out["adv"] = float(np.max(np.abs(g["adv"] - adv) / (GAE_TOL * np.maximum(1.0, np.abs(adv)))))
+    out["ret"] = float(np.max(np.abs(g["ret"] - ret) / (GAE_TOL * np.maximum(1.0, np.abs(ret)))))
+    assert out["adv"] <= 1.0 and out["ret"] <= 1.0, out
+    return out

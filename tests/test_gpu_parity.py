@@ -1,0 +1,219 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2107_01460_b200 import binding, workloads as wl
+
+from parity import check_against_oracle, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+FP32 = binding.MAVA_PRECISION_FP32
+BF16 = binding.MAVA_PRECISION_BF16
+
+
+def _precision(w):
+    return BF16 if w["precision"] == "bf16" else FP32
+
+
+def _tc_available(w):
+    import ctypes as C
+
+    cfg = binding.make_config(w, precision=BF16)
+    return bool(binding.lib().mava_params_count(C.byref(cfg))) and _try_create(cfg)
+
+
+def _try_create(cfg):
+    try:
+        cfg2 = binding.mava_config_t.from_buffer_copy(cfg)
+        cfg2.n_envs, cfg2.max_T = 4, 2
+        binding.Rollout(cfg2).close()
+        return True
+    except binding.MavaError as e:
+        if e.code == binding.MAVA_ERR_UNSUPPORTED:
+            return False
+        raise
+
+
+# ---- whole small config, every environment checked -------------------------------------------
+
+@pytest.mark.parametrize("bias_scale", [0.0, 0.5])
+def test_cfg0_fp32_every_row(bias_scale):
+    w = wl.workload(0)
+    params = wl.make_params(w, bias_scale=bias_scale)
+    ro, _ = run_gpu(w, FP32, w["T"], params=params)
+    out = check_against_oracle(w, ro, params, w["T"], FP32, np.arange(w["n_envs"]))
+    print(out)
+
+
+def test_cfg0_longer_than_the_cap_crosses_resets():
+    w = wl.workload(0)
+    params = wl.make_params(w)
+    T = 120
+    ro, _ = run_gpu(w, FP32, T, params=params)
+    assert int(ro.dones.sum()) >= 2 * w["n_envs"]
+    check_against_oracle(w, ro, params, T, FP32, np.arange(w["n_envs"]))
+
+
+# ---- reduced versions of the larger configs (several tiles and a ragged last tile) -----------
+
+@pytest.mark.parametrize("idx,n_envs,T", [(1, 77, 60), (2, 101, 110), (3, 45, 105), (4, 37, 40)])
+def test_reduced_configs_fp32(idx, n_envs, T):
+    w = wl.workload(idx)
+    params = wl.make_params(w, bias_scale=0.1)
+    ro, _ = run_gpu(w, FP32, T, n_envs=n_envs, params=params)
+    ids = wl.sample_env_ids(n_envs, 6, 6, 6, seed=idx)
+    out = check_against_oracle(w, ro, params, T, FP32, ids)
+    print(idx, out)
+
+
+@pytest.mark.parametrize("idx,n_envs,T", [(1, 333, 60), (2, 300, 110), (3, 200, 105), (4, 150, 40)])
+def test_reduced_configs_bf16(idx, n_envs, T):
+    w = wl.workload(idx)
+    if not _tc_available(w):
+        pytest.skip("bf16 tensor-core path not compiled for this shape")
+    params = wl.make_params(w, bias_scale=0.1)
+    ro, _ = run_gpu(w, BF16, T, n_envs=n_envs, params=params)
+    ids = wl.sample_env_ids(n_envs, 6, 6, 6, seed=idx)
+    out = check_against_oracle(w, ro, params, T, BF16, ids)
+    print(idx, out)
+    # tighter: against the oracle run with bf16-rounded operands
+    ocfg = oracle.make_config(w)
+    acts = ro.actions[:T].cpu().numpy()
+    ref = oracle.rollout(ocfg, w["seed"], params, T, ids, forced_actions=acts[:, ids], want_obs=False,
+                         emulate_bf16=True)
+    lg = ro.logits[:T].cpu().numpy()[:, ids]
+    assert np.max(np.abs(lg - ref.logits) / (1 + np.abs(ref.logits))) < 2e-3
+    v = ro.values[:T + 1].cpu().numpy()[:, ids]
+    assert np.max(np.abs(v - ref.values) / (1 + np.abs(ref.values))) < 2e-3
+
+
+# ---- full-size configs in the launch configuration the benchmark times ------------------------
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_full_size_configs(idx):
+    w = wl.workload(idx)
+    precision = _precision(w) if _tc_available(w) else FP32
+    params = wl.make_params(w)
+    T, E = w["T"], w["n_envs"]
+    ro, _ = run_gpu(w, precision, T, params=params)
+    mlp_ids = wl.sample_env_ids(E, 3, 3, 6, seed=idx)
+    obs_ids = wl.sample_env_ids(E, 64, 64, 128, seed=idx)
+    out = check_against_oracle(w, ro, params, T, precision, mlp_ids, obs_env_ids=obs_ids)
+    print(idx, precision, out)
+
+
+# ---- hand-worked transitions through set_state + forced actions -------------------------------
+
+def test_hand_worked_steps_on_the_gpu():
+    import torch
+
+    w = wl.workload(0)
+    cfg = binding.make_config(w, precision=FP32, max_T=1, n_envs=6)
+    ro = binding.Rollout(cfg)
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    far = [7, 7, 1, 7, 0, 1]
+    # record: a0(r,c,l) a1(r,c,l) f0(r,c,l) f1(r,c,l) step episode total
+    states = np.array([
+        [2, 2, 1, 2, 4, 1, *far, 0, 0, 2],             # head-on to the same cell
+        [2, 2, 1, 2, 3, 1, *far, 0, 0, 2],             # follow into a vacated cell
+        [0, 5, 1, 5, 5, 1, *far, 0, 0, 2],             # wall
+        [3, 2, 1, 2, 3, 2, 3, 3, 3, 6, 6, 2, 0, 0, 5],  # joint load collects level 3 of 5
+        [3, 2, 1, 2, 3, 1, 3, 3, 1, 6, 6, 2, 0, 0, 3],  # collected food still blocks this step
+        [3, 2, 1, 6, 6, 1, *far, 49, 0, 2],            # cap
+    ], dtype=np.int32)
+    acts = np.array([[4, 3], [4, 4], [1, 0], [5, 5], [5, 2], [0, 0]], dtype=np.int32)[None]
+    ro.set_state(states)
+    ro.run_forced(params, 1, torch.from_numpy(acts).cuda())
+    assert ro.status() == 0
+    after = ro.get_state()
+    assert after[0, :6].tolist() == [2, 2, 1, 2, 4, 1]
+    assert after[1, :6].tolist() == [2, 2, 1, 2, 4, 1]
+    assert after[2, :3].tolist() == [0, 5, 1]
+    assert after[3, 8] == 0 and after[3, 11] == 2
+    assert after[4, 8] == 0 and after[4, 3:5].tolist() == [2, 3]
+    rew = ro.rewards[0].cpu().numpy()
+    assert rew[3].tolist() == [np.float32(3) / np.float32(5)] * 2
+    assert rew[4].tolist() == [np.float32(1) / np.float32(3)] * 2
+    assert ro.dones[0].cpu().numpy().tolist() == [0, 0, 0, 0, 0, 1]
+    assert after[5, 12:14].tolist() == [0, 1]  # fresh episode 1
+    fresh = oracle.env_reset(oracle.make_config(w), w["seed"], 5, 1)
+    assert after[5, :2].tolist() == [fresh.agent_r[0], fresh.agent_c[0]]
+
+
+# ---- determinism, continuation, reset ------------------------------------------------------------
+
+def test_two_runs_give_identical_bytes_and_reset_replays():
+    import torch
+
+    w = wl.workload(2)
+    T = 50
+    cfg = binding.make_config(w, precision=FP32, max_T=T, n_envs=95)
+    ro = binding.Rollout(cfg)
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    ro.run(params, T)
+    first = [t.clone() for t in (ro.obs, ro.actions, ro.logp, ro.values, ro.rewards, ro.dones)]
+    ro.reset(w["seed"])
+    ro.run(params, T)
+    for a, b in zip(first, (ro.obs, ro.actions, ro.logp, ro.values, ro.rewards, ro.dones)):
+        assert torch.equal(a, b)
+    assert ro.status() == 0
+
+
+def test_two_calls_continue_like_one():
+    import torch
+
+    w = wl.workload(1)
+    cfg = binding.make_config(w, precision=FP32, max_T=70, n_envs=40)
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    a = binding.Rollout(cfg)
+    a.run(params, 70)
+    b = binding.Rollout(cfg)
+    b.run(params, 30)
+    obs1, act1 = b.obs[:30].clone(), b.actions[:30].clone()
+    b.run(params, 40)
+    assert torch.equal(a.obs[:30], obs1) and torch.equal(a.actions[:30], act1)
+    assert torch.equal(a.obs[30:70], b.obs[:40]) and torch.equal(a.actions[30:70], b.actions[:40])
+    assert torch.equal(a.values[70], b.values[40])
+    assert np.array_equal(a.get_state(), b.get_state())
+
+
+def test_capacity_and_argument_errors():
+    import torch
+
+    w = wl.workload(0)
+    cfg = binding.make_config(w, precision=FP32, max_T=8)
+    ro = binding.Rollout(cfg, with_gae=False)
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    with pytest.raises(binding.MavaError) as e:
+        ro.run(params, 9)
+    assert e.value.code == binding.MAVA_ERR_CAPACITY
+    with pytest.raises(binding.MavaError) as e:
+        ro.gae(0.99, 0.95)  # no run yet and no adv/ret buffers
+    assert e.value.code == binding.MAVA_ERR_INVALID_ARG
+    ro.run(params, 8)
+    assert ro.status() == 0 and ro.launch_count() >= 3
+
+
+# ---- GAE on arbitrary data, odd shapes ------------------------------------------------------------
+
+@pytest.mark.parametrize("idx,n_envs,T", [(0, 16, 1), (0, 5, 13), (2, 47, 37), (4, 33, 64), (1, 300, 128), (3, 9, 250)])
+def test_gae_on_random_trajectories(idx, n_envs, T):
+    import torch
+
+    w = wl.workload(idx)
+    cfg = binding.make_config(w, precision=FP32, max_T=T, n_envs=n_envs)
+    ro = binding.Rollout(cfg)
+    ro.run(torch.from_numpy(wl.make_params(w)).cuda(), T)
+    g = torch.Generator(device="cuda").manual_seed(idx)
+    ro.values.copy_(torch.randn(ro.values.shape, generator=g, device="cuda"))
+    ro.rewards.copy_(torch.rand(ro.rewards.shape, generator=g, device="cuda"))
+    ro.dones.copy_((torch.rand(ro.dones.shape, generator=g, device="cuda") < 0.1).to(torch.uint8))
+    for gamma, lam in [(0.99, 0.95), (1.0, 1.0), (0.9, 0.0)]:
+        ro.gae(gamma, lam)
+        adv, ret = oracle.gae(ro.values.cpu().numpy(), ro.rewards.cpu().numpy(), ro.dones.cpu().numpy(),
+                              float(np.float32(gamma)), float(np.float32(lam)))
+        ga, gr = ro.adv.cpu().numpy(), ro.ret.cpu().numpy()
+        assert np.max(np.abs(ga - adv) / np.maximum(1, np.abs(adv))) <= 1e-5
+        assert np.max(np.abs(gr - ret) / np.maximum(1, np.abs(ret))) <= 1e-5
