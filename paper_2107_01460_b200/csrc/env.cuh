@@ -146,6 +146,42 @@ __device__ __forceinline__ void observe_scatter(const EnvRec *st, int n_rows, in
   }
 }
 
+// Sparse form of the observation of agent `a`: calls sink(j, v) for exactly the elements that can
+// be non-zero (wall cells of a window that crosses the border, entities inside the window, own
+// level, step/cap, the agent's one-hot slot).  Called twice on the same state -- once with the
+// values and once writing zeros -- it maintains an observation row over a zero background.
+template <int N, int F, class Sink>
+__device__ __forceinline__ void observe_sparse(const EnvRec &s, const EnvParams &p, int a, Sink sink) {
+  const int G = p.grid;
+  const int r0 = s.ar[a], c0 = s.ac[a];
+  if (r0 < kViewRadius || r0 >= G - kViewRadius || c0 < kViewRadius || c0 >= G - kViewRadius) {
+#pragma unroll
+    for (int dy = -kViewRadius; dy <= kViewRadius; ++dy) {
+#pragma unroll
+      for (int dx = -kViewRadius; dx <= kViewRadius; ++dx) {
+        const int rr = r0 + dy, cc = c0 + dx;
+        if (rr < 0 || rr >= G || cc < 0 || cc >= G)
+          sink(2 * kPlane + (dy + kViewRadius) * kWindow + (dx + kViewRadius), 1.0f);
+      }
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    const int dy = static_cast<int>(s.ar[k]) - r0, dx = static_cast<int>(s.ac[k]) - c0;
+    if (dy >= -kViewRadius && dy <= kViewRadius && dx >= -kViewRadius && dx <= kViewRadius)
+      sink((dy + kViewRadius) * kWindow + (dx + kViewRadius), static_cast<float>(s.al[k]));
+  }
+#pragma unroll
+  for (int f = 0; f < F; ++f) {
+    const int dy = static_cast<int>(s.fr[f]) - r0, dx = static_cast<int>(s.fc[f]) - c0;
+    if (s.fl[f] > 0 && dy >= -kViewRadius && dy <= kViewRadius && dx >= -kViewRadius && dx <= kViewRadius)
+      sink(kPlane + (dy + kViewRadius) * kWindow + (dx + kViewRadius), static_cast<float>(s.fl[f]));
+  }
+  sink(3 * kPlane, static_cast<float>(s.al[a]));
+  sink(3 * kPlane + 1, __fdiv_rn(static_cast<float>(s.step), static_cast<float>(p.cap)));
+  sink(kObsFixed + a, 1.0f);
+}
+
 // Transition, phase 1 (reads only the start-of-step state).
 //   items [0, n_rows): one agent each -> new position in new_r/new_c.  A move is cancelled when
 //     its target is outside the grid, holds a present food, is another agent's current cell or is
