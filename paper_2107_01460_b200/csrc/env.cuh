@@ -256,3 +256,198 @@ __device__ __forceinline__ void step_apply(EnvRec &s, const EnvParams &p, uint32
 }
 
 }  // namespace mava
+
+// ---------------------------------------------------------------------------------------------
+// Register-resident form of the same environment, for kernels where every agent row has its own
+// thread and the N threads of an environment sit in adjacent lanes of one warp.  Each of those
+// threads keeps a full copy of the environment (entity k packed as row | col << 8 | level << 16;
+// agents first, then food, a food of level 0 is gone) and all of them apply identical integer
+// updates, so the copies never diverge; what one lane decides for its own agent or food reaches
+// the others by warp shuffles and ballots.
+// ---------------------------------------------------------------------------------------------
+namespace mava {
+
+template <int N, int F>
+struct EnvRegs {
+  uint32_t ent[N + F];
+  int32_t step, episode, total;
+};
+
+__device__ __forceinline__ uint32_t pack_entity(int r, int c, int level) {
+  return static_cast<uint32_t>(r) | (static_cast<uint32_t>(c) << 8) | (static_cast<uint32_t>(level) << 16);
+}
+
+template <int N, int F>
+__device__ __forceinline__ void load_env(EnvRegs<N, F> &s, const EnvRec &g) {
+#pragma unroll
+  for (int n = 0; n < N; ++n) s.ent[n] = pack_entity(g.ar[n], g.ac[n], g.al[n]);
+#pragma unroll
+  for (int f = 0; f < F; ++f) s.ent[N + f] = pack_entity(g.fr[f], g.fc[f], g.fl[f]);
+  s.step = g.step; s.episode = g.episode; s.total = g.total;
+}
+
+template <int N, int F>
+__device__ __forceinline__ void store_env(const EnvRegs<N, F> &s, EnvRec &g) {
+#pragma unroll
+  for (int n = 0; n < N; ++n) {
+    g.ar[n] = static_cast<uint8_t>(s.ent[n]); g.ac[n] = static_cast<uint8_t>(s.ent[n] >> 8);
+    g.al[n] = static_cast<uint8_t>(s.ent[n] >> 16);
+  }
+#pragma unroll
+  for (int f = 0; f < F; ++f) {
+    g.fr[f] = static_cast<uint8_t>(s.ent[N + f]); g.fc[f] = static_cast<uint8_t>(s.ent[N + f] >> 8);
+    g.fl[f] = static_cast<uint8_t>(s.ent[N + f] >> 16);
+  }
+  g.step = s.step; g.episode = s.episode; g.total = s.total;
+}
+
+// Same draw order and placement rule as env_reset above.
+template <int N, int F>
+__device__ void reset_env(EnvRegs<N, F> &s, const EnvParams &p, uint32_t env, uint32_t episode) {
+  constexpr int K = N + F;
+  constexpr int NBLK = (2 * K + 3) / 4;
+  uint32_t draws[NBLK * 4];
+#pragma unroll
+  for (int b = 0; b < NBLK; ++b)
+    philox4x32_10(static_cast<uint32_t>(b), env, episode, 0u, p.key_lo, p.key_hi ^ kDomainReset, &draws[4 * b]);
+  int level[K];
+  int level_sum = 0, total = 0;
+#pragma unroll
+  for (int n = 0; n < N; ++n) {
+    level[n] = 1 + static_cast<int>(bounded(draws[n], static_cast<uint32_t>(p.max_level)));
+    level_sum += level[n];
+  }
+#pragma unroll
+  for (int f = 0; f < F; ++f) {
+    level[N + f] = 1 + static_cast<int>(bounded(draws[N + f], static_cast<uint32_t>(level_sum)));
+    total += level[N + f];
+  }
+  const int G = p.grid;
+  int taken[K];
+#pragma unroll
+  for (int k = 0; k < K; ++k) {
+    int cell = static_cast<int>(bounded(draws[K + k], static_cast<uint32_t>(G * G - k)));
+#pragma unroll
+    for (int j = 0; j < K; ++j)
+      if (j < k && taken[j] <= cell) ++cell;
+    const int r = cell / G, c = cell - r * G;
+    s.ent[k] = pack_entity(r, c, level[k]);
+    int carry = cell;
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+      if (j < k) {
+        if (taken[j] > carry) { const int tmp = taken[j]; taken[j] = carry; carry = tmp; }
+      } else if (j == k) {
+        taken[j] = carry;
+      }
+    }
+  }
+  s.step = 0;
+  s.episode = static_cast<int32_t>(episode);
+  s.total = total;
+}
+
+// Non-zero observation entries of agent `ag` (see observe_sparse for the element layout).
+template <int N, int F, class Sink>
+__device__ __forceinline__ void observe_env(const EnvRegs<N, F> &s, const EnvParams &p, int ag, Sink sink) {
+  uint32_t me = s.ent[0];
+#pragma unroll
+  for (int m = 1; m < N; ++m) me = (ag == m) ? s.ent[m] : me;
+  const int G = p.grid;
+  const int r0 = me & 0xFF, c0 = (me >> 8) & 0xFF;
+  bool row_out[kWindow], col_out[kWindow];
+#pragma unroll
+  for (int d = 0; d < kWindow; ++d) {
+    row_out[d] = (r0 + d - kViewRadius < 0) || (r0 + d - kViewRadius >= G);
+    col_out[d] = (c0 + d - kViewRadius < 0) || (c0 + d - kViewRadius >= G);
+  }
+#pragma unroll
+  for (int dy = 0; dy < kWindow; ++dy)
+#pragma unroll
+    for (int dx = 0; dx < kWindow; ++dx)
+      if (row_out[dy] || col_out[dx]) sink(2 * kPlane + dy * kWindow + dx, 1.0f);
+#pragma unroll
+  for (int k = 0; k < N + F; ++k) {
+    const uint32_t e = s.ent[k];
+    const int dy = static_cast<int>(e & 0xFF) - r0 + kViewRadius, dx = static_cast<int>((e >> 8) & 0xFF) - c0 + kViewRadius;
+    const int lvl = static_cast<int>(e >> 16);
+    if (lvl > 0 && dy >= 0 && dy < kWindow && dx >= 0 && dx < kWindow)
+      sink((k < N ? 0 : kPlane) + dy * kWindow + dx, static_cast<float>(lvl));
+  }
+  sink(3 * kPlane, static_cast<float>(me >> 16));
+  sink(3 * kPlane + 1, __fdiv_rn(static_cast<float>(s.step), static_cast<float>(p.cap)));
+  sink(kObsFixed + ag, 1.0f);
+}
+
+// One transition of the environment whose N agent threads occupy lanes [base, base + N) of this
+// warp; every lane of the warp must call it (lanes without an environment pass active = false
+// and base = their own lane).  `action` is this lane's action.  Same rules as step_decide /
+// step_apply; returns the shared reward and the done flag, and has already started the next
+// episode when done.
+template <int N, int F>
+__device__ __forceinline__ void step_env_warp(EnvRegs<N, F> &s, const EnvParams &p, uint32_t env, int ag, int base,
+                                              bool active, int action, float &reward, bool &done) {
+  constexpr unsigned kFull = 0xFFFFFFFFu;
+  const int G = p.grid;
+  int act[N];
+  uint32_t target[N];  // 0xFFFF: not moving
+#pragma unroll
+  for (int m = 0; m < N; ++m) {
+    act[m] = __shfl_sync(kFull, action, base + m);
+    const int r = s.ent[m] & 0xFF, c = (s.ent[m] >> 8) & 0xFF;
+    const int tr = r + (act[m] == 2) - (act[m] == 1), tc = c + (act[m] == 4) - (act[m] == 3);
+    const bool moving = act[m] >= 1 && act[m] <= 4;
+    const bool inside = tr >= 0 && tr < G && tc >= 0 && tc < G;
+    target[m] = moving ? (inside ? (static_cast<uint32_t>(tr) | (static_cast<uint32_t>(tc) << 8)) : 0xFFFEu) : 0xFFFFu;
+  }
+  // this lane's own agent
+  uint32_t my_target = target[0], my_pos = s.ent[0] & 0xFFFFu;
+#pragma unroll
+  for (int m = 1; m < N; ++m) {
+    my_target = (ag == m) ? target[m] : my_target;
+    my_pos = (ag == m) ? (s.ent[m] & 0xFFFFu) : my_pos;
+  }
+  bool ok = my_target < 0xFFFEu;  // moving and inside the grid
+#pragma unroll
+  for (int f = 0; f < F; ++f) ok = ok && !((s.ent[N + f] >> 16) != 0 && (s.ent[N + f] & 0xFFFFu) == my_target);
+#pragma unroll
+  for (int m = 0; m < N; ++m)
+    ok = ok && (m == ag || ((s.ent[m] & 0xFFFFu) != my_target && target[m] != my_target));
+  const uint32_t my_new = ok ? my_target : my_pos;
+  // foods: lane `ag` decides foods ag, ag + N, ...
+  uint32_t collected_mask = 0;  // bit f: food f collected
+#pragma unroll
+  for (int round = 0; round * N < F; ++round) {
+    uint32_t fe = 0;  // level 0: nothing to decide
+#pragma unroll
+    for (int j = 0; j < N; ++j)
+      if (round * N + j < F) fe = (ag == j) ? s.ent[N + round * N + j] : fe;
+    const int fr = fe & 0xFF, fc = (fe >> 8) & 0xFF, fl = static_cast<int>(fe >> 16);
+    int load = 0;
+#pragma unroll
+    for (int m = 0; m < N; ++m) {
+      const int dist = abs(static_cast<int>(s.ent[m] & 0xFF) - fr) + abs(static_cast<int>((s.ent[m] >> 8) & 0xFF) - fc);
+      load += (act[m] == 5 && dist == 1) ? static_cast<int>(s.ent[m] >> 16) : 0;
+    }
+    const uint32_t bal = __ballot_sync(kFull, fl > 0 && load >= fl);
+    collected_mask |= ((bal >> base) & ((1u << N) - 1u)) << (round * N);
+  }
+  // apply: every lane updates its copy identically
+  int gained = 0, left = 0;
+#pragma unroll
+  for (int m = 0; m < N; ++m) {
+    const uint32_t np = __shfl_sync(kFull, my_new, base + m);
+    s.ent[m] = (s.ent[m] & 0xFFFF0000u) | np;
+  }
+#pragma unroll
+  for (int f = 0; f < F; ++f) {
+    if ((collected_mask >> f) & 1u) { gained += static_cast<int>(s.ent[N + f] >> 16); s.ent[N + f] &= 0xFFFFu; }
+    left += (s.ent[N + f] >> 16) != 0;
+  }
+  reward = gained > 0 ? __fdiv_rn(static_cast<float>(gained), static_cast<float>(s.total)) : 0.0f;
+  s.step += 1;
+  done = (left == 0) || (s.step >= p.cap);
+  if (done && active) reset_env<N, F>(s, p, env, static_cast<uint32_t>(s.episode) + 1u);
+}
+
+}  // namespace mava

@@ -128,12 +128,23 @@ template <int N, int H>
 struct TcShape {
   static constexpr int D = kObsFixed + N;
   static constexpr int K1 = (D + 15) / 16 * 16;               // layer-1 K padded to the MMA's K step
-  static constexpr int EPT_MAX = kTileRows / N;                // environments per tile, at most
-  static constexpr uint32_t W1_BYTES = H * K1 * 2, W2_BYTES = H * H * 2, WH_BYTES = kHeadRows * H * 2;
-  static constexpr uint32_t BIAS_FLOATS = 2 * H + kHeadRows;
-  static constexpr uint32_t IMAGE_BYTES = W1_BYTES + W2_BYTES + WH_BYTES + BIAS_FLOATS * 4;
+  static constexpr int EPW = 32 / N;                           // environments per warp (lanes EPW*N.. idle)
+  static constexpr int EPT_MAX = 4 * EPW;                      // environments per tile, at most
+  // Weight image: W1 | W2 | heads | bias tiles of the three layers | the constant "ones" A tile.
+  // A bias tile is an N x 16 operand whose column 0 holds bf16(b) and column 1 the bf16 of the
+  // remainder; multiplied by the ones tile (columns 0 and 1 equal to 1) it seeds the accumulator
+  // with the bias to about 2^-17 relative, so the epilogues need no bias arithmetic.
+  static constexpr uint32_t W1_OFF = 0, W1_BYTES = H * K1 * 2;
+  static constexpr uint32_t W2_OFF = W1_OFF + W1_BYTES, W2_BYTES = H * H * 2;
+  static constexpr uint32_t WH_OFF = W2_OFF + W2_BYTES, WH_BYTES = kHeadRows * H * 2;
+  static constexpr uint32_t B1_OFF = WH_OFF + WH_BYTES, BT_BYTES = H * 16 * 2;
+  static constexpr uint32_t B2_OFF = B1_OFF + BT_BYTES;
+  static constexpr uint32_t BH_OFF = B2_OFF + BT_BYTES, BH_BYTES = kHeadRows * 16 * 2;
+  static constexpr uint32_t ONES_OFF = BH_OFF + BH_BYTES, ONES_BYTES = kTileRows * 16 * 2;
+  static constexpr uint32_t IMAGE_BYTES = ONES_OFF + ONES_BYTES;
   static constexpr uint32_t STAGE_BYTES = (kTileRows * D * 4 + 15) / 16 * 16;
-  static constexpr uint32_t AH_BYTES = kTileRows * (K1 > H ? K1 : H) * 2;
+  static constexpr uint32_t A_BYTES = kTileRows * K1 * 2;
+  static constexpr uint32_t X_BYTES = STAGE_BYTES > kTileRows * H * 2 ? STAGE_BYTES : kTileRows * H * 2;
   static constexpr int ACC_COLS = H;                            // layer accumulators (reused)
   static constexpr int GROUP_COLS = H + 32;                     // + the heads accumulator
   static constexpr int TMEM_COLS = kGroups * GROUP_COLS <= 256 ? 256 : 512;
@@ -142,18 +153,17 @@ struct TcShape {
 template <int N, int F, int H>
 struct TcGroupSmem {
   using S = TcShape<N, H>;
-  alignas(16) unsigned char stage[S::STAGE_BYTES];  // fp32 observation block, global layout
-  alignas(128) unsigned char ah[S::AH_BYTES];       // A operand: observations, then h1, then h2
-  EnvRec st[S::EPT_MAX];
-  int act[kTileRows];
-  uint8_t new_r[kTileRows], new_c[kTileRows], collected[S::EPT_MAX * F];
+  // fp32 observation block in the global layout while a step starts; the hidden activations
+  // (A operand of layer 2 and of the heads) for the rest of the step.
+  alignas(128) unsigned char x[S::X_BYTES];
+  alignas(128) unsigned char a[S::A_BYTES];  // bf16 observations, A operand of layer 1
   alignas(8) uint64_t mma_bar;
 };
 
 template <int N, int F, int H>
 struct TcSmem {
   using S = TcShape<N, H>;
-  alignas(128) unsigned char weights[S::IMAGE_BYTES];  // W1 | W2 | heads | b1 b2 bh (fp32)
+  alignas(128) unsigned char weights[S::IMAGE_BYTES];
   TcGroupSmem<N, F, H> grp[kGroups];
   alignas(8) uint64_t load_bar;
   uint32_t tmem_base;
@@ -170,57 +180,107 @@ template <int N, int H>
 __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, ParamLayout L) {
   using S = TcShape<N, H>;
   constexpr int D = S::D, K1 = S::K1;
-  __nv_bfloat16 *w1 = reinterpret_cast<__nv_bfloat16 *>(image);
-  __nv_bfloat16 *w2 = reinterpret_cast<__nv_bfloat16 *>(image + S::W1_BYTES);
-  __nv_bfloat16 *wh = reinterpret_cast<__nv_bfloat16 *>(image + S::W1_BYTES + S::W2_BYTES);
-  float *bias = reinterpret_cast<float *>(image + S::W1_BYTES + S::W2_BYTES + S::WH_BYTES);
+  auto at = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(image + off); };
   const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   for (int i = tid; i < H * K1; i += nth) {
     const int n = i / K1, k = i - n * K1;
-    w1[canon_offset(n, k, K1) / 2] = __float2bfloat16_rn(k < D ? params[L.W1 + static_cast<size_t>(n) * D + k] : 0.0f);
+    at(S::W1_OFF)[canon_offset(n, k, K1) / 2] =
+        __float2bfloat16_rn(k < D ? params[L.W1 + static_cast<size_t>(n) * D + k] : 0.0f);
   }
   for (int i = tid; i < H * H; i += nth) {
     const int n = i / H, k = i - n * H;
-    w2[canon_offset(n, k, H) / 2] = __float2bfloat16_rn(params[L.W2 + static_cast<size_t>(n) * H + k]);
+    at(S::W2_OFF)[canon_offset(n, k, H) / 2] = __float2bfloat16_rn(params[L.W2 + static_cast<size_t>(n) * H + k]);
   }
   for (int i = tid; i < kHeadRows * H; i += nth) {
     const int n = i / H, k = i - n * H;
     float v = 0.0f;
     if (n < kActions) v = params[L.Wa + static_cast<size_t>(n) * H + k];
     else if (n == kActions) v = params[L.Wv + k];
-    wh[canon_offset(n, k, H) / 2] = __float2bfloat16_rn(v);
+    at(S::WH_OFF)[canon_offset(n, k, H) / 2] = __float2bfloat16_rn(v);
   }
-  for (int i = tid; i < static_cast<int>(S::BIAS_FLOATS); i += nth) {
-    float v = 0.0f;
-    if (i < H) v = params[L.b1 + i];
-    else if (i < 2 * H) v = params[L.b2 + i - H];
-    else if (i - 2 * H < kActions) v = params[L.ba + i - 2 * H];
-    else if (i - 2 * H == kActions) v = params[L.bv];
-    bias[i] = v;
+  // bias tiles (hi, lo, then zeros) and the ones tile
+  for (int i = tid; i < (2 * H + kHeadRows) * 16; i += nth) {
+    const int r = i / 16, k = i - r * 16;
+    float b;
+    uint32_t off;
+    int n;
+    if (r < H) { b = params[L.b1 + r]; off = S::B1_OFF; n = r; }
+    else if (r < 2 * H) { b = params[L.b2 + r - H]; off = S::B2_OFF; n = r - H; }
+    else {
+      n = r - 2 * H;
+      off = S::BH_OFF;
+      b = n < kActions ? params[L.ba + n] : (n == kActions ? params[L.bv] : 0.0f);
+    }
+    const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+    at(off)[canon_offset(n, k, 16) / 2] = k == 0 ? hi : (k == 1 ? lo : __float2bfloat16_rn(0.0f));
+  }
+  for (int i = tid; i < kTileRows * 16; i += nth) {
+    const int r = i / 16, k = i - r * 16;
+    at(S::ONES_OFF)[canon_offset(r, k, 16) / 2] = __float2bfloat16_rn(k < 2 ? 1.0f : 0.0f);
   }
 }
 
 // ---- the rollout kernel ------------------------------------------------------------------------
-// Epilogue of a hidden layer: thread `row` reads its accumulator row from tensor memory, adds the
-// bias, applies ReLU, rounds to bf16 and stores the row as the next A operand (K = H).
+// 32 lanes x 32 bit, 32 consecutive columns (no wait: the caller waits once per batch of loads).
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,"
+      "%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// max(x, 0) of two fp32 values rounded to bf16 and packed (lo in the low half).
+__device__ __forceinline__ uint32_t relu_pack_bf16(uint32_t lo_bits, uint32_t hi_bits) {
+  uint32_t d;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(hi_bits)), "f"(__uint_as_float(lo_bits)));
+  return d;
+}
+
+// Epilogue of a hidden layer: thread `row` reads its accumulator row (bias already inside) from
+// tensor memory, applies ReLU, rounds to bf16 and stores the row as the next A operand (K = H).
+// The load of the next 32 columns is in flight while the current 32 are converted.
 template <int H>
-__device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, const float *bias, unsigned char *ah, int row) {
-#pragma unroll 1
-  for (int c0 = 0; c0 < H; c0 += 16) {
-    float v[16];
-    tmem_ld16(acc_taddr + static_cast<uint32_t>(c0), v);
-    uint32_t packed[8];
+__device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, unsigned char *hbuf, int row) {
+  static_assert(H % 64 == 0, "two 32-column batches per iteration");
+  uint32_t ra[32], rb[32];
+  tmem_ld32_nowait(acc_taddr, ra);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float a = fmaxf(v[2 * i] + bias[c0 + 2 * i], 0.0f);
-      const float b = fmaxf(v[2 * i + 1] + bias[c0 + 2 * i + 1], 0.0f);
-      packed[i] = pack_bf16(a, b);
-    }
-    uint4 *dst0 = reinterpret_cast<uint4 *>(ah + canon_offset(row, c0, H));
-    uint4 *dst1 = reinterpret_cast<uint4 *>(ah + canon_offset(row, c0 + 8, H));
-    *dst0 = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-    *dst1 = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+  for (int c0 = 0; c0 < H; c0 += 64) {
+    tmem_ld_wait();
+    tmem_ld32_nowait(acc_taddr + static_cast<uint32_t>(c0 + 32), rb);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 8 * q, H)) =
+          make_uint4(relu_pack_bf16(ra[8 * q], ra[8 * q + 1]), relu_pack_bf16(ra[8 * q + 2], ra[8 * q + 3]),
+                     relu_pack_bf16(ra[8 * q + 4], ra[8 * q + 5]), relu_pack_bf16(ra[8 * q + 6], ra[8 * q + 7]));
+    tmem_ld_wait();
+    if (c0 + 64 < H) tmem_ld32_nowait(acc_taddr + static_cast<uint32_t>(c0 + 64), ra);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 32 + 8 * q, H)) =
+          make_uint4(relu_pack_bf16(rb[8 * q], rb[8 * q + 1]), relu_pack_bf16(rb[8 * q + 2], rb[8 * q + 3]),
+                     relu_pack_bf16(rb[8 * q + 4], rb[8 * q + 5]), relu_pack_bf16(rb[8 * q + 6], rb[8 * q + 7]));
   }
+}
+
+// One dense layer on the tensor core, issued by a single thread: the accumulator is seeded with
+// the bias (ones tile x bias tile, K = 16) and then accumulates K / 16 steps of A x W^T.
+template <int K, int NOUT>
+__device__ __forceinline__ void issue_layer(uint32_t d_tmem, uint32_t a_addr, uint32_t w_addr, uint32_t ones_addr,
+                                            uint32_t bias_addr, uint32_t bar) {
+  constexpr uint32_t idesc = instr_desc(kTileRows, NOUT);
+  mma_bf16(d_tmem, smem_desc(ones_addr, 128, 256), smem_desc(bias_addr, 128, 256), idesc, 0);
+#pragma unroll
+  for (int k = 0; k < K / 16; ++k)
+    mma_bf16(d_tmem, smem_desc(a_addr + k * 256, 128, K * 16), smem_desc(w_addr + k * 256, 128, K * 16), idesc, 1);
+  mma_commit(bar);
 }
 
 template <int N, int F, int H>
@@ -248,11 +308,11 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  {  // zero the observation block and the A operand once (the block keeps a zero background)
-    uint4 *z = reinterpret_cast<uint4 *>(gs.stage);
-    for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
-    z = reinterpret_cast<uint4 *>(gs.ah);
-    for (int i = row; i < static_cast<int>(S::AH_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
+  {  // zero the observation block and the A operand once
+    uint4 *z = reinterpret_cast<uint4 *>(gs.x);
+    for (int i = row; i < static_cast<int>(S::X_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
+    z = reinterpret_cast<uint4 *>(gs.a);
+    for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
   }
   tc_fence_before();
   __syncthreads();
@@ -274,32 +334,52 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const uint32_t acc_col = tmem_base + static_cast<uint32_t>(g * S::GROUP_COLS);
   const uint32_t head_col = acc_col + static_cast<uint32_t>(S::ACC_COLS);
   const uint32_t lane_off = static_cast<uint32_t>((warp % 4) * 32) << 16;  // this warp's TMEM lanes
-  const uint32_t w1_addr = smem_u32(sm.weights), w2_addr = w1_addr + S::W1_BYTES, wh_addr = w2_addr + S::W2_BYTES;
-  const float *bias = reinterpret_cast<const float *>(sm.weights + S::W1_BYTES + S::W2_BYTES + S::WH_BYTES);
-  const uint32_t ah_addr = smem_u32(gs.ah);
+  const uint32_t w_addr = smem_u32(sm.weights);
+  const uint32_t a_addr = smem_u32(gs.a), x_addr = smem_u32(gs.x);
   const uint32_t bar = smem_u32(&gs.mma_bar);
-  float *stage = reinterpret_cast<float *>(gs.stage);
+  float *stage = reinterpret_cast<float *>(gs.x);
   uint32_t phase = 0;
   const size_t M = static_cast<size_t>(a.env.n_envs) * N;
 
   // ---- tiles of this group ---------------------------------------------------------------------
+  const int lane = tid & 31;
+  const int le = ((tid % kGroupThreads) / 32) * S::EPW + lane / N;  // local environment of this lane
+  const int ag = lane % N;                                         // its agent
+  const int crow = le * N + ag;                                    // compact row inside the tile's block
   for (int tile = blockIdx.x * kGroups + g; tile < n_tiles && !timed_out; tile += gridDim.x * kGroups) {
     const int e0 = tile * ept;
     const int n_env = min(ept, a.env.n_envs - e0);
     const int n_rows = n_env * N;
-    for (int i = row; i < n_env * static_cast<int>(sizeof(EnvRec) / 4); i += kGroupThreads)
-      reinterpret_cast<uint32_t *>(gs.st)[i] = reinterpret_cast<const uint32_t *>(a.state + e0)[i];
-    group_sync(g);
-    const int le = row / N, ag = row - le * N;  // this thread's environment and agent (if row < n_rows)
+    const bool active = lane < S::EPW * N && le < n_env;
+    const int base = active ? lane - ag : lane;
+    const uint32_t env_id = static_cast<uint32_t>(a.env.first_env + e0 + le);
+    EnvRegs<N, F> env;
+    if (active) {
+      load_env(env, a.state[e0 + le]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < N + F; ++k) env.ent[k] = 0;
+      env.step = 0; env.episode = 0; env.total = 1;
+    }
 
     for (int t = 0; t <= a.T; ++t) {
       const bool last = (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
-      // 1. non-zero observation entries over the zero background
-      if (row < n_rows)
-        observe_sparse<N, F>(gs.st[le], a.env, ag, [&](int j, float v) { stage[row * D + j] = v; });
+      // 1. non-zero observation entries: fp32 into the zeroed block, bf16 into the zeroed A tile
+      if (active)
+        observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
+          stage[crow * D + j] = v;
+          *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, j, K1)) = __float2bfloat16_rn(v);
+        });
+      fence_async_smem();
+      tc_fence_before();
       group_sync(g);
-      // 2a. observation block -> obs[t] (one contiguous block of the time-major array)
+      // 2. layer 1 runs while the block goes to obs[t] (one contiguous piece of the time-major
+      //    array) and the uniform of this step's action draw is computed
+      if (row == 0) {
+        tc_fence_after();
+        issue_layer<K1, H>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF, w_addr + S::B1_OFF, bar);
+      }
       if (!last) {
         float *dst = a.buf.obs + row0 * D;
         const int count = n_rows * D;
@@ -310,85 +390,57 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
           for (int i = row; i < count; i += kGroupThreads) dst[i] = stage[i];
         }
       }
-      // 2b. the same rows as the bf16 A operand of layer 1 (K padded with zeros)
-      if (row < n_rows) {
-#pragma unroll
-        for (int kc = 0; kc < K1 / 8; ++kc) {
-          float x[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) x[i] = (kc * 8 + i < D) ? stage[row * D + kc * 8 + i] : 0.0f;
-          *reinterpret_cast<uint4 *>(gs.ah + canon_offset(row, kc * 8, K1)) =
-              make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
-        }
-      }
-      fence_async_smem();
-      tc_fence_before();
-      group_sync(g);
-      // 3. layer 1; meanwhile the other threads restore the zero background
-      if (row == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < K1 / 16; ++k)
-          mma_bf16(acc_col, smem_desc(ah_addr + k * 256, 128, K1 * 16), smem_desc(w1_addr + k * 256, 128, K1 * 16),
-                   instr_desc(kTileRows, H), k > 0);
-        mma_commit(bar);
-      }
-      if (row < n_rows) observe_sparse<N, F>(gs.st[le], a.env, ag, [&](int j, float) { stage[row * D + j] = 0.0f; });
+      float u = 0.0f;
+      if (active && !last) u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag));
+      group_sync(g);  // every read of the block is done before the epilogue reuses its memory
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       tc_fence_after();
-      hidden_epilogue<H>(acc_col + lane_off, bias, gs.ah, row);
+      hidden_epilogue<H>(acc_col + lane_off, gs.x, row);
+      for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads)  // layer 1 is done with A
+        reinterpret_cast<uint4 *>(gs.a)[i] = make_uint4(0, 0, 0, 0);
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
-      // 4. layer 2
+      // 3. layer 2
       if (row == 0) {
         tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < H / 16; ++k)
-          mma_bf16(acc_col, smem_desc(ah_addr + k * 256, 128, H * 16), smem_desc(w2_addr + k * 256, 128, H * 16),
-                   instr_desc(kTileRows, H), k > 0);
-        mma_commit(bar);
+        issue_layer<H, H>(acc_col, x_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       tc_fence_after();
-      hidden_epilogue<H>(acc_col + lane_off, bias + H, gs.ah, row);
+      hidden_epilogue<H>(acc_col + lane_off, gs.x, row);
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
-      // 5. heads: six logits and the value, N padded to 16
+      // 4. heads: six logits and the value, N padded to 16
       if (row == 0) {
         tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < H / 16; ++k)
-          mma_bf16(head_col, smem_desc(ah_addr + k * 256, 128, H * 16), smem_desc(wh_addr + k * 256, 128, H * 16),
-                   instr_desc(kTileRows, kHeadRows), k > 0);
-        mma_commit(bar);
+        issue_layer<H, kHeadRows>(head_col, x_addr, w_addr + S::WH_OFF, w_addr + S::ONES_OFF, w_addr + S::BH_OFF, bar);
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       tc_fence_after();
+      int action = 0;
       {
         float hv[16];
         tmem_ld16(head_col + lane_off, hv);
-        if (row < n_rows) {
-          const float *bh = bias + 2 * H;
-          a.buf.values[row0 + row] = hv[kActions] + bh[kActions];
+        // the hidden activations are dead: zero the observation block for the next step
+        for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads)
+          reinterpret_cast<uint4 *>(gs.x)[i] = make_uint4(0, 0, 0, 0);
+        if (active) {
+          a.buf.values[row0 + crow] = hv[kActions];
           if (!last) {
-            float l[kActions], e[kActions];
+            float e[kActions];
+            float m = hv[0];
 #pragma unroll
-            for (int k = 0; k < kActions; ++k) l[k] = hv[k] + bh[k];
-            float m = l[0];
-#pragma unroll
-            for (int k = 1; k < kActions; ++k) m = fmaxf(m, l[k]);
+            for (int k = 1; k < kActions; ++k) m = fmaxf(m, hv[k]);
             float sum = 0.0f;
 #pragma unroll
-            for (int k = 0; k < kActions; ++k) { e[k] = expf(l[k] - m); sum += e[k]; }
-            const float u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t),
-                                           static_cast<uint32_t>(a.env.first_env + e0 + le), static_cast<uint32_t>(ag));
+            for (int k = 0; k < kActions; ++k) { e[k] = __expf(hv[k] - m); sum += e[k]; }
             const float target = u * sum;
-            int action = kActions - 1;
+            action = kActions - 1;
             float cdf = 0.0f;
             bool found = false;
 #pragma unroll
@@ -397,18 +449,17 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
               if (!found && target < cdf) { action = k; found = true; }
             }
             if (a.forced) {
-              action = a.forced[row0 + row];
+              action = a.forced[row0 + crow];
               if (action < 0 || action >= kActions) action = 0;
             }
-            float la = l[0];
+            float la = hv[0];
 #pragma unroll
-            for (int k = 1; k < kActions; ++k) la = (action == k) ? l[k] : la;
-            gs.act[row] = action;
-            a.buf.actions[row0 + row] = action;
-            a.buf.logp[row0 + row] = la - m - logf(sum);
+            for (int k = 1; k < kActions; ++k) la = (action == k) ? hv[k] : la;
+            a.buf.actions[row0 + crow] = action;
+            a.buf.logp[row0 + crow] = la - m - __logf(sum);
             if (a.write_logits) {
 #pragma unroll
-              for (int k = 0; k < kActions; ++k) a.buf.logits[(row0 + row) * kActions + k] = l[k];
+              for (int k = 0; k < kActions; ++k) a.buf.logits[(row0 + crow) * kActions + k] = hv[k];
             }
           }
         }
@@ -416,23 +467,16 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       tc_fence_before();
       if (group_any(g, timed_out)) { timed_out = true; break; }
       if (last) break;
-      // 6. transition and auto-reset
-      step_decide<N, F>(gs.st, a.env, gs.act, n_env, gs.new_r, gs.new_c, gs.collected, row, kGroupThreads);
-      group_sync(g);
-      if (row < n_env) {
-        float reward;
-        bool done;
-        step_apply<N, F>(gs.st[row], a.env, static_cast<uint32_t>(a.env.first_env + e0 + row), gs.new_r, gs.new_c,
-                         gs.collected, row, reward, done);
-        for (int n = 0; n < N; ++n) a.buf.rewards[row0 + row * N + n] = reward;
-        a.buf.dones[static_cast<size_t>(t) * a.env.n_envs + e0 + row] = done ? 1 : 0;
+      // 5. transition and auto-reset, inside the warp
+      float reward;
+      bool done;
+      step_env_warp<N, F>(env, a.env, env_id, ag, base, active, action, reward, done);
+      if (active) {
+        a.buf.rewards[row0 + crow] = reward;
+        if (ag == 0) a.buf.dones[static_cast<size_t>(t) * a.env.n_envs + e0 + le] = done ? 1 : 0;
       }
-      group_sync(g);
     }
-    if (!timed_out)
-      for (int i = row; i < n_env * static_cast<int>(sizeof(EnvRec) / 4); i += kGroupThreads)
-        reinterpret_cast<uint32_t *>(a.state + e0)[i] = reinterpret_cast<const uint32_t *>(gs.st)[i];
-    group_sync(g);
+    if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
 
