@@ -51,6 +51,8 @@ extern "C" {
 #define MAVA_PRECISION_BF16 1 /* bf16 operands, fp32 accumulation on the tcgen05 tensor cores      */
 
 #define MAVA_FLAG_WRITE_LOGITS 1 /* also write the six logits of every row to buffers.logits       */
+#define MAVA_FLAG_HIDDEN_IN_TMEM 2 /* bf16 path, H <= 128: keep hidden activations in tensor memory
+                                      (the layout H = 256 always uses); results are identical     */
 
 typedef struct mava_rollout mava_rollout_t; /* opaque, owned by the library */
 

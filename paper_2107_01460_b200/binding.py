@@ -21,6 +21,7 @@ MAVA_NET_CENTRAL_CRITIC = 1
 MAVA_PRECISION_FP32 = 0
 MAVA_PRECISION_BF16 = 1
 MAVA_FLAG_WRITE_LOGITS = 1
+MAVA_FLAG_HIDDEN_IN_TMEM = 2
 N_ACTIONS = 6
 
 EXPORTS = [

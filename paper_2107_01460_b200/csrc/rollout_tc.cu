@@ -1,19 +1,26 @@
 // bf16 tensor-core rollout for sm_100a: tcgen05.mma with fp32 accumulators in tensor memory.
 //
 // One persistent CTA per SM keeps the bf16 weights resident in shared memory (loaded once with
-// bulk async copies, in the canonical K-major core-matrix layout the MMA reads) and runs
-// kGroups independent groups of 128 threads.  A group owns one tile of environments (up to 128
-// agent rows = the M of the MMA) for all T steps, then takes its next tile.  Per step a group
-//   1. writes the non-zero entries of its observation rows over a zero background (fp32),
-//   2. copies that block to the time-major obs array and re-packs it as the bf16 A operand,
-//   3. runs layer 1, layer 2 and the heads as three MMAs (thread 0 issues; completion arrives on
-//      an mbarrier), each followed by an epilogue out of tensor memory: thread r owns row r
-//      (bias, ReLU, bf16, store as the next A operand; for the heads: softmax, Philox draw,
+// bulk async copies, in the canonical K-major core-matrix layout the MMA reads) and runs one or
+// two independent groups of 128 threads.  A group owns one tile of environments (up to 128
+// agent rows = the M of the MMA; thread r owns row r and tensor-memory lane r) for all T steps,
+// then takes its next tile.  The environment lives in registers (env.cuh).  Per step a group
+//   1. writes the non-zero entries of its observation rows into a zeroed bf16 A tile,
+//   2. starts layer 1 and, while it runs, sends the observation block to the time-major obs
+//      array and draws the Philox uniform of the step,
+//   3. runs layer 2 and the heads, each MMA batch issued by one thread and completing on an
+//      mbarrier; the epilogues read the accumulators out of tensor memory (ReLU, bf16) and hand
+//      the row back as the next A operand; the heads' epilogue is the sampler (softmax,
 //      inverse-CDF action, log-prob),
-//   4. applies the transition and auto-reset.
-// Groups never wait for one another, so while one group sits in an MMA or a tensor-memory
-// round trip the other fills the SM.  Every wait on an mbarrier is bounded: when it runs out
-// the group records kStatusTimeout, stops stepping and falls through to the common exit.
+//   4. applies the transition and auto-reset with warp shuffles and ballots.
+// Two layouts of the per-step data are compiled:
+//   TM = false (H <= 128): the fp32 observation block is staged in shared memory in the global
+//     layout (one vectorised contiguous copy) and the hidden activations go back to shared memory;
+//   TM = true (H = 256, where the weights leave no room): the hidden activations stay in tensor
+//     memory as the A operand of the next MMA and the observation block is expanded from the
+//     bf16 A tile on its way out.
+// Groups never wait for one another.  Every wait on an mbarrier is bounded: when it runs out the
+// group records kStatusTimeout, stops stepping and falls through to the common exit.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -23,9 +30,7 @@
 namespace mava {
 namespace {
 
-constexpr int kGroups = 2;
 constexpr int kGroupThreads = 128;
-constexpr int kTcThreads = kGroups * kGroupThreads;
 constexpr int kTileRows = 128;       // M of every MMA
 constexpr int kHeadRows = 16;        // heads padded to the smallest N the MMA takes at M = 128
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -124,47 +129,58 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // ---- shapes ------------------------------------------------------------------------------------
-template <int N, int H>
+template <int N, int H, bool TM>
 struct TcShape {
   static constexpr int D = kObsFixed + N;
   static constexpr int K1 = (D + 15) / 16 * 16;               // layer-1 K padded to the MMA's K step
   static constexpr int EPW = 32 / N;                           // environments per warp (lanes EPW*N.. idle)
+  static constexpr int RPW = EPW * N;                          // agent rows per warp
   static constexpr int EPT_MAX = 4 * EPW;                      // environments per tile, at most
-  // Weight image: W1 | W2 | heads | bias tiles of the three layers | the constant "ones" A tile.
-  // A bias tile is an N x 16 operand whose column 0 holds bf16(b) and column 1 the bf16 of the
-  // remainder; multiplied by the ones tile (columns 0 and 1 equal to 1) it seeds the accumulator
-  // with the bias to about 2^-17 relative, so the epilogues need no bias arithmetic.
+  // With two spare K columns the layer-1 bias rides in W1 (A columns D, D+1 are set to 1).
+  static constexpr bool FOLD1 = (K1 - D >= 2);
+  // Weight image: W1 | W2 | heads | bias tiles | the constant "ones" A tile.  A bias tile is an
+  // N x 16 operand whose column 0 holds bf16(b) and column 1 the bf16 of the remainder; multiplied
+  // by the ones tile (columns 0 and 1 equal to 1) it seeds the accumulator with the bias to about
+  // 2^-17 relative, so the epilogues need no bias arithmetic.
   static constexpr uint32_t W1_OFF = 0, W1_BYTES = H * K1 * 2;
   static constexpr uint32_t W2_OFF = W1_OFF + W1_BYTES, W2_BYTES = H * H * 2;
   static constexpr uint32_t WH_OFF = W2_OFF + W2_BYTES, WH_BYTES = kHeadRows * H * 2;
-  static constexpr uint32_t B1_OFF = WH_OFF + WH_BYTES, BT_BYTES = H * 16 * 2;
-  static constexpr uint32_t B2_OFF = B1_OFF + BT_BYTES;
+  static constexpr uint32_t BT_BYTES = H * 16 * 2;
+  static constexpr uint32_t B1_OFF = WH_OFF + WH_BYTES;
+  static constexpr uint32_t B2_OFF = B1_OFF + (FOLD1 ? 0 : BT_BYTES);
   static constexpr uint32_t BH_OFF = B2_OFF + BT_BYTES, BH_BYTES = kHeadRows * 16 * 2;
   static constexpr uint32_t ONES_OFF = BH_OFF + BH_BYTES, ONES_BYTES = kTileRows * 16 * 2;
   static constexpr uint32_t IMAGE_BYTES = ONES_OFF + ONES_BYTES;
-  static constexpr uint32_t STAGE_BYTES = (kTileRows * D * 4 + 15) / 16 * 16;
   static constexpr uint32_t A_BYTES = kTileRows * K1 * 2;
-  static constexpr uint32_t X_BYTES = STAGE_BYTES > kTileRows * H * 2 ? STAGE_BYTES : kTileRows * H * 2;
-  static constexpr int ACC_COLS = H;                            // layer accumulators (reused)
-  static constexpr int GROUP_COLS = H + 32;                     // + the heads accumulator
-  static constexpr int TMEM_COLS = kGroups * GROUP_COLS <= 256 ? 256 : 512;
+  static constexpr uint32_t STAGE_BYTES = (kTileRows * D * 4 + 15) / 16 * 16;
+  static constexpr uint32_t X_BYTES =
+      TM ? 16 : (STAGE_BYTES > kTileRows * H * 2 ? STAGE_BYTES : kTileRows * H * 2);
+  // Tensor-memory columns of one group: accumulator (reused by both hidden layers), the bf16
+  // hidden activations (two per column) when TM, the heads accumulator.
+  static constexpr int HID_COL = H;
+  static constexpr int HEAD_COL = H + (TM ? H / 2 : 0);
+  static constexpr int GROUP_COLS = HEAD_COL + 32;
+  static constexpr int GROUPS = (2 * GROUP_COLS <= 512 && 2 * (A_BYTES + X_BYTES) + IMAGE_BYTES <= 220 * 1024) ? 2 : 1;
+  static constexpr int TMEM_COLS = GROUPS * GROUP_COLS <= 256 ? 256 : 512;
+  static constexpr int THREADS = GROUPS * kGroupThreads;
 };
 
-template <int N, int F, int H>
+template <int N, int F, int H, bool TM>
 struct TcGroupSmem {
-  using S = TcShape<N, H>;
-  // fp32 observation block in the global layout while a step starts; the hidden activations
-  // (A operand of layer 2 and of the heads) for the rest of the step.
+  using S = TcShape<N, H, TM>;
+  // TM = false: the fp32 observation block in the global layout while a step starts, the hidden
+  // activations (A operand of layer 2 and of the heads) for the rest of the step.
   alignas(128) unsigned char x[S::X_BYTES];
   alignas(128) unsigned char a[S::A_BYTES];  // bf16 observations, A operand of layer 1
+  float step_frac[kTileRows];                // exact step/cap of each row (bf16 in A is rounded)
   alignas(8) uint64_t mma_bar;
 };
 
-template <int N, int F, int H>
+template <int N, int F, int H, bool TM>
 struct TcSmem {
-  using S = TcShape<N, H>;
+  using S = TcShape<N, H, TM>;
   alignas(128) unsigned char weights[S::IMAGE_BYTES];
-  TcGroupSmem<N, F, H> grp[kGroups];
+  TcGroupSmem<N, F, H, TM> grp[S::GROUPS];
   alignas(8) uint64_t load_bar;
   uint32_t tmem_base;
 };
@@ -176,16 +192,26 @@ __host__ __device__ constexpr uint32_t canon_offset(int n, int k, int K) {
   return static_cast<uint32_t>((n >> 3) * (K * 16) + (k >> 3) * 128 + (n & 7) * 16 + (k & 7) * 2);
 }
 
-template <int N, int H>
+__device__ __forceinline__ void split_bf16(float b, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+  hi = __float2bfloat16_rn(b);
+  lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+}
+
+template <int N, int H, bool TM>
 __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, ParamLayout L) {
-  using S = TcShape<N, H>;
+  using S = TcShape<N, H, TM>;
   constexpr int D = S::D, K1 = S::K1;
   auto at = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(image + off); };
   const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   for (int i = tid; i < H * K1; i += nth) {
     const int n = i / K1, k = i - n * K1;
-    at(S::W1_OFF)[canon_offset(n, k, K1) / 2] =
-        __float2bfloat16_rn(k < D ? params[L.W1 + static_cast<size_t>(n) * D + k] : 0.0f);
+    __nv_bfloat16 v = __float2bfloat16_rn(k < D ? params[L.W1 + static_cast<size_t>(n) * D + k] : 0.0f);
+    if (S::FOLD1 && (k == D || k == D + 1)) {
+      __nv_bfloat16 hi, lo;
+      split_bf16(params[L.b1 + n], hi, lo);
+      v = (k == D) ? hi : lo;
+    }
+    at(S::W1_OFF)[canon_offset(n, k, K1) / 2] = v;
   }
   for (int i = tid; i < H * H; i += nth) {
     const int n = i / H, k = i - n * H;
@@ -204,15 +230,18 @@ __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *
     float b;
     uint32_t off;
     int n;
-    if (r < H) { b = params[L.b1 + r]; off = S::B1_OFF; n = r; }
-    else if (r < 2 * H) { b = params[L.b2 + r - H]; off = S::B2_OFF; n = r - H; }
-    else {
+    if (r < H) {
+      if (S::FOLD1) continue;
+      b = params[L.b1 + r]; off = S::B1_OFF; n = r;
+    } else if (r < 2 * H) {
+      b = params[L.b2 + r - H]; off = S::B2_OFF; n = r - H;
+    } else {
       n = r - 2 * H;
       off = S::BH_OFF;
       b = n < kActions ? params[L.ba + n] : (n == kActions ? params[L.bv] : 0.0f);
     }
-    const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+    __nv_bfloat16 hi, lo;
+    split_bf16(b, hi, lo);
     at(off)[canon_offset(n, k, 16) / 2] = k == 0 ? hi : (k == 1 ? lo : __float2bfloat16_rn(0.0f));
   }
   for (int i = tid; i < kTileRows * 16; i += nth) {
@@ -221,7 +250,7 @@ __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *
   }
 }
 
-// ---- the rollout kernel ------------------------------------------------------------------------
+// ---- tensor-memory helpers ---------------------------------------------------------------------
 // 32 lanes x 32 bit, 32 consecutive columns (no wait: the caller waits once per batch of loads).
 __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
   asm volatile(
@@ -236,70 +265,110 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Thread i of the warp writes 16 consecutive 32-bit columns of lane (lane base + i).
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // max(x, 0) of two fp32 values rounded to bf16 and packed (lo in the low half).
 __device__ __forceinline__ uint32_t relu_pack_bf16(uint32_t lo_bits, uint32_t hi_bits) {
   uint32_t d;
   asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(hi_bits)), "f"(__uint_as_float(lo_bits)));
   return d;
 }
+__device__ __forceinline__ void relu_pack32(const uint32_t *r, uint32_t *packed) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) packed[i] = relu_pack_bf16(r[2 * i], r[2 * i + 1]);
+}
 
 // Epilogue of a hidden layer: thread `row` reads its accumulator row (bias already inside) from
-// tensor memory, applies ReLU, rounds to bf16 and stores the row as the next A operand (K = H).
-// The load of the next 32 columns is in flight while the current 32 are converted.
-template <int H>
-__device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, unsigned char *hbuf, int row) {
+// tensor memory, applies ReLU and rounds to bf16; the row becomes the A operand of the next
+// layer, either in shared memory (canonical layout, K = H) or, packed two per column, in tensor
+// memory.  The load of the next 32 columns is in flight while the current 32 are converted.
+template <int H, bool TM>
+__device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, uint32_t hid_taddr, unsigned char *hbuf, int row) {
   static_assert(H % 64 == 0, "two 32-column batches per iteration");
-  uint32_t ra[32], rb[32];
+  uint32_t ra[32], rb[32], pk[16];
   tmem_ld32_nowait(acc_taddr, ra);
 #pragma unroll
   for (int c0 = 0; c0 < H; c0 += 64) {
     tmem_ld_wait();
     tmem_ld32_nowait(acc_taddr + static_cast<uint32_t>(c0 + 32), rb);
+    relu_pack32(ra, pk);
+    if (TM) {
+      tmem_st16(hid_taddr + static_cast<uint32_t>(c0 / 2), pk);
+    } else {
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 8 * q, H)) =
-          make_uint4(relu_pack_bf16(ra[8 * q], ra[8 * q + 1]), relu_pack_bf16(ra[8 * q + 2], ra[8 * q + 3]),
-                     relu_pack_bf16(ra[8 * q + 4], ra[8 * q + 5]), relu_pack_bf16(ra[8 * q + 6], ra[8 * q + 7]));
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 8 * q, H)) =
+            make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+    }
     tmem_ld_wait();
     if (c0 + 64 < H) tmem_ld32_nowait(acc_taddr + static_cast<uint32_t>(c0 + 64), ra);
+    relu_pack32(rb, pk);
+    if (TM) {
+      tmem_st16(hid_taddr + static_cast<uint32_t>(c0 / 2 + 16), pk);
+    } else {
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 32 + 8 * q, H)) =
-          make_uint4(relu_pack_bf16(rb[8 * q], rb[8 * q + 1]), relu_pack_bf16(rb[8 * q + 2], rb[8 * q + 3]),
-                     relu_pack_bf16(rb[8 * q + 4], rb[8 * q + 5]), relu_pack_bf16(rb[8 * q + 6], rb[8 * q + 7]));
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 32 + 8 * q, H)) =
+            make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+    }
   }
+  if (TM) tmem_st_wait();
+}
+
+// A from tensor memory (lane = row, two bf16 per 32-bit column, 8 columns per K step of 16).
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
 
 // One dense layer on the tensor core, issued by a single thread: the accumulator is seeded with
-// the bias (ones tile x bias tile, K = 16) and then accumulates K / 16 steps of A x W^T.
-template <int K, int NOUT>
+// the bias (ones tile x bias tile, K = 16) unless the bias rides in the weights, and then
+// accumulates K / 16 steps of A x W^T, A from shared memory or from tensor memory.
+template <int K, int NOUT, bool BIAS_TILE, bool A_TMEM>
 __device__ __forceinline__ void issue_layer(uint32_t d_tmem, uint32_t a_addr, uint32_t w_addr, uint32_t ones_addr,
                                             uint32_t bias_addr, uint32_t bar) {
   constexpr uint32_t idesc = instr_desc(kTileRows, NOUT);
-  mma_bf16(d_tmem, smem_desc(ones_addr, 128, 256), smem_desc(bias_addr, 128, 256), idesc, 0);
+  if (BIAS_TILE) mma_bf16(d_tmem, smem_desc(ones_addr, 128, 256), smem_desc(bias_addr, 128, 256), idesc, 0);
 #pragma unroll
-  for (int k = 0; k < K / 16; ++k)
-    mma_bf16(d_tmem, smem_desc(a_addr + k * 256, 128, K * 16), smem_desc(w_addr + k * 256, 128, K * 16), idesc, 1);
+  for (int k = 0; k < K / 16; ++k) {
+    const uint32_t acc = (BIAS_TILE || k > 0) ? 1u : 0u;
+    if (A_TMEM) mma_bf16_ts(d_tmem, a_addr + k * 8, smem_desc(w_addr + k * 256, 128, K * 16), idesc, acc);
+    else mma_bf16(d_tmem, smem_desc(a_addr + k * 256, 128, K * 16), smem_desc(w_addr + k * 256, 128, K * 16), idesc, acc);
+  }
   mma_commit(bar);
 }
 
-template <int N, int F, int H>
-__global__ void __launch_bounds__(kTcThreads, 1)
+// ---- the rollout kernel ------------------------------------------------------------------------
+template <int N, int F, int H, bool TM>
+__global__ void __launch_bounds__(TcShape<N, H, TM>::THREADS, 1)
 rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles) {
-  using S = TcShape<N, H>;
-  constexpr int D = S::D, K1 = S::K1;
+  using S = TcShape<N, H, TM>;
+  constexpr int D = S::D, K1 = S::K1, G = S::GROUPS;
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  TcSmem<N, F, H> &sm = *reinterpret_cast<TcSmem<N, F, H> *>(smem_raw);
+  TcSmem<N, F, H, TM> &sm = *reinterpret_cast<TcSmem<N, F, H, TM> *>(smem_raw);
   const int tid = threadIdx.x;
   const int g = tid / kGroupThreads;   // group index
   const int row = tid % kGroupThreads; // row of the tile this thread owns; also its TMEM lane
-  const int warp = tid / 32;
-  TcGroupSmem<N, F, H> &gs = sm.grp[g];
+  const int warp = tid / 32, lane = tid & 31;
+  const int wg = row / 32;             // warp inside the group
+  TcGroupSmem<N, F, H, TM> &gs = sm.grp[g];
 
   // ---- one-time set-up: barriers, tensor memory, weights -------------------------------------
   if (tid == 0) {
     mbar_init(smem_u32(&sm.load_bar), 1);
-    for (int i = 0; i < kGroups; ++i) mbar_init(smem_u32(&sm.grp[i].mma_bar), 1);
+    for (int i = 0; i < G; ++i) mbar_init(smem_u32(&sm.grp[i].mma_bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -332,25 +401,26 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
 
   const uint32_t tmem_base = sm.tmem_base;
   const uint32_t acc_col = tmem_base + static_cast<uint32_t>(g * S::GROUP_COLS);
-  const uint32_t head_col = acc_col + static_cast<uint32_t>(S::ACC_COLS);
-  const uint32_t lane_off = static_cast<uint32_t>((warp % 4) * 32) << 16;  // this warp's TMEM lanes
+  const uint32_t hid_col = acc_col + static_cast<uint32_t>(S::HID_COL);
+  const uint32_t head_col = acc_col + static_cast<uint32_t>(S::HEAD_COL);
+  const uint32_t lane_off = static_cast<uint32_t>(wg * 32) << 16;  // this warp's TMEM lanes
   const uint32_t w_addr = smem_u32(sm.weights);
-  const uint32_t a_addr = smem_u32(gs.a), x_addr = smem_u32(gs.x);
+  const uint32_t a_addr = smem_u32(gs.a);
+  const uint32_t h_addr = TM ? hid_col : smem_u32(gs.x);  // A operand of layer 2 and of the heads
   const uint32_t bar = smem_u32(&gs.mma_bar);
   float *stage = reinterpret_cast<float *>(gs.x);
   uint32_t phase = 0;
   const size_t M = static_cast<size_t>(a.env.n_envs) * N;
 
   // ---- tiles of this group ---------------------------------------------------------------------
-  const int lane = tid & 31;
-  const int le = ((tid % kGroupThreads) / 32) * S::EPW + lane / N;  // local environment of this lane
-  const int ag = lane % N;                                         // its agent
-  const int crow = le * N + ag;                                    // compact row inside the tile's block
-  for (int tile = blockIdx.x * kGroups + g; tile < n_tiles && !timed_out; tile += gridDim.x * kGroups) {
+  const int le = wg * S::EPW + lane / N;  // local environment of this lane
+  const int ag = lane % N;                // its agent
+  const int crow = le * N + ag;           // compact row inside the tile's block
+  for (int tile = blockIdx.x * G + g; tile < n_tiles && !timed_out; tile += gridDim.x * G) {
     const int e0 = tile * ept;
     const int n_env = min(ept, a.env.n_envs - e0);
     const int n_rows = n_env * N;
-    const bool active = lane < S::EPW * N && le < n_env;
+    const bool active = lane < S::RPW && le < n_env;
     const int base = active ? lane - ag : lane;
     const uint32_t env_id = static_cast<uint32_t>(a.env.first_env + e0 + le);
     EnvRegs<N, F> env;
@@ -365,12 +435,18 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     for (int t = 0; t <= a.T; ++t) {
       const bool last = (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
-      // 1. non-zero observation entries: fp32 into the zeroed block, bf16 into the zeroed A tile
-      if (active)
+      // 1. non-zero observation entries into the zeroed A tile (and the zeroed fp32 block)
+      if (active) {
         observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
-          stage[crow * D + j] = v;
+          if (!TM) stage[crow * D + j] = v;
+          else if (j == 3 * kPlane + 1) gs.step_frac[row] = v;
           *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, j, K1)) = __float2bfloat16_rn(v);
         });
+        if (S::FOLD1) {  // the two columns that pick up the bias rows of W1
+          *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, D, K1)) = __float2bfloat16_rn(1.0f);
+          *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, D + 1, K1)) = __float2bfloat16_rn(1.0f);
+        }
+      }
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
@@ -378,46 +454,78 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       //    array) and the uniform of this step's action draw is computed
       if (row == 0) {
         tc_fence_after();
-        issue_layer<K1, H>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF, w_addr + S::B1_OFF, bar);
+        issue_layer<K1, H, !S::FOLD1, false>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF,
+                                             w_addr + S::B1_OFF, bar);
       }
       if (!last) {
         float *dst = a.buf.obs + row0 * D;
-        const int count = n_rows * D;
-        if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
-          for (int i = row; i < count / 4; i += kGroupThreads)
-            reinterpret_cast<float4 *>(dst)[i] = reinterpret_cast<const float4 *>(stage)[i];
+        if (!TM) {
+          const int count = n_rows * D;
+          if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
+            for (int i = row; i < count / 4; i += kGroupThreads)
+              reinterpret_cast<float4 *>(dst)[i] = reinterpret_cast<const float4 *>(stage)[i];
+          } else {
+            for (int i = row; i < count; i += kGroupThreads) dst[i] = stage[i];
+          }
         } else {
-          for (int i = row; i < count; i += kGroupThreads) dst[i] = stage[i];
+          // this warp's rows, expanded from the bf16 tile; consecutive lanes write consecutive floats
+          uint32_t off[(D + 31) / 32];
+#pragma unroll
+          for (int q = 0; q < (D + 31) / 32; ++q) off[q] = canon_offset(0, lane + 32 * q, K1);
+          const int first = wg * S::RPW;
+          for (int l = 0; l < S::RPW && first + l < n_rows; ++l) {
+            const int r = wg * 32 + l;  // tile row (tensor-memory lane) of compact row first + l
+            const unsigned char *arow = gs.a + canon_offset(r, 0, K1);
+            float *orow = dst + static_cast<size_t>(first + l) * D;
+#pragma unroll
+            for (int q = 0; q < (D + 31) / 32; ++q) {
+              const int j = lane + 32 * q;
+              if (j < D) {
+                float v = __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t *>(arow + off[q])) << 16);
+                if (j == 3 * kPlane + 1) v = gs.step_frac[r];
+                orow[j] = v;
+              }
+            }
+          }
+          __syncwarp();
         }
       }
       float u = 0.0f;
       if (active && !last) u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag));
-      group_sync(g);  // every read of the block is done before the epilogue reuses its memory
+      if (!TM) group_sync(g);  // every read of the block is done before the epilogue reuses its memory
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       tc_fence_after();
-      hidden_epilogue<H>(acc_col + lane_off, gs.x, row);
-      for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads)  // layer 1 is done with A
-        reinterpret_cast<uint4 *>(gs.a)[i] = make_uint4(0, 0, 0, 0);
+      hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
+      // layer 1 is done with A: zero it for the next step (TM: own row only, its readers are in this warp)
+      if (TM) {
+#pragma unroll
+        for (int kc = 0; kc < K1 / 8; ++kc)
+          *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
+      } else {
+        for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads)
+          reinterpret_cast<uint4 *>(gs.a)[i] = make_uint4(0, 0, 0, 0);
+      }
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
       // 3. layer 2
       if (row == 0) {
         tc_fence_after();
-        issue_layer<H, H>(acc_col, x_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
+        issue_layer<H, H, true, TM>(acc_col, h_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       tc_fence_after();
-      hidden_epilogue<H>(acc_col + lane_off, gs.x, row);
+      hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
       // 4. heads: six logits and the value, N padded to 16
       if (row == 0) {
         tc_fence_after();
-        issue_layer<H, kHeadRows>(head_col, x_addr, w_addr + S::WH_OFF, w_addr + S::ONES_OFF, w_addr + S::BH_OFF, bar);
+        issue_layer<H, kHeadRows, true, TM>(head_col, h_addr, w_addr + S::WH_OFF, w_addr + S::ONES_OFF,
+                                            w_addr + S::BH_OFF, bar);
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
@@ -426,9 +534,9 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       {
         float hv[16];
         tmem_ld16(head_col + lane_off, hv);
-        // the hidden activations are dead: zero the observation block for the next step
-        for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads)
-          reinterpret_cast<uint4 *>(gs.x)[i] = make_uint4(0, 0, 0, 0);
+        if (!TM)  // the hidden activations are dead: zero the observation block for the next step
+          for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads)
+            reinterpret_cast<uint4 *>(gs.x)[i] = make_uint4(0, 0, 0, 0);
         if (active) {
           a.buf.values[row0 + crow] = hv[kActions];
           if (!last) {
@@ -489,11 +597,11 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   }
 }
 
-template <int N, int F, int H>
+template <int N, int F, int H, bool TM>
 cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
-  using S = TcShape<N, H>;
-  auto kern = rollout_tc_kernel<N, F, H>;
-  const size_t smem = sizeof(TcSmem<N, F, H>);
+  using S = TcShape<N, H, TM>;
+  auto kern = rollout_tc_kernel<N, F, H, TM>;
+  const size_t smem = sizeof(TcSmem<N, F, H, TM>);
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (err != cudaSuccess) return err;
   int sms = 0;
@@ -501,55 +609,65 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   if (err != cudaSuccess) return err;
   // Environments per tile: full tiles when there is enough work for every group of every SM,
   // otherwise smaller tiles so that all groups have one (the per-step chain is latency-bound).
-  const int slots = sms * kGroups;
+  const int slots = sms * S::GROUPS;
   int ept = (h->cfg.n_envs + slots - 1) / slots;
   if (ept > S::EPT_MAX) ept = S::EPT_MAX;
   if (ept < 1) ept = 1;
   const int n_tiles = (h->cfg.n_envs + ept - 1) / ept;
-  const int grid = (n_tiles + kGroups - 1) / kGroups < sms ? (n_tiles + kGroups - 1) / kGroups : sms;
-  kern<<<grid, kTcThreads, smem, h->stream>>>(args, static_cast<const unsigned char *>(h->d_wtc), ept, n_tiles);
+  const int ctas = (n_tiles + S::GROUPS - 1) / S::GROUPS;
+  kern<<<ctas < sms ? ctas : sms, S::THREADS, smem, h->stream>>>(args, static_cast<const unsigned char *>(h->d_wtc), ept,
+                                                                 n_tiles);
   h->launches += 1;
   return cudaGetLastError();
 }
 
-template <int N, int H>
+template <int N, int H, bool TM>
 cudaError_t launch_prep_variant(mava_rollout *h, const float *params_dev) {
-  prep_tc_kernel<N, H><<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(h->d_wtc),
-                                                 param_layout(h->cfg, h->D, 1));
+  prep_tc_kernel<N, H, TM><<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(h->d_wtc),
+                                                     param_layout(h->cfg, h->D, 1));
   h->launches += 1;
   return cudaGetLastError();
 }
 
 }  // namespace
 
+// Shared-torso shapes run on the tensor cores; the centralised critic does not yet.
 bool tc_supported(const mava_config_t &cfg) {
   const int v = find_variant(cfg);
-  return v == 0 || v == 1 || v == 2;  // shared torso, H <= 128
+  return v == 0 || v == 1 || v == 2 || v == 4;
 }
 
+// Hidden activations in tensor memory: always for H = 256; for the smaller shapes only when the
+// handle asks for it (MAVA_FLAG_HIDDEN_IN_TMEM), which lets small cases exercise that path.
+static bool use_tm(const mava_rollout *h) { return h->variant == 4 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0; }
+
 size_t tc_weight_bytes(const mava_config_t &cfg, int) {
-  switch (find_variant(cfg)) {
-    case 0: return TcShape<2, 64>::IMAGE_BYTES;
-    case 1: return TcShape<2, 128>::IMAGE_BYTES;
-    case 2: return TcShape<3, 128>::IMAGE_BYTES;
+  switch (find_variant(cfg)) {  // the two layouts of a shape have the same image size
+    case 0: return TcShape<2, 64, false>::IMAGE_BYTES;
+    case 1: return TcShape<2, 128, false>::IMAGE_BYTES;
+    case 2: return TcShape<3, 128, false>::IMAGE_BYTES;
+    case 4: return TcShape<8, 256, true>::IMAGE_BYTES;
     default: return 16;
   }
 }
 
 cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev) {
   switch (h->variant) {
-    case 0: return launch_prep_variant<2, 64>(h, params_dev);
-    case 1: return launch_prep_variant<2, 128>(h, params_dev);
-    case 2: return launch_prep_variant<3, 128>(h, params_dev);
+    case 0: return launch_prep_variant<2, 64, false>(h, params_dev);
+    case 1: return launch_prep_variant<2, 128, false>(h, params_dev);
+    case 2: return launch_prep_variant<3, 128, false>(h, params_dev);
+    case 4: return launch_prep_variant<8, 256, true>(h, params_dev);
     default: return cudaErrorNotSupported;
   }
 }
 
 cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args) {
+  const bool tm = use_tm(h);
   switch (h->variant) {
-    case 0: return launch_tc_variant<2, 2, 64>(h, args);
-    case 1: return launch_tc_variant<2, 2, 128>(h, args);
-    case 2: return launch_tc_variant<3, 3, 128>(h, args);
+    case 0: return tm ? launch_tc_variant<2, 2, 64, true>(h, args) : launch_tc_variant<2, 2, 64, false>(h, args);
+    case 1: return tm ? launch_tc_variant<2, 2, 128, true>(h, args) : launch_tc_variant<2, 2, 128, false>(h, args);
+    case 2: return tm ? launch_tc_variant<3, 3, 128, true>(h, args) : launch_tc_variant<3, 3, 128, false>(h, args);
+    case 4: return launch_tc_variant<8, 8, 256, true>(h, args);
     default: return cudaErrorNotSupported;
   }
 }

@@ -68,13 +68,17 @@ def test_reduced_configs_fp32(idx, n_envs, T):
     print(idx, out)
 
 
-@pytest.mark.parametrize("idx,n_envs,T", [(1, 333, 60), (2, 300, 110), (3, 200, 105), (4, 150, 40)])
-def test_reduced_configs_bf16(idx, n_envs, T):
+@pytest.mark.parametrize("idx,n_envs,T,tmem", [(1, 333, 60, False), (2, 300, 110, False), (3, 200, 105, False),
+                                               (4, 150, 40, False), (0, 16, 32, True), (1, 333, 60, True),
+                                               (2, 300, 110, True)])
+def test_reduced_configs_bf16(idx, n_envs, T, tmem):
+    """tmem=True keeps the hidden activations in tensor memory (the layout H = 256 always uses)."""
     w = wl.workload(idx)
     if not _tc_available(w):
         pytest.skip("bf16 tensor-core path not compiled for this shape")
     params = wl.make_params(w, bias_scale=0.1)
-    ro, _ = run_gpu(w, BF16, T, n_envs=n_envs, params=params)
+    flags = binding.MAVA_FLAG_WRITE_LOGITS | (binding.MAVA_FLAG_HIDDEN_IN_TMEM if tmem else 0)
+    ro, _ = run_gpu(w, BF16, T, n_envs=n_envs, params=params, flags=flags)
     ids = wl.sample_env_ids(n_envs, 6, 6, 6, seed=idx)
     out = check_against_oracle(w, ro, params, T, BF16, ids)
     print(idx, out)
