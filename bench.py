@@ -273,7 +273,7 @@ def run_gpu(args):
     torch.cuda.synchronize()
     sampler.start()
     ro, params, t_roll, t_gae, launches = time_workload(torch, binding, w, precision, args.steps, args.warmup,
-                                                        first_env=rank * E, flush=flush)
+                                                        first_env=wl.shard_first_env(E, rank), flush=flush)
     torch.cuda.synchronize()
     clocks = sampler.stop()
     if dist is not None:

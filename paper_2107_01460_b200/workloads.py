@@ -91,3 +91,9 @@ def sample_env_ids(n_envs: int, head: int, tail: int, rand: int, seed: int = 0) 
     mid = rng.choice(np.arange(head, n_envs - tail), size=rand, replace=False)
     ids = np.concatenate([np.arange(head), mid, np.arange(n_envs - tail, n_envs)])
     return np.unique(ids).astype(np.int32)
+
+
+def shard_first_env(envs_per_rank: int, rank: int) -> int:
+    """Global index of a rank's environment 0 when every rank rolls `envs_per_rank` environments
+    of one batch of world*envs_per_rank (weak scaling; environments never communicate)."""
+    return envs_per_rank * rank
