@@ -156,6 +156,30 @@ int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host);
 int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32_t T, float gamma,
                               float lambda, const mava_host_buffers_t *out);
 
+/* Allocation-free rollout (the paper has no counterpart; it exists for callers that cannot
+ * allocate).  Some users of this library must not call cudaMalloc/cudaFree while they run: a
+ * process that handed all device memory to its own pool, a serving or control loop in which the
+ * implicit device-wide synchronisation of an allocation is not acceptable, or code that runs after
+ * its start-up phase under a "no further allocations" rule.  This entry point does what
+ * create + run do for a fresh handle -- every environment starts episode 0 at global step 0 under
+ * cfg->seed, then T steps are rolled out into the caller's buffers -- but it creates no handle
+ * and calls no allocating routine: the library's scratch (status word, environment states,
+ * re-laid-out weights) lives in one static device array of MAVA_STATIC_SCRATCH_BYTES that every
+ * GPU loading the library holds until the process exits.
+ *   - Shapes whose scratch does not fit (60 bytes per environment plus up to 201 KB of weights,
+ *     i.e. roughly 13 000 environments) are refused with MAVA_ERR_CAPACITY; T > cfg->max_T too.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress);
+ *     make that first call before any stream capture.
+ *   - All calls share the array and it keeps the previous call's contents; the call clears what
+ *     must start at zero.  Two calls that overlap on the GPU (different streams or threads) race:
+ *     serialise them.  It does not touch handles made by mava_rollout_create.
+ *   - cfg, buffers, params_dev and T mean what they mean for create and run; GAE is not included
+ *     (mava_gae needs no scratch).  The call waits for the stream and returns MAVA_OK,
+ *     MAVA_ERR_DEVICE_TIMEOUT, or the errors of create/run. */
+#define MAVA_STATIC_SCRATCH_BYTES (1u << 20)
+int mava_rollout_run_static(const mava_config_t *cfg, const mava_buffers_t *buffers, const float *params_dev,
+                            int32_t T, void *cuda_stream);
+
 /* Number of kernels this handle has launched so far (for launch accounting). */
 int64_t mava_rollout_launch_count(const mava_rollout_t *h);
 

@@ -28,7 +28,7 @@ EXPORTS = [
     "mava_params_count", "mava_rollout_create", "mava_rollout_run", "mava_rollout_run_forced", "mava_gae",
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
-    "mava_strerror",
+    "mava_strerror", "mava_rollout_run_static",
 ]
 
 
@@ -76,6 +76,8 @@ def lib():
         L.mava_rollout_launch_count.argtypes = [vp]; L.mava_rollout_launch_count.restype = C.c_int64
         L.mava_rollout_destroy.argtypes = [vp]; L.mava_rollout_destroy.restype = None
         L.mava_strerror.argtypes = [C.c_int]; L.mava_strerror.restype = C.c_char_p
+        L.mava_rollout_run_static.argtypes = [cfgp, bufp, vp, C.c_int32, vp]
+        L.mava_rollout_run_static.restype = C.c_int
         _lib = L
     return _lib
 
@@ -99,6 +101,13 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
 def _check(code: int, where: str):
     if code != MAVA_OK:
         raise MavaError(code, where)
+
+
+def mava_rollout_run_static(cfg: mava_config_t, buffers: mava_buffers_t, params_dev_ptr: int, T: int,
+                            cuda_stream: int | None = None) -> int:
+    """The allocation-free rollout for callers that must not allocate device memory (see the
+    header): returns the C status code; `buffers` holds raw device pointers the caller owns."""
+    return int(lib().mava_rollout_run_static(C.byref(cfg), C.byref(buffers), params_dev_ptr, T, cuda_stream))
 
 
 class Rollout:

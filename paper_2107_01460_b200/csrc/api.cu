@@ -1,4 +1,5 @@
 // C ABI of libmava_rollout.so: argument checks, handle life cycle and kernel enqueueing.
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -255,6 +256,89 @@ int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32
 }
 
 int64_t mava_rollout_launch_count(const mava_rollout_t *h) { return h ? h->launches : 0; }
+
+// ---- allocation-free variant ----------------------------------------------------------------
+// Scratch of mava_rollout_run_static: every GPU that loads this library carries these bytes
+// until the process exits.  In host code `g_static_scratch` is only a stand-in for the symbol;
+// the device address comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[MAVA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+unsigned char *g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device` (which must be current), resolved on first use.
+unsigned char *static_scratch(int device) {
+  if (device < 0 || device >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[device]) {
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    g_scratch_addr[device] = static_cast<unsigned char *>(ptr);
+  }
+  return g_scratch_addr[device];
+}
+
+size_t round256(size_t n) { return (n + 255) / 256 * 256; }
+}  // namespace
+
+int mava_rollout_run_static(const mava_config_t *cfg, const mava_buffers_t *buffers, const float *params_dev,
+                            int32_t T, void *cuda_stream) {
+  if (!cfg || !buffers || !params_dev) return MAVA_ERR_INVALID_ARG;
+  if (!config_ok(*cfg) || T < 1) return MAVA_ERR_INVALID_ARG;
+  if (T > cfg->max_T) return MAVA_ERR_CAPACITY;
+  if (cfg->view_radius != kViewRadius || cfg->n_agents * cfg->max_agent_level > 31) return MAVA_ERR_UNSUPPORTED;
+  const mava_buffers_t &b = *buffers;
+  if (!b.obs || !b.actions || !b.logp || !b.values || !b.rewards || !b.dones) return MAVA_ERR_INVALID_ARG;
+  if ((cfg->flags & MAVA_FLAG_WRITE_LOGITS) && !b.logits) return MAVA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(b.obs) % 16 != 0) return MAVA_ERR_INVALID_ARG;
+  const int variant = find_variant(*cfg);
+  if (variant < 0) return MAVA_ERR_UNSUPPORTED;
+  const bool bf16 = cfg->precision == MAVA_PRECISION_BF16;
+  if (bf16 && !tc_supported(*cfg)) return MAVA_ERR_UNSUPPORTED;
+
+  // carve the scratch: status word | environment states | re-laid-out weights
+  const int D = obs_dim(*cfg);
+  const size_t state_bytes = round256(sizeof(EnvRec) * static_cast<size_t>(cfg->n_envs));
+  const size_t weight_bytes = round256(bf16 ? tc_weight_bytes(*cfg, D) : sizeof(float) * simt_weight_floats(*cfg, D));
+  if (256 + state_bytes + weight_bytes > MAVA_STATIC_SCRATCH_BYTES) return MAVA_ERR_CAPACITY;
+
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) return MAVA_ERR_CUDA;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return MAVA_ERR_CUDA;
+  if (major != 10) return MAVA_ERR_UNSUPPORTED;
+  unsigned char *scratch = static_scratch(device);
+  if (!scratch) return MAVA_ERR_CUDA;
+
+  mava_rollout h{};  // a handle on the stack whose device state lives in the static array
+  h.cfg = *cfg;
+  h.buf = b;
+  h.stream = static_cast<cudaStream_t>(cuda_stream);
+  h.device = device;
+  h.D = D;
+  h.variant = variant;
+  h.d_status = reinterpret_cast<int *>(scratch);
+  h.d_state = reinterpret_cast<EnvRec *>(scratch + 256);
+  if (bf16) h.d_wtc = scratch + 256 + state_bytes;
+  else h.d_wsimt = reinterpret_cast<float *>(scratch + 256 + state_bytes);
+
+  // the array keeps what the previous call left: the status word must start at zero; the
+  // states and the weights are fully rewritten by the kernels below
+  if (cudaMemsetAsync(h.d_status, 0, sizeof(int), h.stream) != cudaSuccess) return MAVA_ERR_CUDA;
+  if (launch_env_init(&h) != cudaSuccess) return MAVA_ERR_CUDA;
+  const int rc = run_common(&h, params_dev, T, nullptr);
+  if (rc != MAVA_OK) return rc;
+  int status = 0;
+  if (cudaMemcpyAsync(&status, h.d_status, sizeof(int), cudaMemcpyDeviceToHost, h.stream) != cudaSuccess ||
+      cudaStreamSynchronize(h.stream) != cudaSuccess)
+    return MAVA_ERR_CUDA;
+  return status != 0 ? MAVA_ERR_DEVICE_TIMEOUT : MAVA_OK;
+}
 
 void mava_rollout_destroy(mava_rollout_t *h) {
   if (!h) return;
