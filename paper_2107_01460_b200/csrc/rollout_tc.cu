@@ -73,6 +73,14 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void group_sync(int g) {
   asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "r"(kGroupThreads) : "memory");
 }
+// Producer/consumer halves of a named barrier shared by the group and its helper threads.
+__device__ __forceinline__ void pair_arrive(int id) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
+}
+__device__ __forceinline__ void pair_sync(int id) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
+}
+constexpr int kBarTileReady = 8, kBarTileFree = 9;  // ids 1..2 belong to the groups
 // Barrier of the group that also ORs a predicate over its threads.
 __device__ __forceinline__ bool group_any(int g, bool pred) {
   uint32_t out;
@@ -162,7 +170,10 @@ struct TcShape {
   static constexpr int GROUP_COLS = HEAD_COL + 32;
   static constexpr int GROUPS = (2 * GROUP_COLS <= 512 && 2 * (A_BYTES + X_BYTES) + IMAGE_BYTES <= 220 * 1024) ? 2 : 1;
   static constexpr int TMEM_COLS = GROUPS * GROUP_COLS <= 256 ? 256 : 512;
-  static constexpr int THREADS = GROUPS * kGroupThreads;
+  // With a single group there is register room for a second set of 128 threads that only ship
+  // the observation block to global memory, off the group's critical path.
+  static constexpr bool HELPERS = TM && GROUPS == 1;
+  static constexpr int THREADS = (GROUPS + (HELPERS ? 1 : 0)) * kGroupThreads;
 };
 
 template <int N, int F, int H, bool TM>
@@ -173,6 +184,7 @@ struct TcGroupSmem {
   alignas(128) unsigned char x[S::X_BYTES];
   alignas(128) unsigned char a[S::A_BYTES];  // bf16 observations, A operand of layer 1
   float step_frac[kTileRows];                // exact step/cap of each row (bf16 in A is rounded)
+  int abort;                                 // set by the group when it stops early (helpers watch it)
   alignas(8) uint64_t mma_bar;
 };
 
@@ -350,6 +362,42 @@ __device__ __forceinline__ void issue_layer(uint32_t d_tmem, uint32_t a_addr, ui
   mma_commit(bar);
 }
 
+// Observation rows [first, first + n) of a tile (compact numbering; tile row = tile_row0 + i),
+// expanded from the bf16 A tile to fp32 and written to `dst` (row stride D); consecutive lanes
+// write consecutive floats.  The exact step/cap replaces the rounded bf16 one.  Four rows are in
+// flight at a time.
+template <int D, int K1>
+__device__ __forceinline__ void expand_rows(const unsigned char *a_tile, const float *step_frac, float *dst,
+                                            int first, int n, int tile_row0, int lane) {
+  constexpr int Q = (D + 31) / 32;
+  uint32_t off[Q];
+#pragma unroll
+  for (int q = 0; q < Q; ++q) off[q] = (static_cast<uint32_t>(lane + 32 * q) >> 3) * 128 + ((lane + 32 * q) & 7) * 2;
+  for (int l0 = 0; l0 < n; l0 += 4) {
+    uint16_t raw[4][Q];
+    float sf[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int tr = tile_row0 + min(l0 + r, n - 1);
+      const unsigned char *arow = a_tile + (tr >> 3) * (K1 * 16) + (tr & 7) * 16;
+#pragma unroll
+      for (int q = 0; q < Q; ++q) raw[r][q] = (lane + 32 * q < D) ? *reinterpret_cast<const uint16_t *>(arow + off[q]) : 0;
+      sf[r] = step_frac[tr];
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      if (l0 + r < n) {
+        float *orow = dst + static_cast<size_t>(first + l0 + r) * D;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+          const int j = lane + 32 * q;
+          if (j < D) orow[j] = (j == 3 * kPlane + 1) ? sf[r] : __uint_as_float(static_cast<uint32_t>(raw[r][q]) << 16);
+        }
+      }
+    }
+  }
+}
+
 // ---- the rollout kernel ------------------------------------------------------------------------
 template <int N, int F, int H, bool TM>
 __global__ void __launch_bounds__(TcShape<N, H, TM>::THREADS, 1)
@@ -363,10 +411,12 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const int row = tid % kGroupThreads; // row of the tile this thread owns; also its TMEM lane
   const int warp = tid / 32, lane = tid & 31;
   const int wg = row / 32;             // warp inside the group
-  TcGroupSmem<N, F, H, TM> &gs = sm.grp[g];
+  const bool is_helper = S::HELPERS && tid >= G * kGroupThreads;
+  TcGroupSmem<N, F, H, TM> &gs = sm.grp[is_helper ? 0 : g];
 
   // ---- one-time set-up: barriers, tensor memory, weights -------------------------------------
   if (tid == 0) {
+    for (int i = 0; i < G; ++i) sm.grp[i].abort = 0;
     mbar_init(smem_u32(&sm.load_bar), 1);
     for (int i = 0; i < G; ++i) mbar_init(smem_u32(&sm.grp[i].mma_bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -377,7 +427,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  {  // zero the observation block and the A operand once
+  if (!is_helper) {  // zero the observation block and the A operand once
     uint4 *z = reinterpret_cast<uint4 *>(gs.x);
     for (int i = row; i < static_cast<int>(S::X_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
     z = reinterpret_cast<uint4 *>(gs.a);
@@ -412,6 +462,26 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   uint32_t phase = 0;
   const size_t M = static_cast<size_t>(a.env.n_envs) * N;
 
+  // ---- helper threads: ship each step's observation block, then leave -------------------------
+  if (is_helper) {
+    TcGroupSmem<N, F, H, TM> &g0 = sm.grp[0];
+    const int hw = (tid - kGroupThreads) / 32;
+    pair_arrive(kBarTileFree);  // the tile starts out free
+    bool stop = timed_out;
+    for (int tile = blockIdx.x; tile < n_tiles && !stop; tile += gridDim.x) {
+      const int e0 = tile * ept;
+      const int n_rows = min(ept, a.env.n_envs - e0) * N;
+      for (int t = 0; t <= a.T && !stop; ++t) {
+        pair_sync(kBarTileReady);
+        if (*reinterpret_cast<volatile int *>(&g0.abort)) { stop = true; break; }
+        if (t < a.T) {
+          float *dst = a.buf.obs + (static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N) * D;
+          expand_rows<D, K1>(g0.a, g0.step_frac, dst, hw * S::RPW, min(S::RPW, n_rows - hw * S::RPW), hw * 32, lane);
+        }
+        pair_arrive(kBarTileFree);
+      }
+    }
+  } else {
   // ---- tiles of this group ---------------------------------------------------------------------
   const int le = wg * S::EPW + lane / N;  // local environment of this lane
   const int ag = lane % N;                // its agent
@@ -436,6 +506,12 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       const bool last = (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
       // 1. non-zero observation entries into the zeroed A tile (and the zeroed fp32 block)
+      if (S::HELPERS) {
+        pair_sync(kBarTileFree);  // the helpers have shipped the previous step's block
+#pragma unroll
+        for (int kc = 0; kc < K1 / 8; ++kc)
+          *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
+      }
       if (active) {
         observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
           if (!TM) stage[crow * D + j] = v;
@@ -450,6 +526,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
+      if (S::HELPERS) pair_arrive(kBarTileReady);
       // 2. layer 1 runs while the block goes to obs[t] (one contiguous piece of the time-major
       //    array) and the uniform of this step's action draw is computed
       if (row == 0) {
@@ -468,25 +545,9 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
             for (int i = row; i < count; i += kGroupThreads) dst[i] = stage[i];
           }
         } else {
-          // this warp's rows, expanded from the bf16 tile; consecutive lanes write consecutive floats
-          uint32_t off[(D + 31) / 32];
-#pragma unroll
-          for (int q = 0; q < (D + 31) / 32; ++q) off[q] = canon_offset(0, lane + 32 * q, K1);
-          const int first = wg * S::RPW;
-          for (int l = 0; l < S::RPW && first + l < n_rows; ++l) {
-            const int r = wg * 32 + l;  // tile row (tensor-memory lane) of compact row first + l
-            const unsigned char *arow = gs.a + canon_offset(r, 0, K1);
-            float *orow = dst + static_cast<size_t>(first + l) * D;
-#pragma unroll
-            for (int q = 0; q < (D + 31) / 32; ++q) {
-              const int j = lane + 32 * q;
-              if (j < D) {
-                float v = __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t *>(arow + off[q])) << 16);
-                if (j == 3 * kPlane + 1) v = gs.step_frac[r];
-                orow[j] = v;
-              }
-            }
-          }
+          // this warp's rows, expanded from the bf16 tile (helper threads do it when there are any)
+          if (!S::HELPERS)
+            expand_rows<D, K1>(gs.a, gs.step_frac, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
           __syncwarp();
         }
       }
@@ -498,7 +559,9 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
       // layer 1 is done with A: zero it for the next step (TM: own row only, its readers are in this warp)
-      if (TM) {
+      if (S::HELPERS) {
+        // zeroed at the top of the next step, once the helpers are done reading it
+      } else if (TM) {
 #pragma unroll
         for (int kc = 0; kc < K1 / 8; ++kc)
           *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
@@ -573,7 +636,15 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         }
       }
       tc_fence_before();
-      if (group_any(g, timed_out)) { timed_out = true; break; }
+      if (group_any(g, timed_out)) {
+        timed_out = true;
+        if (S::HELPERS) {  // release the helpers, which wait for the next step's tile
+          if (row == 0) *reinterpret_cast<volatile int *>(&gs.abort) = 1;
+          __threadfence_block();
+          pair_arrive(kBarTileReady);
+        }
+        break;
+      }
       if (last) break;
       // 5. transition and auto-reset, inside the warp
       float reward;
@@ -587,6 +658,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
+  }  // group threads
 
   // ---- common exit: every thread arrives here; tensor memory is returned ----------------------
   tc_fence_before();
