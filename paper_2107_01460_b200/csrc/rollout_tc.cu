@@ -73,14 +73,16 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void group_sync(int g) {
   asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "r"(kGroupThreads) : "memory");
 }
-// Producer/consumer halves of a named barrier shared by the group and its helper threads.
+// Producer/consumer halves of a named barrier shared by the two thread groups of a CTA.
 __device__ __forceinline__ void pair_arrive(int id) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
 }
 __device__ __forceinline__ void pair_sync(int id) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
 }
-constexpr int kBarTileReady = 8, kBarTileFree = 9;  // ids 1..2 belong to the groups
+// Ping-pong hand-over barriers (ids 1..2 belong to the groups): group g waits on kBar* + g for
+// the A tile / the tensor-memory columns, and the other group arrives there when it lets go.
+constexpr int kBarTile = 8, kBarTmem = 10;
 // Barrier of the group that also ORs a predicate over its threads.
 __device__ __forceinline__ bool group_any(int g, bool pred) {
   uint32_t out;
@@ -168,12 +170,15 @@ struct TcShape {
   static constexpr int HID_COL = H;
   static constexpr int HEAD_COL = H + (TM ? H / 2 : 0);
   static constexpr int GROUP_COLS = HEAD_COL + 32;
+  // independent sets of tile resources (A tile, block, tensor-memory columns) per CTA
   static constexpr int GROUPS = (2 * GROUP_COLS <= 512 && 2 * (A_BYTES + X_BYTES) + IMAGE_BYTES <= 220 * 1024) ? 2 : 1;
   static constexpr int TMEM_COLS = GROUPS * GROUP_COLS <= 256 ? 256 : 512;
-  // With a single group there is register room for a second set of 128 threads that only ship
-  // the observation block to global memory, off the group's critical path.
-  static constexpr bool HELPERS = TM && GROUPS == 1;
-  static constexpr int THREADS = (GROUPS + (HELPERS ? 1 : 0)) * kGroupThreads;
+  // When only one set of tile resources fits (H = 256), two thread groups still run, in
+  // anti-phase: they take turns on the one A tile and the one set of tensor-memory columns, so
+  // that one group's environment phase (sampler, transition, observation) overlaps the other's
+  // network phase (the three MMAs and their epilogues).
+  static constexpr bool PINGPONG = TM && GROUPS == 1;
+  static constexpr int THREADS = 2 * kGroupThreads;
 };
 
 template <int N, int F, int H, bool TM>
@@ -184,8 +189,6 @@ struct TcGroupSmem {
   alignas(128) unsigned char x[S::X_BYTES];
   alignas(128) unsigned char a[S::A_BYTES];  // bf16 observations, A operand of layer 1
   float step_frac[kTileRows];                // exact step/cap of each row (bf16 in A is rounded)
-  int abort;                                 // set by the group when it stops early (helpers watch it)
-  alignas(8) uint64_t mma_bar;
 };
 
 template <int N, int F, int H, bool TM>
@@ -193,8 +196,10 @@ struct TcSmem {
   using S = TcShape<N, H, TM>;
   alignas(128) unsigned char weights[S::IMAGE_BYTES];
   TcGroupSmem<N, F, H, TM> grp[S::GROUPS];
+  alignas(8) uint64_t mma_bar[2];  // one per thread group
   alignas(8) uint64_t load_bar;
   uint32_t tmem_base;
+  int abort;  // ping-pong mode: a group gave up; both finish their barrier protocol without work
 };
 
 // ---- weight image ------------------------------------------------------------------------------
@@ -403,22 +408,24 @@ template <int N, int F, int H, bool TM>
 __global__ void __launch_bounds__(TcShape<N, H, TM>::THREADS, 1)
 rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles) {
   using S = TcShape<N, H, TM>;
-  constexpr int D = S::D, K1 = S::K1, G = S::GROUPS;
+  constexpr int D = S::D, K1 = S::K1;
+  constexpr bool PP = S::PINGPONG;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TcSmem<N, F, H, TM> &sm = *reinterpret_cast<TcSmem<N, F, H, TM> *>(smem_raw);
   const int tid = threadIdx.x;
-  const int g = tid / kGroupThreads;   // group index
+  const int g = tid / kGroupThreads;   // thread group
+  const int dg = PP ? 0 : g;           // the set of tile resources it uses
   const int row = tid % kGroupThreads; // row of the tile this thread owns; also its TMEM lane
   const int warp = tid / 32, lane = tid & 31;
   const int wg = row / 32;             // warp inside the group
-  const bool is_helper = S::HELPERS && tid >= G * kGroupThreads;
-  TcGroupSmem<N, F, H, TM> &gs = sm.grp[is_helper ? 0 : g];
+  TcGroupSmem<N, F, H, TM> &gs = sm.grp[dg];
 
   // ---- one-time set-up: barriers, tensor memory, weights -------------------------------------
   if (tid == 0) {
-    for (int i = 0; i < G; ++i) sm.grp[i].abort = 0;
+    sm.abort = 0;
     mbar_init(smem_u32(&sm.load_bar), 1);
-    for (int i = 0; i < G; ++i) mbar_init(smem_u32(&sm.grp[i].mma_bar), 1);
+    mbar_init(smem_u32(&sm.mma_bar[0]), 1);
+    mbar_init(smem_u32(&sm.mma_bar[1]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -427,7 +434,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (!is_helper) {  // zero the observation block and the A operand once
+  if (!PP || g == 0) {  // zero the observation block and the A operand once
     uint4 *z = reinterpret_cast<uint4 *>(gs.x);
     for (int i = row; i < static_cast<int>(S::X_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
     z = reinterpret_cast<uint4 *>(gs.a);
@@ -447,48 +454,40 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     }
   }
   timed_out = !mbar_wait(smem_u32(&sm.load_bar), 0);
-  timed_out = __syncthreads_or(timed_out) != 0;  // uniform: the tile loops below depend on it
+  timed_out = __syncthreads_or(timed_out) != 0;  // uniform: the loops below depend on it
 
   const uint32_t tmem_base = sm.tmem_base;
-  const uint32_t acc_col = tmem_base + static_cast<uint32_t>(g * S::GROUP_COLS);
+  const uint32_t acc_col = tmem_base + static_cast<uint32_t>(dg * S::GROUP_COLS);
   const uint32_t hid_col = acc_col + static_cast<uint32_t>(S::HID_COL);
   const uint32_t head_col = acc_col + static_cast<uint32_t>(S::HEAD_COL);
   const uint32_t lane_off = static_cast<uint32_t>(wg * 32) << 16;  // this warp's TMEM lanes
   const uint32_t w_addr = smem_u32(sm.weights);
   const uint32_t a_addr = smem_u32(gs.a);
   const uint32_t h_addr = TM ? hid_col : smem_u32(gs.x);  // A operand of layer 2 and of the heads
-  const uint32_t bar = smem_u32(&gs.mma_bar);
+  const uint32_t bar = smem_u32(&sm.mma_bar[g]);
   float *stage = reinterpret_cast<float *>(gs.x);
   uint32_t phase = 0;
   const size_t M = static_cast<size_t>(a.env.n_envs) * N;
-
-  // ---- helper threads: ship each step's observation block, then leave -------------------------
-  if (is_helper) {
-    TcGroupSmem<N, F, H, TM> &g0 = sm.grp[0];
-    const int hw = (tid - kGroupThreads) / 32;
-    pair_arrive(kBarTileFree);  // the tile starts out free
-    bool stop = timed_out;
-    for (int tile = blockIdx.x; tile < n_tiles && !stop; tile += gridDim.x) {
-      const int e0 = tile * ept;
-      const int n_rows = min(ept, a.env.n_envs - e0) * N;
-      for (int t = 0; t <= a.T && !stop; ++t) {
-        pair_sync(kBarTileReady);
-        if (*reinterpret_cast<volatile int *>(&g0.abort)) { stop = true; break; }
-        if (t < a.T) {
-          float *dst = a.buf.obs + (static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N) * D;
-          expand_rows<D, K1>(g0.a, g0.step_frac, dst, hw * S::RPW, min(S::RPW, n_rows - hw * S::RPW), hw * 32, lane);
-        }
-        pair_arrive(kBarTileFree);
-      }
-    }
-  } else {
-  // ---- tiles of this group ---------------------------------------------------------------------
   const int le = wg * S::EPW + lane / N;  // local environment of this lane
   const int ag = lane % N;                // its agent
   const int crow = le * N + ag;           // compact row inside the tile's block
-  for (int tile = blockIdx.x * G + g; tile < n_tiles && !timed_out; tile += gridDim.x * G) {
+
+  if (PP && g == 1) {  // group 0 goes first on both shared resources
+    pair_arrive(kBarTile + 0);
+    pair_arrive(kBarTmem + 0);
+  }
+
+  // ---- tiles: in round `it` group g works on tile (it * gridDim.x + blockIdx.x) * 2 + g ----------
+  for (int it = 0; !timed_out || PP; ++it) {
+    const int tile0 = (it * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x)) * 2;
+    if (tile0 >= n_tiles) break;  // same for both groups
+    const int tile = tile0 + g;
+    if (!PP && tile >= n_tiles) break;
+    // ping-pong: a group without a tile (or after a time-out) still walks through the hand-over
+    // barriers of every step, so that its partner never waits for it in vain
+    bool idle = PP && (tile >= n_tiles || timed_out);
     const int e0 = tile * ept;
-    const int n_env = min(ept, a.env.n_envs - e0);
+    const int n_env = idle ? 0 : min(ept, a.env.n_envs - e0);
     const int n_rows = n_env * N;
     const bool active = lane < S::RPW && le < n_env;
     const int base = active ? lane - ag : lane;
@@ -505,13 +504,21 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     for (int t = 0; t <= a.T; ++t) {
       const bool last = (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
-      // 1. non-zero observation entries into the zeroed A tile (and the zeroed fp32 block)
-      if (S::HELPERS) {
-        pair_sync(kBarTileFree);  // the helpers have shipped the previous step's block
+      if (PP) {
+        pair_sync(kBarTile + g);  // the other group is done with the A tile
+        // one verdict for the whole group (its threads may see the flag at different times)
+        idle = group_any(g, idle || *reinterpret_cast<volatile int *>(&sm.abort) != 0);
+        if (idle) {  // keep the hand-over order of a working step: tile, tensor memory, tile, tensor memory
+          pair_sync(kBarTmem + g);
+          pair_arrive(kBarTile + (1 - g));
+          pair_arrive(kBarTmem + (1 - g));
+          continue;
+        }
 #pragma unroll
         for (int kc = 0; kc < K1 / 8; ++kc)
           *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
       }
+      // 1. non-zero observation entries into the zeroed A tile (and the zeroed fp32 block)
       if (active) {
         observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
           if (!TM) stage[crow * D + j] = v;
@@ -526,28 +533,26 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
-      if (S::HELPERS) pair_arrive(kBarTileReady);
-      // 2. layer 1 runs while the block goes to obs[t] (one contiguous piece of the time-major
-      //    array) and the uniform of this step's action draw is computed
+      if (PP) pair_sync(kBarTmem + g);  // the other group has read its heads out of tensor memory
+      // 2. layer 1 runs while the uniform of this step's action draw is computed and (when the
+      //    block is not needed later) the observation block goes to obs[t]
       if (row == 0) {
         tc_fence_after();
         issue_layer<K1, H, !S::FOLD1, false>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF,
                                              w_addr + S::B1_OFF, bar);
       }
-      if (!last) {
-        float *dst = a.buf.obs + row0 * D;
-        if (!TM) {
+      float *obs_dst = a.buf.obs + row0 * D;
+      if (!last && !PP) {
+        if (!TM) {  // one contiguous piece of the time-major array
           const int count = n_rows * D;
           if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
             for (int i = row; i < count / 4; i += kGroupThreads)
-              reinterpret_cast<float4 *>(dst)[i] = reinterpret_cast<const float4 *>(stage)[i];
+              reinterpret_cast<float4 *>(obs_dst)[i] = reinterpret_cast<const float4 *>(stage)[i];
           } else {
-            for (int i = row; i < count; i += kGroupThreads) dst[i] = stage[i];
+            for (int i = row; i < count; i += kGroupThreads) obs_dst[i] = stage[i];
           }
-        } else {
-          // this warp's rows, expanded from the bf16 tile (helper threads do it when there are any)
-          if (!S::HELPERS)
-            expand_rows<D, K1>(gs.a, gs.step_frac, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+        } else {  // this warp's rows, expanded from the bf16 tile
+          expand_rows<D, K1>(gs.a, gs.step_frac, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
           __syncwarp();
         }
       }
@@ -558,24 +563,27 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       phase ^= 1;
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
-      // layer 1 is done with A: zero it for the next step (TM: own row only, its readers are in this warp)
-      if (S::HELPERS) {
-        // zeroed at the top of the next step, once the helpers are done reading it
-      } else if (TM) {
+      // layer 1 is done with A: zero it for the next step (ping-pong: the next user does that)
+      if (TM && !PP) {  // own row only, its readers are in this warp
 #pragma unroll
         for (int kc = 0; kc < K1 / 8; ++kc)
           *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
-      } else {
+      } else if (!TM) {
         for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads)
           reinterpret_cast<uint4 *>(gs.a)[i] = make_uint4(0, 0, 0, 0);
       }
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
-      // 3. layer 2
+      // 3. layer 2; in ping-pong mode its (long) run time hides the observation block's way out
       if (row == 0) {
         tc_fence_after();
         issue_layer<H, H, true, TM>(acc_col, h_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
+      }
+      if (PP) {
+        if (!last)
+          expand_rows<D, K1>(gs.a, gs.step_frac, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+        pair_arrive(kBarTile + (1 - g));  // this thread no longer needs the A tile
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
@@ -597,6 +605,10 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       {
         float hv[16];
         tmem_ld16(head_col + lane_off, hv);
+        if (PP) {  // this thread is done with tensor memory for this step
+          tc_fence_before();
+          pair_arrive(kBarTmem + (1 - g));
+        }
         if (!TM)  // the hidden activations are dead: zero the observation block for the next step
           for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads)
             reinterpret_cast<uint4 *>(gs.x)[i] = make_uint4(0, 0, 0, 0);
@@ -638,12 +650,10 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       tc_fence_before();
       if (group_any(g, timed_out)) {
         timed_out = true;
-        if (S::HELPERS) {  // release the helpers, which wait for the next step's tile
-          if (row == 0) *reinterpret_cast<volatile int *>(&gs.abort) = 1;
-          __threadfence_block();
-          pair_arrive(kBarTileReady);
-        }
-        break;
+        if (!PP) break;
+        if (row == 0) *reinterpret_cast<volatile int *>(&sm.abort) = 1;  // both groups go idle from their next step on
+        idle = true;
+        continue;
       }
       if (last) break;
       // 5. transition and auto-reset, inside the warp
@@ -658,7 +668,6 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
-  }  // group threads
 
   // ---- common exit: every thread arrives here; tensor memory is returned ----------------------
   tc_fence_before();
@@ -681,12 +690,12 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   if (err != cudaSuccess) return err;
   // Environments per tile: full tiles when there is enough work for every group of every SM,
   // otherwise smaller tiles so that all groups have one (the per-step chain is latency-bound).
-  const int slots = sms * S::GROUPS;
+  const int slots = sms * 2;  // two thread groups per CTA
   int ept = (h->cfg.n_envs + slots - 1) / slots;
   if (ept > S::EPT_MAX) ept = S::EPT_MAX;
   if (ept < 1) ept = 1;
   const int n_tiles = (h->cfg.n_envs + ept - 1) / ept;
-  const int ctas = (n_tiles + S::GROUPS - 1) / S::GROUPS;
+  const int ctas = (n_tiles + 1) / 2;
   kern<<<ctas < sms ? ctas : sms, S::THREADS, smem, h->stream>>>(args, static_cast<const unsigned char *>(h->d_wtc), ept,
                                                                  n_tiles);
   h->launches += 1;
