@@ -389,23 +389,27 @@ __device__ __forceinline__ void step_env_warp(EnvRegs<N, F> &s, const EnvParams 
                                               bool active, int action, float &reward, bool &done) {
   constexpr unsigned kFull = 0xFFFFFFFFu;
   const int G = p.grid;
+  // this lane's own agent: where it wants to go (0xFFFF: not moving, 0xFFFE: off the grid)
+  uint32_t my_pos = s.ent[0] & 0xFFFFu;
+#pragma unroll
+  for (int m = 1; m < N; ++m) my_pos = (ag == m) ? (s.ent[m] & 0xFFFFu) : my_pos;
+  uint32_t my_target;
+  {
+    const int r = my_pos & 0xFF, c = my_pos >> 8;
+    const int tr = r + (action == 2) - (action == 1), tc = c + (action == 4) - (action == 3);
+    const bool moving = action >= 1 && action <= 4;
+    const bool inside = tr >= 0 && tr < G && tc >= 0 && tc < G;
+    my_target = moving ? (inside ? (static_cast<uint32_t>(tr) | (static_cast<uint32_t>(tc) << 8)) : 0xFFFEu) : 0xFFFFu;
+  }
+  // everybody's action and target, one shuffle per agent
   int act[N];
-  uint32_t target[N];  // 0xFFFF: not moving
+  uint32_t target[N];
+  const uint32_t mine_packed = my_target | (static_cast<uint32_t>(action) << 16);
 #pragma unroll
   for (int m = 0; m < N; ++m) {
-    act[m] = __shfl_sync(kFull, action, base + m);
-    const int r = s.ent[m] & 0xFF, c = (s.ent[m] >> 8) & 0xFF;
-    const int tr = r + (act[m] == 2) - (act[m] == 1), tc = c + (act[m] == 4) - (act[m] == 3);
-    const bool moving = act[m] >= 1 && act[m] <= 4;
-    const bool inside = tr >= 0 && tr < G && tc >= 0 && tc < G;
-    target[m] = moving ? (inside ? (static_cast<uint32_t>(tr) | (static_cast<uint32_t>(tc) << 8)) : 0xFFFEu) : 0xFFFFu;
-  }
-  // this lane's own agent
-  uint32_t my_target = target[0], my_pos = s.ent[0] & 0xFFFFu;
-#pragma unroll
-  for (int m = 1; m < N; ++m) {
-    my_target = (ag == m) ? target[m] : my_target;
-    my_pos = (ag == m) ? (s.ent[m] & 0xFFFFu) : my_pos;
+    const uint32_t w = __shfl_sync(kFull, mine_packed, base + m);
+    act[m] = static_cast<int>(w >> 16);
+    target[m] = w & 0xFFFFu;
   }
   bool ok = my_target < 0xFFFEu;  // moving and inside the grid
 #pragma unroll

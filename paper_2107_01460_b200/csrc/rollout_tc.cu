@@ -67,6 +67,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+// Shared -> global bulk copy (both addresses 16-byte aligned, size a multiple of 16) and the wait
+// for its source to have been read, so that the shared memory may be reused.
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -467,6 +475,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const uint32_t bar = smem_u32(&sm.mma_bar[g]);
   float *stage = reinterpret_cast<float *>(gs.x);
   uint32_t phase = 0;
+  bool bulk_pending = false;  // thread 0 of a group: a bulk store of the observation block is in flight
   const size_t M = static_cast<size_t>(a.env.n_envs) * N;
   const int le = wg * S::EPW + lane / N;  // local environment of this lane
   const int ag = lane % N;                // its agent
@@ -501,6 +510,31 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       env.step = 0; env.episode = 0; env.total = 1;
     }
 
+    // Per-row outputs of a step wait in registers and go to global memory while the next step's
+    // layer 1 runs: a named barrier also waits for the stores issued before it, so stores placed
+    // right before one would put their round trip to L2 on the critical path.
+    bool pend = false, pend_step = false, pend_done = false;
+    size_t pend_row0 = 0, pend_done_idx = 0;
+    float pend_value = 0.0f, pend_logp = 0.0f, pend_reward = 0.0f, pend_logit[kActions];
+    int pend_action = 0;
+#pragma unroll
+    for (int k = 0; k < kActions; ++k) pend_logit[k] = 0.0f;
+    auto flush_outputs = [&]() {
+      if (pend && active) {
+        a.buf.values[pend_row0 + crow] = pend_value;
+        if (pend_step) {
+          a.buf.actions[pend_row0 + crow] = pend_action;
+          a.buf.logp[pend_row0 + crow] = pend_logp;
+          a.buf.rewards[pend_row0 + crow] = pend_reward;
+          if (ag == 0) a.buf.dones[pend_done_idx] = pend_done ? 1 : 0;
+          if (a.write_logits) {
+#pragma unroll
+            for (int k = 0; k < kActions; ++k) a.buf.logits[(pend_row0 + crow) * kActions + k] = pend_logit[k];
+          }
+        }
+      }
+      pend = false;
+    };
     for (int t = 0; t <= a.T; ++t) {
       const bool last = (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
@@ -541,13 +575,18 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         issue_layer<K1, H, !S::FOLD1, false>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF,
                                              w_addr + S::B1_OFF, bar);
       }
+      flush_outputs();  // the previous step's rows
       float *obs_dst = a.buf.obs + row0 * D;
       if (!last && !PP) {
         if (!TM) {  // one contiguous piece of the time-major array
+          // by the bulk-copy engine when alignment allows: it leaves the load/store pipe to the
+          // other group; the block was fenced for the async proxy together with the A tile
           const int count = n_rows * D;
           if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
-            for (int i = row; i < count / 4; i += kGroupThreads)
-              reinterpret_cast<float4 *>(obs_dst)[i] = reinterpret_cast<const float4 *>(stage)[i];
+            if (row == 0) {
+              bulk_store(obs_dst, smem_u32(stage), static_cast<uint32_t>(count) * 4u);
+              bulk_pending = true;
+            }
           } else {
             for (int i = row; i < count; i += kGroupThreads) obs_dst[i] = stage[i];
           }
@@ -558,9 +597,12 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       }
       float u = 0.0f;
       if (active && !last) u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag));
-      if (!TM) group_sync(g);  // every read of the block is done before the epilogue reuses its memory
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
+      if (!TM) {  // every read of the block is done before the epilogue reuses its memory
+        if (bulk_pending) { bulk_store_wait_read(); bulk_pending = false; }
+        group_sync(g);
+      }
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
       // layer 1 is done with A: zero it for the next step (ping-pong: the next user does that)
@@ -613,7 +655,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
           for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads)
             reinterpret_cast<uint4 *>(gs.x)[i] = make_uint4(0, 0, 0, 0);
         if (active) {
-          a.buf.values[row0 + crow] = hv[kActions];
+          pend = true; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
           if (!last) {
             float e[kActions];
             float m = hv[0];
@@ -638,12 +680,10 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
             float la = hv[0];
 #pragma unroll
             for (int k = 1; k < kActions; ++k) la = (action == k) ? hv[k] : la;
-            a.buf.actions[row0 + crow] = action;
-            a.buf.logp[row0 + crow] = la - m - __logf(sum);
-            if (a.write_logits) {
+            pend_action = action;
+            pend_logp = la - m - __logf(sum);
 #pragma unroll
-              for (int k = 0; k < kActions; ++k) a.buf.logits[(row0 + crow) * kActions + k] = hv[k];
-            }
+            for (int k = 0; k < kActions; ++k) pend_logit[k] = hv[k];
           }
         }
       }
@@ -660,15 +700,16 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       float reward;
       bool done;
       step_env_warp<N, F>(env, a.env, env_id, ag, base, active, action, reward, done);
-      if (active) {
-        a.buf.rewards[row0 + crow] = reward;
-        if (ag == 0) a.buf.dones[static_cast<size_t>(t) * a.env.n_envs + e0 + le] = done ? 1 : 0;
-      }
+      pend_reward = reward;
+      pend_done = done;
+      pend_done_idx = static_cast<size_t>(t) * a.env.n_envs + e0 + le;
     }
+    flush_outputs();  // the last step's rows (the bootstrap values among them)
     if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
 
+  bulk_store_wait_all();  // bulk stores of this thread, if any, have landed
   // ---- common exit: every thread arrives here; tensor memory is returned ----------------------
   tc_fence_before();
   __syncthreads();
