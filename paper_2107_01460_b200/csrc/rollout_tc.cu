@@ -75,6 +75,40 @@ __device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t byt
 }
 __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Explicit shared-window accesses (32-bit shared addresses).  Left to itself the compiler emits
+// generic loads and stores for pointers into the dynamic shared array, and a generic load that
+// follows this thread's global stores waits for them; these never do.
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ int lds_s32(uint32_t addr) {
+  int v;
+  asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint16_t v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void sts_zero16(uint32_t addr) {  // 16 bytes of zeros
+  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint16_t bf16_bits(float v) {
+  const __nv_bfloat16 b = __float2bfloat16_rn(v);
+  return *reinterpret_cast<const uint16_t *>(&b);
+}
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -166,10 +200,10 @@ struct TcShape {
   static constexpr uint32_t BT_BYTES = H * 16 * 2;
   static constexpr uint32_t B1_OFF = WH_OFF + WH_BYTES;
   static constexpr uint32_t B2_OFF = B1_OFF + (FOLD1 ? 0 : BT_BYTES);
-  static constexpr uint32_t BH_OFF = B2_OFF + BT_BYTES, BH_BYTES = kHeadRows * 16 * 2;
+  static constexpr uint32_t BH_OFF = B2_OFF + BT_BYTES, BH_BYTES = 32;  // 8 floats: ba[0..5], bv, 0
   static constexpr uint32_t ONES_OFF = BH_OFF + BH_BYTES, ONES_BYTES = kTileRows * 16 * 2;
   static constexpr uint32_t IMAGE_BYTES = ONES_OFF + ONES_BYTES;
-  static constexpr uint32_t A_BYTES = kTileRows * K1 * 2;
+  static constexpr uint32_t A_BYTES = (kTileRows / 8) * (K1 / 8) * 144;  // padded core-matrix pitch, see a_offset
   static constexpr uint32_t STAGE_BYTES = (kTileRows * D * 4 + 15) / 16 * 16;
   static constexpr uint32_t X_BYTES =
       TM ? 16 : (STAGE_BYTES > kTileRows * H * 2 ? STAGE_BYTES : kTileRows * H * 2);
@@ -217,6 +251,15 @@ __host__ __device__ constexpr uint32_t canon_offset(int n, int k, int K) {
   return static_cast<uint32_t>((n >> 3) * (K * 16) + (k >> 3) * 128 + (n & 7) * 16 + (k & 7) * 2);
 }
 
+// The A tile of layer 1 uses the same layout with the core matrices along K 144 instead of 128
+// bytes apart: the row-wise 2-byte accesses of the observation writer and of the obs copy-out
+// then spread over the banks instead of all landing on the four banks of one core-matrix row.
+constexpr uint32_t kALbo = 144;
+template <int K1>
+__host__ __device__ constexpr uint32_t a_offset(int r, int k) {
+  return static_cast<uint32_t>((r >> 3) * ((K1 / 8) * kALbo) + (k >> 3) * kALbo + (r & 7) * 16 + (k & 7) * 2);
+}
+
 __device__ __forceinline__ void split_bf16(float b, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
   hi = __float2bfloat16_rn(b);
   lo = __float2bfloat16_rn(b - __bfloat162float(hi));
@@ -249,8 +292,8 @@ __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *
     else if (n == kActions) v = params[L.Wv + k];
     at(S::WH_OFF)[canon_offset(n, k, H) / 2] = __float2bfloat16_rn(v);
   }
-  // bias tiles (hi, lo, then zeros) and the ones tile
-  for (int i = tid; i < (2 * H + kHeadRows) * 16; i += nth) {
+  // bias tiles of the hidden layers (hi, lo, then zeros), the heads' biases as fp32, the ones tile
+  for (int i = tid; i < 2 * H * 16; i += nth) {
     const int r = i / 16, k = i - r * 16;
     float b;
     uint32_t off;
@@ -258,17 +301,16 @@ __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *
     if (r < H) {
       if (S::FOLD1) continue;
       b = params[L.b1 + r]; off = S::B1_OFF; n = r;
-    } else if (r < 2 * H) {
-      b = params[L.b2 + r - H]; off = S::B2_OFF; n = r - H;
     } else {
-      n = r - 2 * H;
-      off = S::BH_OFF;
-      b = n < kActions ? params[L.ba + n] : (n == kActions ? params[L.bv] : 0.0f);
+      b = params[L.b2 + r - H]; off = S::B2_OFF; n = r - H;
     }
     __nv_bfloat16 hi, lo;
     split_bf16(b, hi, lo);
     at(off)[canon_offset(n, k, 16) / 2] = k == 0 ? hi : (k == 1 ? lo : __float2bfloat16_rn(0.0f));
   }
+  if (tid < 8)
+    reinterpret_cast<float *>(image + S::BH_OFF)[tid] =
+        tid < kActions ? params[L.ba + tid] : (tid == kActions ? params[L.bv] : 0.0f);
   for (int i = tid; i < kTileRows * 16; i += nth) {
     const int r = i / 16, k = i - r * 16;
     at(S::ONES_OFF)[canon_offset(r, k, 16) / 2] = __float2bfloat16_rn(k < 2 ? 1.0f : 0.0f);
@@ -315,7 +357,7 @@ __device__ __forceinline__ void relu_pack32(const uint32_t *r, uint32_t *packed)
 // layer, either in shared memory (canonical layout, K = H) or, packed two per column, in tensor
 // memory.  The load of the next 32 columns is in flight while the current 32 are converted.
 template <int H, bool TM>
-__device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, uint32_t hid_taddr, unsigned char *hbuf, int row) {
+__device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, uint32_t hid_taddr, uint32_t hbuf, int row) {
   static_assert(H % 64 == 0, "two 32-column batches per iteration");
   uint32_t ra[32], rb[32], pk[16];
   tmem_ld32_nowait(acc_taddr, ra);
@@ -329,8 +371,7 @@ __device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, uint32_t hid
     } else {
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 8 * q, H)) =
-            make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        sts_v4(hbuf + canon_offset(row, c0 + 8 * q, H), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
     }
     tmem_ld_wait();
     if (c0 + 64 < H) tmem_ld32_nowait(acc_taddr + static_cast<uint32_t>(c0 + 64), ra);
@@ -340,8 +381,7 @@ __device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, uint32_t hid
     } else {
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<uint4 *>(hbuf + canon_offset(row, c0 + 32 + 8 * q, H)) =
-            make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        sts_v4(hbuf + canon_offset(row, c0 + 32 + 8 * q, H), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
     }
   }
   if (TM) tmem_st_wait();
@@ -361,7 +401,7 @@ __device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, ui
 // One dense layer on the tensor core, issued by a single thread: the accumulator is seeded with
 // the bias (ones tile x bias tile, K = 16) unless the bias rides in the weights, and then
 // accumulates K / 16 steps of A x W^T, A from shared memory or from tensor memory.
-template <int K, int NOUT, bool BIAS_TILE, bool A_TMEM>
+template <int K, int NOUT, bool BIAS_TILE, bool A_TMEM, uint32_t A_LBO = 128>
 __device__ __forceinline__ void issue_layer(uint32_t d_tmem, uint32_t a_addr, uint32_t w_addr, uint32_t ones_addr,
                                             uint32_t bias_addr, uint32_t bar) {
   constexpr uint32_t idesc = instr_desc(kTileRows, NOUT);
@@ -370,7 +410,9 @@ __device__ __forceinline__ void issue_layer(uint32_t d_tmem, uint32_t a_addr, ui
   for (int k = 0; k < K / 16; ++k) {
     const uint32_t acc = (BIAS_TILE || k > 0) ? 1u : 0u;
     if (A_TMEM) mma_bf16_ts(d_tmem, a_addr + k * 8, smem_desc(w_addr + k * 256, 128, K * 16), idesc, acc);
-    else mma_bf16(d_tmem, smem_desc(a_addr + k * 256, 128, K * 16), smem_desc(w_addr + k * 256, 128, K * 16), idesc, acc);
+    else
+      mma_bf16(d_tmem, smem_desc(a_addr + k * 2 * A_LBO, A_LBO, (K / 8) * A_LBO), smem_desc(w_addr + k * 256, 128, K * 16),
+               idesc, acc);
   }
   mma_commit(bar);
 }
@@ -380,22 +422,22 @@ __device__ __forceinline__ void issue_layer(uint32_t d_tmem, uint32_t a_addr, ui
 // write consecutive floats.  The exact step/cap replaces the rounded bf16 one.  Four rows are in
 // flight at a time.
 template <int D, int K1>
-__device__ __forceinline__ void expand_rows(const unsigned char *a_tile, const float *step_frac, float *dst,
-                                            int first, int n, int tile_row0, int lane) {
+__device__ __forceinline__ void expand_rows(uint32_t a_tile, uint32_t step_frac, float *dst, int first, int n,
+                                            int tile_row0, int lane) {
   constexpr int Q = (D + 31) / 32;
   uint32_t off[Q];
 #pragma unroll
-  for (int q = 0; q < Q; ++q) off[q] = (static_cast<uint32_t>(lane + 32 * q) >> 3) * 128 + ((lane + 32 * q) & 7) * 2;
+  for (int q = 0; q < Q; ++q) off[q] = a_offset<K1>(0, lane + 32 * q);
   for (int l0 = 0; l0 < n; l0 += 4) {
-    uint16_t raw[4][Q];
+    uint32_t raw[4][Q];
     float sf[4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const int tr = tile_row0 + min(l0 + r, n - 1);
-      const unsigned char *arow = a_tile + (tr >> 3) * (K1 * 16) + (tr & 7) * 16;
+      const uint32_t arow = a_tile + a_offset<K1>(tr, 0);
 #pragma unroll
-      for (int q = 0; q < Q; ++q) raw[r][q] = (lane + 32 * q < D) ? *reinterpret_cast<const uint16_t *>(arow + off[q]) : 0;
-      sf[r] = step_frac[tr];
+      for (int q = 0; q < Q; ++q) raw[r][q] = (lane + 32 * q < D) ? lds_u16(arow + off[q]) : 0u;
+      sf[r] = lds_f32(step_frac + 4u * static_cast<uint32_t>(tr));
     }
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
@@ -404,8 +446,62 @@ __device__ __forceinline__ void expand_rows(const unsigned char *a_tile, const f
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
           const int j = lane + 32 * q;
-          if (j < D) orow[j] = (j == 3 * kPlane + 1) ? sf[r] : __uint_as_float(static_cast<uint32_t>(raw[r][q]) << 16);
+          if (j < D) orow[j] = (j == 3 * kPlane + 1) ? sf[r] : __uint_as_float(raw[r][q] << 16);
         }
+      }
+    }
+  }
+}
+
+// The same job for row counts that are multiples of four: four rows are one 16-byte aligned run
+// of 4*D floats, written as float4 by consecutive lanes.  Which (row of the four, column) a lane's
+// elements are does not depend on the quad, so their tile offsets are computed once.
+template <int D, int K1>
+struct QuadPlan {
+  static constexpr int V = (D + 31) / 32;  // float4 per lane per quad (D float4 in all)
+  uint32_t off[V][4];                      // byte offset inside the A tile relative to the quad's first row
+  uint32_t frac_row[V];                    // row (0..3) whose step/cap this lane's float4 may contain
+  bool is_frac[V][4];                      // element i of float4 v is a step/cap entry
+};
+template <int D, int K1>
+__device__ __forceinline__ void plan_quads(QuadPlan<D, K1> &p, int lane) {
+#pragma unroll
+  for (int v = 0; v < QuadPlan<D, K1>::V; ++v) {
+    p.frac_row[v] = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int f = 4 * (lane + 32 * v) + i;  // float index inside the quad (< 4*D when the lane takes part)
+      const int r = f / D, j = f - r * D;
+      p.off[v][i] = a_offset<K1>(r & 3, j);   // a quad starts at a multiple of four rows: no carry into the 8-row group
+      p.is_frac[v][i] = (j == 3 * kPlane + 1 && r < 4);
+      if (p.is_frac[v][i]) p.frac_row[v] = r;
+    }
+  }
+}
+// All loads of a quad are issued before the first use, so only one shared-memory latency is paid.
+template <int D, int K1>
+__device__ __forceinline__ void expand_quads(const QuadPlan<D, K1> &p, uint32_t a_tile, uint32_t step_frac, float *dst,
+                                             int first, int n, int tile_row0, int lane) {
+  constexpr int V = QuadPlan<D, K1>::V;
+  for (int l0 = 0; l0 < n; l0 += 4) {
+    const int tr = tile_row0 + l0;
+    const uint32_t qbase = a_tile + a_offset<K1>(tr, 0);
+    float4 *out = reinterpret_cast<float4 *>(dst + static_cast<size_t>(first + l0) * D);
+    uint32_t raw[V][4];
+    float sf[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) raw[v][i] = (lane + 32 * v < D) ? lds_u16(qbase + p.off[v][i]) : 0u;
+      sf[v] = lds_f32(step_frac + 4u * (static_cast<uint32_t>(tr) + p.frac_row[v]));
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      if (lane + 32 * v < D) {
+        float e[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) e[i] = p.is_frac[v][i] ? sf[v] : __uint_as_float(raw[v][i] << 16);
+        out[lane + 32 * v] = make_float4(e[0], e[1], e[2], e[3]);
       }
     }
   }
@@ -471,8 +567,10 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const uint32_t lane_off = static_cast<uint32_t>(wg * 32) << 16;  // this warp's TMEM lanes
   const uint32_t w_addr = smem_u32(sm.weights);
   const uint32_t a_addr = smem_u32(gs.a);
+  const uint32_t frac_addr = smem_u32(gs.step_frac), stage_addr = smem_u32(gs.x), abort_addr = smem_u32(&sm.abort);
   const uint32_t h_addr = TM ? hid_col : smem_u32(gs.x);  // A operand of layer 2 and of the heads
   const uint32_t bar = smem_u32(&sm.mma_bar[g]);
+  const float *head_bias = reinterpret_cast<const float *>(sm.weights + S::BH_OFF);
   float *stage = reinterpret_cast<float *>(gs.x);
   uint32_t phase = 0;
   bool bulk_pending = false;  // thread 0 of a group: a bulk store of the observation block is in flight
@@ -481,6 +579,8 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const int ag = lane % N;                // its agent
   const int crow = le * N + ag;           // compact row inside the tile's block
 
+  QuadPlan<D, K1> quad_plan;
+  if (PP && N % 4 == 0) plan_quads<D, K1>(quad_plan, lane);
   if (PP && g == 1) {  // group 0 goes first on both shared resources
     pair_arrive(kBarTile + 0);
     pair_arrive(kBarTmem + 0);
@@ -541,7 +641,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       if (PP) {
         pair_sync(kBarTile + g);  // the other group is done with the A tile
         // one verdict for the whole group (its threads may see the flag at different times)
-        idle = group_any(g, idle || *reinterpret_cast<volatile int *>(&sm.abort) != 0);
+        idle = group_any(g, idle || lds_s32(abort_addr) != 0);
         if (idle) {  // keep the hand-over order of a working step: tile, tensor memory, tile, tensor memory
           pair_sync(kBarTmem + g);
           pair_arrive(kBarTile + (1 - g));
@@ -550,18 +650,19 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         }
 #pragma unroll
         for (int kc = 0; kc < K1 / 8; ++kc)
-          *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
+          sts_zero16(a_addr + a_offset<K1>(row, kc * 8));
       }
       // 1. non-zero observation entries into the zeroed A tile (and the zeroed fp32 block)
       if (active) {
+        const uint32_t a_row = a_addr + a_offset<K1>(row, 0);
         observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
-          if (!TM) stage[crow * D + j] = v;
-          else if (j == 3 * kPlane + 1) gs.step_frac[row] = v;
-          *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, j, K1)) = __float2bfloat16_rn(v);
+          if (!TM) sts_f32(stage_addr + 4u * static_cast<uint32_t>(crow * D + j), v);
+          else if (j == 3 * kPlane + 1) sts_f32(frac_addr + 4u * static_cast<uint32_t>(row), v);
+          sts_u16(a_row + a_offset<K1>(0, j), bf16_bits(v));
         });
         if (S::FOLD1) {  // the two columns that pick up the bias rows of W1
-          *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, D, K1)) = __float2bfloat16_rn(1.0f);
-          *reinterpret_cast<__nv_bfloat16 *>(gs.a + canon_offset(row, D + 1, K1)) = __float2bfloat16_rn(1.0f);
+          sts_u16(a_row + a_offset<K1>(0, D), 0x3F80);
+          sts_u16(a_row + a_offset<K1>(0, D + 1), 0x3F80);
         }
       }
       fence_async_smem();
@@ -572,7 +673,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       //    block is not needed later) the observation block goes to obs[t]
       if (row == 0) {
         tc_fence_after();
-        issue_layer<K1, H, !S::FOLD1, false>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF,
+        issue_layer<K1, H, !S::FOLD1, false, kALbo>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF,
                                              w_addr + S::B1_OFF, bar);
       }
       flush_outputs();  // the previous step's rows
@@ -591,7 +692,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
             for (int i = row; i < count; i += kGroupThreads) obs_dst[i] = stage[i];
           }
         } else {  // this warp's rows, expanded from the bf16 tile
-          expand_rows<D, K1>(gs.a, gs.step_frac, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+          expand_rows<D, K1>(a_addr, frac_addr, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
           __syncwarp();
         }
       }
@@ -604,15 +705,14 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         group_sync(g);
       }
       tc_fence_after();
-      hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
+      hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, stage_addr, row);
       // layer 1 is done with A: zero it for the next step (ping-pong: the next user does that)
       if (TM && !PP) {  // own row only, its readers are in this warp
 #pragma unroll
         for (int kc = 0; kc < K1 / 8; ++kc)
-          *reinterpret_cast<uint4 *>(gs.a + canon_offset(row, kc * 8, K1)) = make_uint4(0, 0, 0, 0);
+          sts_zero16(a_addr + a_offset<K1>(row, kc * 8));
       } else if (!TM) {
-        for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads)
-          reinterpret_cast<uint4 *>(gs.a)[i] = make_uint4(0, 0, 0, 0);
+        for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads) sts_zero16(a_addr + 16u * i);
       }
       fence_async_smem();
       tc_fence_before();
@@ -623,22 +723,26 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         issue_layer<H, H, true, TM>(acc_col, h_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
       }
       if (PP) {
-        if (!last)
-          expand_rows<D, K1>(gs.a, gs.step_frac, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+        if (!last) {
+          if constexpr (N % 4 == 0)
+            expand_quads<D, K1>(quad_plan, a_addr, frac_addr, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW),
+                                wg * 32, lane);
+          else
+            expand_rows<D, K1>(a_addr, frac_addr, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+        }
         pair_arrive(kBarTile + (1 - g));  // this thread no longer needs the A tile
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       tc_fence_after();
-      hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, gs.x, row);
+      hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, stage_addr, row);
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
       // 4. heads: six logits and the value, N padded to 16
       if (row == 0) {
         tc_fence_after();
-        issue_layer<H, kHeadRows, true, TM>(head_col, h_addr, w_addr + S::WH_OFF, w_addr + S::ONES_OFF,
-                                            w_addr + S::BH_OFF, bar);
+        issue_layer<H, kHeadRows, false, TM>(head_col, h_addr, w_addr + S::WH_OFF, 0u, 0u, bar);
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
@@ -647,13 +751,14 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       {
         float hv[16];
         tmem_ld16(head_col + lane_off, hv);
+#pragma unroll
+        for (int k = 0; k <= kActions; ++k) hv[k] += head_bias[k];  // the heads' biases stay fp32
         if (PP) {  // this thread is done with tensor memory for this step
           tc_fence_before();
           pair_arrive(kBarTmem + (1 - g));
         }
         if (!TM)  // the hidden activations are dead: zero the observation block for the next step
-          for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads)
-            reinterpret_cast<uint4 *>(gs.x)[i] = make_uint4(0, 0, 0, 0);
+          for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
         if (active) {
           pend = true; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
           if (!last) {
