@@ -483,25 +483,34 @@ template <int D, int K1>
 __device__ __forceinline__ void expand_quads(const QuadPlan<D, K1> &p, uint32_t a_tile, uint32_t step_frac, float *dst,
                                              int first, int n, int tile_row0, int lane) {
   constexpr int V = QuadPlan<D, K1>::V;
-  for (int l0 = 0; l0 < n; l0 += 4) {
-    const int tr = tile_row0 + l0;
-    const uint32_t qbase = a_tile + a_offset<K1>(tr, 0);
-    float4 *out = reinterpret_cast<float4 *>(dst + static_cast<size_t>(first + l0) * D);
-    uint32_t raw[V][4];
-    float sf[V];
+  constexpr int U = 2;  // quads in flight
+  for (int l0 = 0; l0 < n; l0 += 4 * U) {
+    uint32_t raw[U][V][4];
+    float sf[U][V];
 #pragma unroll
-    for (int v = 0; v < V; ++v) {
+    for (int u = 0; u < U; ++u) {
+      const int tr = tile_row0 + min(l0 + 4 * u, n - 4);
+      const uint32_t qbase = a_tile + a_offset<K1>(tr, 0);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) raw[v][i] = (lane + 32 * v < D) ? lds_u16(qbase + p.off[v][i]) : 0u;
-      sf[v] = lds_f32(step_frac + 4u * (static_cast<uint32_t>(tr) + p.frac_row[v]));
+      for (int v = 0; v < V; ++v) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) raw[u][v][i] = (lane + 32 * v < D) ? lds_u16(qbase + p.off[v][i]) : 0u;
+        sf[u][v] = lds_f32(step_frac + 4u * (static_cast<uint32_t>(tr) + p.frac_row[v]));
+      }
     }
 #pragma unroll
-    for (int v = 0; v < V; ++v) {
-      if (lane + 32 * v < D) {
-        float e[4];
+    for (int u = 0; u < U; ++u) {
+      if (l0 + 4 * u < n) {
+        float4 *out = reinterpret_cast<float4 *>(dst + static_cast<size_t>(first + l0 + 4 * u) * D);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) e[i] = p.is_frac[v][i] ? sf[v] : __uint_as_float(raw[v][i] << 16);
-        out[lane + 32 * v] = make_float4(e[0], e[1], e[2], e[3]);
+        for (int v = 0; v < V; ++v) {
+          if (lane + 32 * v < D) {
+            float e[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) e[i] = p.is_frac[v][i] ? sf[u][v] : __uint_as_float(raw[u][v][i] << 16);
+            out[lane + 32 * v] = make_float4(e[0], e[1], e[2], e[3]);
+          }
+        }
       }
     }
   }
@@ -640,8 +649,9 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
       if (PP) {
         pair_sync(kBarTile + g);  // the other group is done with the A tile
-        // one verdict for the whole group (its threads may see the flag at different times)
-        idle = group_any(g, idle || lds_s32(abort_addr) != 0);
+        // one verdict for the whole group (its threads may see the flag at different times); the flag
+        // is looked at every eighth step only: the load would queue behind the partner's copy-out
+        idle = group_any(g, idle || ((t & 7) == 0 && lds_s32(abort_addr) != 0));
         if (idle) {  // keep the hand-over order of a working step: tile, tensor memory, tile, tensor memory
           pair_sync(kBarTmem + g);
           pair_arrive(kBarTile + (1 - g));
