@@ -52,10 +52,12 @@ int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_
   args.t_global0 = h->t_global;
   args.write_logits = (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) ? 1 : 0;
   args.status = h->d_status;
+  args.obs_last = h->d_obs_last;
   cudaError_t err;
   if (h->cfg.precision == MAVA_PRECISION_BF16) {
     err = launch_prep_tc(h, params_dev);
     if (err == cudaSuccess) err = launch_rollout_tc(h, args);
+    if (err == cudaSuccess && h->cfg.net_kind == MAVA_NET_CENTRAL_CRITIC) err = launch_critic_tc(h, params_dev, T);
   } else {
     err = launch_prep_simt(h, params_dev);
     if (err == cudaSuccess) err = launch_rollout_simt(h, args);
@@ -116,6 +118,10 @@ int mava_rollout_create(const mava_config_t *cfg, const mava_buffers_t *buffers,
             cudaMalloc(&h->d_params_stage, sizeof(float) * np) == cudaSuccess;
   if (ok && cfg->precision == MAVA_PRECISION_BF16)
     ok = cudaMalloc(&h->d_wtc, tc_weight_bytes(*cfg, h->D)) == cudaSuccess;
+  if (ok && cfg->precision == MAVA_PRECISION_BF16 && cfg->net_kind == MAVA_NET_CENTRAL_CRITIC)
+    ok = cudaMalloc(&h->d_critic, critic_weight_bytes(*cfg)) == cudaSuccess &&
+         cudaMalloc(&h->d_critic_h1, critic_hidden_bytes(*cfg)) == cudaSuccess &&
+         cudaMalloc(&h->d_obs_last, sizeof(float) * static_cast<size_t>(cfg->n_envs) * cfg->n_agents * h->D) == cudaSuccess;
   if (ok) ok = cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream) == cudaSuccess;
   if (ok) ok = launch_env_init(h) == cudaSuccess;
   if (ok) ok = cudaStreamSynchronize(h->stream) == cudaSuccess;
@@ -300,6 +306,7 @@ int mava_rollout_run_static(const mava_config_t *cfg, const mava_buffers_t *buff
   if (variant < 0) return MAVA_ERR_UNSUPPORTED;
   const bool bf16 = cfg->precision == MAVA_PRECISION_BF16;
   if (bf16 && !tc_supported(*cfg)) return MAVA_ERR_UNSUPPORTED;
+  if (bf16 && cfg->net_kind == MAVA_NET_CENTRAL_CRITIC) return MAVA_ERR_UNSUPPORTED;  // its scratch is far beyond the array
 
   // carve the scratch: status word | environment states | re-laid-out weights
   const int D = obs_dim(*cfg);
@@ -349,6 +356,9 @@ void mava_rollout_destroy(mava_rollout_t *h) {
   cudaFree(h->d_wsimt);
   cudaFree(h->d_wtc);
   cudaFree(h->d_params_stage);
+  cudaFree(h->d_critic);
+  cudaFree(h->d_critic_h1);
+  cudaFree(h->d_obs_last);
   delete h;
 }
 

@@ -46,6 +46,7 @@ struct RolloutArgs {
   uint32_t t_global0;
   int32_t write_logits;
   int *status;
+  float *obs_last;  // bf16 path with a centralised critic: where the observation after the last step goes
 };
 
 // Re-laid-out fp32 weights of the SIMT path: every dense layer transposed to [in][out].
@@ -68,6 +69,9 @@ struct mava_rollout {
   float *d_wsimt;   // transposed fp32 weights (SIMT path)
   void *d_wtc;      // bf16 weights in tensor-core layout (bf16 path)
   float *d_params_stage;  // device copy of host params (collect_host)
+  void *d_critic;      // centralised critic on the bf16 path: weight images,
+  void *d_critic_h1;   //   hidden activations of all environment-steps (bf16 tiles),
+  float *d_obs_last;   //   and the observations after the last step [E][N][D]
   uint32_t t_global;
   int32_t last_T;
   int64_t launches;
@@ -90,5 +94,8 @@ size_t tc_weight_bytes(const mava_config_t &cfg, int D);
 cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev);
 cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args);
 bool tc_supported(const mava_config_t &cfg);
+size_t critic_weight_bytes(const mava_config_t &cfg);
+size_t critic_hidden_bytes(const mava_config_t &cfg);
+cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T);
 
 }  // namespace mava

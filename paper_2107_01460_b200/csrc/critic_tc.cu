@@ -1,0 +1,376 @@
+// Centralised critic (MAPPO) on the tensor cores, as two batched kernels over the stored
+// trajectory: the critic's value does not feed the next environment step, so it is taken off the
+// rollout's serial chain and computed for all (T+1)*E environment-steps at once.
+//   layer-1 kernel: h1 = relu(X C1^T + c1), X = the N observations of an environment-step
+//     concatenated (N*D fp32, contiguous in the time-major obs array).  C1 (bf16, canonical K-major
+//     layout) stays in shared memory; each of two thread groups streams its 128-row tiles through
+//     two 48-column A buffers (fp32 -> bf16 on the way in) and leaves h1 as bf16 tiles, already in
+//     the operand layout, in a scratch array.
+//   layer-2 kernel: v = Cv relu(h1 C2^T + c2) + cv.  C2 stays in shared memory, the h1 tiles come
+//     in by bulk copies; two thread groups alternate tiles, one in its epilogue (ReLU, bf16
+//     rounding, dot product with Cv) while the other's MMAs run.  The value is written to the N
+//     slots of its environment-step.
+// Every mbarrier wait is bounded; a group that gives up records kStatusTimeout and leaves.
+#include "common.cuh"
+#include "layout.h"
+#include "tc_common.cuh"
+
+namespace mava {
+namespace {
+
+constexpr int kCH = 256;  // hidden width of the compiled critic
+
+template <int N>
+struct CriticShape {
+  static constexpr int D = kObsFixed + N;
+  static constexpr int KJ = N * D;                        // joint observation width
+  static constexpr int K1 = (KJ + 2 + 15) / 16 * 16;      // + two ones columns that carry c1
+  static constexpr int CHUNK = 48;                        // K columns per A buffer (3 MMA K steps)
+  static constexpr int NCHUNK = K1 / CHUNK;
+  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0, "chunking assumes float4 rows and whole chunks");
+  static constexpr uint32_t C1_BYTES = kCH * K1 * 2;
+  static constexpr uint32_t A_BUF_BYTES = kTileRows * CHUNK * 2;
+  static constexpr uint32_t A_SBO = (CHUNK / 8) * 128;
+  // layer-2 image: C2 | c2 bias tile | ones tile | Cv (bf16-rounded, as fp32) | cv
+  static constexpr uint32_t C2_OFF = 0, C2_BYTES = kCH * kCH * 2;
+  static constexpr uint32_t B2_OFF = C2_OFF + C2_BYTES, B2_BYTES = kCH * 16 * 2;
+  static constexpr uint32_t ONES_OFF = B2_OFF + B2_BYTES, ONES_BYTES = kTileRows * 16 * 2;
+  static constexpr uint32_t CV_OFF = ONES_OFF + ONES_BYTES, CV_BYTES = kCH * 4 + 16;
+  static constexpr uint32_t L2_BYTES = CV_OFF + CV_BYTES;
+  static constexpr uint32_t H1_TILE_BYTES = kTileRows * kCH * 2;
+  static constexpr uint32_t IMAGE_BYTES = C1_BYTES + L2_BYTES;
+};
+
+template <int N>
+__global__ void prep_critic_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, ParamLayout L) {
+  using S = CriticShape<N>;
+  constexpr int KJ = S::KJ, K1 = S::K1;
+  auto at = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(image + off); };
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  for (int i = tid; i < kCH * K1; i += nth) {
+    const int n = i / K1, k = i - n * K1;
+    __nv_bfloat16 v = __float2bfloat16_rn(k < KJ ? params[L.C1 + static_cast<size_t>(n) * KJ + k] : 0.0f);
+    if (k == KJ || k == KJ + 1) {
+      __nv_bfloat16 hi, lo;
+      split_bf16(params[L.c1 + n], hi, lo);
+      v = (k == KJ) ? hi : lo;
+    }
+    at(0)[canon_offset(n, k, K1) / 2] = v;
+  }
+  unsigned char *l2 = image + S::C1_BYTES;
+  auto at2 = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(l2 + off); };
+  for (int i = tid; i < kCH * kCH; i += nth) {
+    const int n = i / kCH, k = i - n * kCH;
+    at2(S::C2_OFF)[canon_offset(n, k, kCH) / 2] = __float2bfloat16_rn(params[L.C2 + static_cast<size_t>(n) * kCH + k]);
+  }
+  for (int i = tid; i < kCH * 16; i += nth) {
+    const int n = i / 16, k = i - n * 16;
+    __nv_bfloat16 hi, lo;
+    split_bf16(params[L.c2 + n], hi, lo);
+    at2(S::B2_OFF)[canon_offset(n, k, 16) / 2] = k == 0 ? hi : (k == 1 ? lo : __float2bfloat16_rn(0.0f));
+  }
+  for (int i = tid; i < kTileRows * 16; i += nth) {
+    const int r = i / 16, k = i - r * 16;
+    at2(S::ONES_OFF)[canon_offset(r, k, 16) / 2] = __float2bfloat16_rn(k < 2 ? 1.0f : 0.0f);
+  }
+  float *cv = reinterpret_cast<float *>(l2 + S::CV_OFF);
+  for (int i = tid; i <= kCH; i += nth)
+    cv[i] = i < kCH ? __bfloat162float(__float2bfloat16_rn(params[L.Cv + i])) : params[L.cv];
+}
+
+// ---- layer 1 -----------------------------------------------------------------------------------
+template <int N>
+struct CriticL1Smem {
+  using S = CriticShape<N>;
+  alignas(128) unsigned char c1[S::C1_BYTES];
+  alignas(128) unsigned char abuf[2][2][S::A_BUF_BYTES];  // [group][buffer]
+  alignas(8) uint64_t load_bar;
+  alignas(8) uint64_t mma_bar[2][2];
+  uint32_t tmem_base;
+};
+
+template <int N>
+__global__ void __launch_bounds__(2 * kGroupThreads, 1)
+critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_last, long long rows_main,
+                 long long rows_total, const unsigned char *__restrict__ image, unsigned char *__restrict__ h1, int n_tiles,
+                 int *status) {
+  using S = CriticShape<N>;
+  constexpr int KJ = S::KJ, K1 = S::K1, CHUNK = S::CHUNK, NCHUNK = S::NCHUNK, V = CHUNK / 4;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  CriticL1Smem<N> &sm = *reinterpret_cast<CriticL1Smem<N> *>(smem_raw);
+  const int tid = threadIdx.x, g = tid / kGroupThreads, row = tid % kGroupThreads, warp = tid / 32;
+  if (tid == 0) {
+    mbar_init(smem_u32(&sm.load_bar), 1);
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm.mma_bar[i / 2][i % 2]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (tid == 0) {
+    const uint32_t bar = smem_u32(&sm.load_bar);
+    mbar_expect_tx(bar, S::C1_BYTES);
+    constexpr uint32_t kChunk = 16384;
+    for (uint32_t off = 0; off < S::C1_BYTES; off += kChunk)
+      bulk_load(smem_u32(sm.c1 + off), image + off, S::C1_BYTES - off < kChunk ? S::C1_BYTES - off : kChunk, bar);
+  }
+  bool timed_out = !mbar_wait(smem_u32(&sm.load_bar), 0);
+  timed_out = __syncthreads_or(timed_out) != 0;
+
+  const uint32_t tmem_base = sm.tmem_base;
+  const uint32_t acc = tmem_base + static_cast<uint32_t>(g * kCH);
+  const uint32_t lane_off = static_cast<uint32_t>((row / 32) * 32) << 16;
+  const uint32_t c1_addr = smem_u32(sm.c1);
+  const uint32_t abuf0 = smem_u32(sm.abuf[g][0]);  // buffer b at abuf0 + b * A_BUF_BYTES
+  const uint32_t bar0 = smem_u32(&sm.mma_bar[g][0]);  // its barrier at bar0 + 8 b
+  uint32_t waits0 = 0, waits1 = 0;  // completed waits per buffer: the next wait's parity
+  auto wait_buffer = [&](int b) {
+    const uint32_t parity = (b ? waits1 : waits0) & 1u;
+    const bool ok = mbar_wait(bar0 + 8u * b, parity);
+    if (b) waits1 += 1; else waits0 += 1;
+    return ok;
+  };
+
+  for (int tile = blockIdx.x * 2 + g; tile < n_tiles && !timed_out; tile += gridDim.x * 2) {
+    const long long r_idx = static_cast<long long>(tile) * kTileRows + row;
+    const bool valid = r_idx < rows_total;
+    const float *src = obs;
+    if (valid) src = r_idx < rows_main ? obs + r_idx * KJ : obs_last + (r_idx - rows_main) * KJ;
+    auto load_chunk = [&](int c, float4 *dst) {
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        const int k = c * CHUNK + 4 * v;
+        dst[v] = (valid && k < KJ) ? __ldg(reinterpret_cast<const float4 *>(src + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    float4 cur[V], nxt[V];
+    load_chunk(0, cur);
+#pragma unroll 1
+    for (int c = 0; c < NCHUNK; ++c) {
+      if (c + 1 < NCHUNK) load_chunk(c + 1, nxt);
+      const int b = c & 1;
+      const uint32_t abuf = abuf0 + static_cast<uint32_t>(b) * S::A_BUF_BYTES;
+      if (c >= 2) timed_out |= !wait_buffer(b);  // the MMAs of chunk c-2 have finished reading this buffer
+      if (valid && c == NCHUNK - 1) {  // the two ones columns that pick up c1
+        constexpr int o = KJ - (NCHUNK - 1) * CHUNK;
+        static_assert(o % 4 == 0 && o + 1 < CHUNK, "ones columns inside the last chunk, at the start of a float4");
+        cur[o / 4].x = 1.0f;
+        cur[o / 4].y = 1.0f;
+      }
+#pragma unroll
+      for (int kc = 0; kc < CHUNK / 8; ++kc) {
+        const float4 lo = cur[2 * kc], hi = cur[2 * kc + 1];
+        sts_v4(abuf + (row >> 3) * S::A_SBO + kc * 128 + (row & 7) * 16, pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w),
+               pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
+      }
+      fence_async_smem();
+      tc_fence_before();
+      group_sync(g);
+      if (row == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < CHUNK / 16; ++j)
+          mma_bf16(acc, smem_desc(abuf + j * 256, 128, S::A_SBO),
+                   smem_desc(c1_addr + (c * (CHUNK / 16) + j) * 256, 128, K1 * 16), instr_desc(kTileRows, kCH),
+                   (c > 0 || j > 0) ? 1u : 0u);
+        mma_commit(bar0 + 8u * b);
+      }
+#pragma unroll
+      for (int v = 0; v < V; ++v) cur[v] = nxt[v];
+    }
+    // the last two chunks are still outstanding, one per buffer
+    timed_out |= !wait_buffer(NCHUNK & 1);
+    timed_out |= !wait_buffer((NCHUNK + 1) & 1);
+    tc_fence_after();
+    // epilogue: ReLU, bf16, the row goes out in the operand layout of layer 2
+    unsigned char *tile_out = h1 + static_cast<size_t>(tile) * S::H1_TILE_BYTES;
+    uint32_t ra[32], pk[16];
+#pragma unroll 1
+    for (int c0 = 0; c0 < kCH; c0 += 32) {
+      tmem_ld32_nowait(acc + lane_off + static_cast<uint32_t>(c0), ra);
+      tmem_ld_wait();
+      relu_pack32(ra, pk);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4 *>(tile_out + canon_offset(row, c0 + 8 * q, kCH)) =
+            make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+    }
+    tc_fence_before();
+    if (group_any(g, timed_out)) timed_out = true;
+  }
+  if (timed_out && row == 0) atomicExch(status, kStatusTimeout);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+// ---- layer 2 and the value head ----------------------------------------------------------------
+template <int N>
+struct CriticL2Smem {
+  using S = CriticShape<N>;
+  alignas(128) unsigned char w[S::L2_BYTES];
+  alignas(128) unsigned char a[S::H1_TILE_BYTES];
+  alignas(8) uint64_t w_bar;
+  alignas(8) uint64_t load_bar[2];  // round k's tile completes load_bar[k % 2]: each group has its own
+  alignas(8) uint64_t mma_bar[2];
+  uint32_t tmem_base;
+};
+
+template <int N>
+__global__ void __launch_bounds__(2 * kGroupThreads, 1)
+critic_l2_kernel(const unsigned char *__restrict__ h1, const unsigned char *__restrict__ image, float *__restrict__ values,
+                 long long rows_total, int n_tiles, int *status) {
+  using S = CriticShape<N>;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  CriticL2Smem<N> &sm = *reinterpret_cast<CriticL2Smem<N> *>(smem_raw);
+  const int tid = threadIdx.x, g = tid / kGroupThreads, row = tid % kGroupThreads, warp = tid / 32;
+  const uint32_t load_bar0 = smem_u32(&sm.load_bar[0]);
+  auto load_tile = [&](int tile, int round) {  // one thread: the tile's 64 KB in four bulk copies
+    const uint32_t lb = load_bar0 + 8u * (round & 1);
+    mbar_expect_tx(lb, S::H1_TILE_BYTES);
+    for (uint32_t off = 0; off < S::H1_TILE_BYTES; off += 16384)
+      bulk_load(smem_u32(sm.a + off), h1 + static_cast<size_t>(tile) * S::H1_TILE_BYTES + off, 16384, lb);
+  };
+  if (tid == 0) {
+    mbar_init(smem_u32(&sm.w_bar), 1);
+    mbar_init(load_bar0, 1);
+    mbar_init(load_bar0 + 8, 1);
+    mbar_init(smem_u32(&sm.mma_bar[0]), 1);
+    mbar_init(smem_u32(&sm.mma_bar[1]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (tid == 0) {
+    const uint32_t bar = smem_u32(&sm.w_bar);
+    mbar_expect_tx(bar, S::L2_BYTES);
+    for (uint32_t off = 0; off < S::L2_BYTES; off += 16384)
+      bulk_load(smem_u32(sm.w + off), image + off, S::L2_BYTES - off < 16384 ? S::L2_BYTES - off : 16384, bar);
+    if (static_cast<int>(blockIdx.x) < n_tiles) load_tile(blockIdx.x, 0);  // round 0 belongs to group 0
+  }
+  bool timed_out = !mbar_wait(smem_u32(&sm.w_bar), 0);
+  timed_out = __syncthreads_or(timed_out) != 0;
+
+  const uint32_t tmem_base = sm.tmem_base;
+  const uint32_t acc = tmem_base + static_cast<uint32_t>(g * kCH);
+  const uint32_t lane_off = static_cast<uint32_t>((row / 32) * 32) << 16;
+  const uint32_t w_addr = smem_u32(sm.w), a_addr = smem_u32(sm.a), cv_addr = w_addr + S::CV_OFF;
+  const uint32_t mma_bar = smem_u32(&sm.mma_bar[g]);
+
+  // round k of this CTA works on tile blockIdx.x + k * gridDim.x and belongs to group k % 2
+  for (int k = g; !timed_out; k += 2) {
+    const int tile = blockIdx.x + k * static_cast<int>(gridDim.x);
+    if (tile >= n_tiles) break;
+    timed_out |= !mbar_wait(load_bar0 + 8u * g, (k >> 1) & 1);  // this round's tile has landed
+    if (row == 0 && !timed_out) {
+      tc_fence_after();
+      constexpr uint32_t idesc = instr_desc(kTileRows, kCH);
+      mma_bf16(acc, smem_desc(w_addr + S::ONES_OFF, 128, 256), smem_desc(w_addr + S::B2_OFF, 128, 256), idesc, 0);
+#pragma unroll
+      for (int j = 0; j < kCH / 16; ++j)
+        mma_bf16(acc, smem_desc(a_addr + j * 256, 128, kCH * 16), smem_desc(w_addr + S::C2_OFF + j * 256, 128, kCH * 16),
+                 idesc, 1);
+      mma_commit(mma_bar);
+    }
+    if (!timed_out) timed_out |= !mbar_wait(mma_bar, (k >> 1) & 1);
+    // the tile buffer is free: fetch the next round's tile (the other group's) behind this epilogue
+    if (row == 0 && !timed_out && tile + static_cast<int>(gridDim.x) < n_tiles) load_tile(tile + gridDim.x, k + 1);
+    tc_fence_after();
+    float v = 0.0f;
+    uint32_t ra[32];
+#pragma unroll 1
+    for (int c0 = 0; c0 < kCH; c0 += 32) {
+      tmem_ld32_nowait(acc + lane_off + static_cast<uint32_t>(c0), ra);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const uint32_t p = relu_pack_bf16(ra[2 * i], ra[2 * i + 1]);  // h2 rounded to bf16, as the operands of the head are
+        v = fmaf(__uint_as_float(p << 16), lds_f32(cv_addr + 4u * (c0 + 2 * i)), v);
+        v = fmaf(__uint_as_float(p & 0xFFFF0000u), lds_f32(cv_addr + 4u * (c0 + 2 * i + 1)), v);
+      }
+    }
+    v += lds_f32(cv_addr + 4u * kCH);
+    const long long r_idx = static_cast<long long>(tile) * kTileRows + row;
+    if (r_idx < rows_total && !timed_out) {
+      float *out = values + r_idx * N;
+#pragma unroll
+      for (int n = 0; n < N; ++n) out[n] = v;
+    }
+    tc_fence_before();
+    if (group_any(g, timed_out)) timed_out = true;
+  }
+  if (timed_out && row == 0) atomicExch(status, kStatusTimeout);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+}  // namespace
+
+size_t critic_weight_bytes(const mava_config_t &cfg) {
+  return find_variant(cfg) == 3 ? CriticShape<4>::IMAGE_BYTES : 16;
+}
+
+size_t critic_hidden_bytes(const mava_config_t &cfg) {
+  if (find_variant(cfg) != 3) return 16;
+  const long long rows = static_cast<long long>(cfg.max_T + 1) * cfg.n_envs;
+  return static_cast<size_t>((rows + kTileRows - 1) / kTileRows) * CriticShape<4>::H1_TILE_BYTES;
+}
+
+cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T) {
+  if (h->variant != 3 || !h->d_critic || !h->d_critic_h1 || !h->d_obs_last) return cudaErrorNotSupported;
+  using S = CriticShape<4>;
+  unsigned char *image = static_cast<unsigned char *>(h->d_critic);
+  prep_critic_kernel<4><<<128, 256, 0, h->stream>>>(params_dev, image, param_layout(h->cfg, h->D, 1));
+  h->launches += 1;
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  int sms = 0;
+  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+  if (err != cudaSuccess) return err;
+  const long long rows_main = static_cast<long long>(T) * h->cfg.n_envs, rows_total = rows_main + h->cfg.n_envs;
+  const int n_tiles = static_cast<int>((rows_total + kTileRows - 1) / kTileRows);
+  {
+    auto kern = critic_l1_kernel<4>;
+    const size_t smem = sizeof(CriticL1Smem<4>);
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+    const int ctas = (n_tiles + 1) / 2 < sms ? (n_tiles + 1) / 2 : sms;
+    kern<<<ctas, 2 * kGroupThreads, smem, h->stream>>>(h->buf.obs, h->d_obs_last, rows_main, rows_total, image,
+                                                       static_cast<unsigned char *>(h->d_critic_h1), n_tiles, h->d_status);
+    h->launches += 1;
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+  }
+  {
+    auto kern = critic_l2_kernel<4>;
+    const size_t smem = sizeof(CriticL2Smem<4>);
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+    const int ctas = n_tiles < sms ? n_tiles : sms;
+    kern<<<ctas, 2 * kGroupThreads, smem, h->stream>>>(static_cast<const unsigned char *>(h->d_critic_h1), image + S::C1_BYTES,
+                                                       h->buf.values, rows_total, n_tiles, h->d_status);
+    h->launches += 1;
+    err = cudaGetLastError();
+  }
+  return err;
+}
+
+}  // namespace mava

@@ -26,159 +26,11 @@
 #include "common.cuh"
 #include "env.cuh"
 #include "layout.h"
+#include "tc_common.cuh"
 
 namespace mava {
 namespace {
 
-constexpr int kGroupThreads = 128;
-constexpr int kTileRows = 128;       // M of every MMA
-constexpr int kHeadRows = 16;        // heads padded to the smallest N the MMA takes at M = 128
-constexpr uint32_t kSpinLimit = 1u << 22;
-
-// ---- PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-// Shared -> global bulk copy (both addresses 16-byte aligned, size a multiple of 16) and the wait
-// for its source to have been read, so that the shared memory may be reused.
-__device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// Explicit shared-window accesses (32-bit shared addresses).  Left to itself the compiler emits
-// generic loads and stores for pointers into the dynamic shared array, and a generic load that
-// follows this thread's global stores waits for them; these never do.
-__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
-  uint16_t v;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ float lds_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ int lds_s32(uint32_t addr) {
-  int v;
-  asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ void sts_u16(uint32_t addr, uint16_t v) {
-  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
-}
-__device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
-  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void sts_zero16(uint32_t addr) {  // 16 bytes of zeros
-  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
-}
-__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ uint16_t bf16_bits(float v) {
-  const __nv_bfloat16 b = __float2bfloat16_rn(v);
-  return *reinterpret_cast<const uint16_t *>(&b);
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void group_sync(int g) {
-  asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "r"(kGroupThreads) : "memory");
-}
-// Producer/consumer halves of a named barrier shared by the two thread groups of a CTA.
-__device__ __forceinline__ void pair_arrive(int id) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
-}
-__device__ __forceinline__ void pair_sync(int id) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
-}
-// Ping-pong hand-over barriers (ids 1..2 belong to the groups): group g waits on kBar* + g for
-// the A tile / the tensor-memory columns, and the other group arrives there when it lets go.
-constexpr int kBarTile = 8, kBarTmem = 10;
-// Barrier of the group that also ORs a predicate over its threads.
-__device__ __forceinline__ bool group_any(int g, bool pred) {
-  uint32_t out;
-  asm volatile(
-      "{\n.reg .pred p, q;\n"
-      "setp.ne.u32 p, %1, 0;\n"
-      "barrier.cta.red.or.pred q, %2, %3, p;\n"
-      "selp.u32 %0, 1, 0, q;\n}"
-      : "=r"(out)
-      : "r"(static_cast<uint32_t>(pred)), "r"(g + 1), "r"(kGroupThreads)
-      : "memory");
-  return out != 0;
-}
-
-// Shared-memory matrix descriptor, no swizzle, K-major: core matrices of 8 rows x 16 bytes;
-// lbo = byte step between core matrices along K, sbo = byte step between 8-row groups.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16) |
-         (static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
-}
-// Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, both K-major, M x N.
-__host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
-         (static_cast<uint32_t>(m >> 4) << 24);
-}
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 32 lanes x 32 bit, 16 consecutive columns: thread i of the warp reads lane (lane base + i).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);  // .x = lo (low half), .y = hi
-  return *reinterpret_cast<const uint32_t *>(&b);
-}
 
 // ---- shapes ------------------------------------------------------------------------------------
 template <int N, int H, bool TM>
@@ -244,28 +96,8 @@ struct TcSmem {
   int abort;  // ping-pong mode: a group gave up; both finish their barrier protocol without work
 };
 
-// ---- weight image ------------------------------------------------------------------------------
-// Byte offset of element (n, k) of an N x K bf16 operand in the canonical no-swizzle K-major
-// layout used here: 8-row groups are K*16 bytes apart, core matrices along K 128 bytes apart.
-__host__ __device__ constexpr uint32_t canon_offset(int n, int k, int K) {
-  return static_cast<uint32_t>((n >> 3) * (K * 16) + (k >> 3) * 128 + (n & 7) * 16 + (k & 7) * 2);
-}
 
-// The A tile of layer 1 uses the same layout with the core matrices along K 144 instead of 128
-// bytes apart: the row-wise 2-byte accesses of the observation writer and of the obs copy-out
-// then spread over the banks instead of all landing on the four banks of one core-matrix row.
-constexpr uint32_t kALbo = 144;
-template <int K1>
-__host__ __device__ constexpr uint32_t a_offset(int r, int k) {
-  return static_cast<uint32_t>((r >> 3) * ((K1 / 8) * kALbo) + (k >> 3) * kALbo + (r & 7) * 16 + (k & 7) * 2);
-}
-
-__device__ __forceinline__ void split_bf16(float b, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
-  hi = __float2bfloat16_rn(b);
-  lo = __float2bfloat16_rn(b - __bfloat162float(hi));
-}
-
-template <int N, int H, bool TM>
+template <int N, int H, bool TM, bool CENTRAL>
 __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, ParamLayout L) {
   using S = TcShape<N, H, TM>;
   constexpr int D = S::D, K1 = S::K1;
@@ -289,7 +121,7 @@ __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *
     const int n = i / H, k = i - n * H;
     float v = 0.0f;
     if (n < kActions) v = params[L.Wa + static_cast<size_t>(n) * H + k];
-    else if (n == kActions) v = params[L.Wv + k];
+    else if (n == kActions && !CENTRAL) v = params[L.Wv + k];  // the centralised critic has its own kernels
     at(S::WH_OFF)[canon_offset(n, k, H) / 2] = __float2bfloat16_rn(v);
   }
   // bias tiles of the hidden layers (hi, lo, then zeros), the heads' biases as fp32, the ones tile
@@ -310,47 +142,13 @@ __global__ void prep_tc_kernel(const float *__restrict__ params, unsigned char *
   }
   if (tid < 8)
     reinterpret_cast<float *>(image + S::BH_OFF)[tid] =
-        tid < kActions ? params[L.ba + tid] : (tid == kActions ? params[L.bv] : 0.0f);
+        tid < kActions ? params[L.ba + tid] : ((tid == kActions && !CENTRAL) ? params[L.bv] : 0.0f);
   for (int i = tid; i < kTileRows * 16; i += nth) {
     const int r = i / 16, k = i - r * 16;
     at(S::ONES_OFF)[canon_offset(r, k, 16) / 2] = __float2bfloat16_rn(k < 2 ? 1.0f : 0.0f);
   }
 }
 
-// ---- tensor-memory helpers ---------------------------------------------------------------------
-// 32 lanes x 32 bit, 32 consecutive columns (no wait: the caller waits once per batch of loads).
-__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,"
-      "%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Thread i of the warp writes 16 consecutive 32-bit columns of lane (lane base + i).
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// max(x, 0) of two fp32 values rounded to bf16 and packed (lo in the low half).
-__device__ __forceinline__ uint32_t relu_pack_bf16(uint32_t lo_bits, uint32_t hi_bits) {
-  uint32_t d;
-  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(hi_bits)), "f"(__uint_as_float(lo_bits)));
-  return d;
-}
-__device__ __forceinline__ void relu_pack32(const uint32_t *r, uint32_t *packed) {
-#pragma unroll
-  for (int i = 0; i < 16; ++i) packed[i] = relu_pack_bf16(r[2 * i], r[2 * i + 1]);
-}
 
 // Epilogue of a hidden layer: thread `row` reads its accumulator row (bias already inside) from
 // tensor memory, applies ReLU and rounds to bf16; the row becomes the A operand of the next
@@ -387,16 +185,6 @@ __device__ __forceinline__ void hidden_epilogue(uint32_t acc_taddr, uint32_t hid
   if (TM) tmem_st_wait();
 }
 
-// A from tensor memory (lane = row, two bf16 per 32-bit column, 8 columns per K step of 16).
-__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 
 // One dense layer on the tensor core, issued by a single thread: the accumulator is seeded with
 // the bias (ones tile x bias tile, K = 16) unless the bias rides in the weights, and then
@@ -733,12 +521,13 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         issue_layer<H, H, true, TM>(acc_col, h_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
       }
       if (PP) {
-        if (!last) {
+        if (!last || a.obs_last != nullptr) {  // the observation after the last step feeds a centralised critic
+          float *dst = last ? a.obs_last + static_cast<size_t>(e0) * N * D : obs_dst;
           if constexpr (N % 4 == 0)
-            expand_quads<D, K1>(quad_plan, a_addr, frac_addr, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW),
-                                wg * 32, lane);
+            expand_quads<D, K1>(quad_plan, a_addr, frac_addr, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32,
+                                lane);
           else
-            expand_rows<D, K1>(a_addr, frac_addr, obs_dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+            expand_rows<D, K1>(a_addr, frac_addr, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
         }
         pair_arrive(kBarTile + (1 - g));  // this thread no longer needs the A tile
       }
@@ -858,9 +647,9 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   return cudaGetLastError();
 }
 
-template <int N, int H, bool TM>
+template <int N, int H, bool TM, bool CENTRAL = false>
 cudaError_t launch_prep_variant(mava_rollout *h, const float *params_dev) {
-  prep_tc_kernel<N, H, TM><<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(h->d_wtc),
+  prep_tc_kernel<N, H, TM, CENTRAL><<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(h->d_wtc),
                                                      param_layout(h->cfg, h->D, 1));
   h->launches += 1;
   return cudaGetLastError();
@@ -868,21 +657,22 @@ cudaError_t launch_prep_variant(mava_rollout *h, const float *params_dev) {
 
 }  // namespace
 
-// Shared-torso shapes run on the tensor cores; the centralised critic does not yet.
+// All compiled shapes run on the tensor cores (the centralised critic through critic_tc.cu).
 bool tc_supported(const mava_config_t &cfg) {
   const int v = find_variant(cfg);
-  return v == 0 || v == 1 || v == 2 || v == 4;
+  return v == 0 || v == 1 || v == 2 || v == 3 || v == 4;
 }
 
 // Hidden activations in tensor memory: always for H = 256; for the smaller shapes only when the
 // handle asks for it (MAVA_FLAG_HIDDEN_IN_TMEM), which lets small cases exercise that path.
-static bool use_tm(const mava_rollout *h) { return h->variant == 4 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0; }
+static bool use_tm(const mava_rollout *h) { return h->variant >= 3 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0; }
 
 size_t tc_weight_bytes(const mava_config_t &cfg, int) {
   switch (find_variant(cfg)) {  // the two layouts of a shape have the same image size
     case 0: return TcShape<2, 64, false>::IMAGE_BYTES;
     case 1: return TcShape<2, 128, false>::IMAGE_BYTES;
     case 2: return TcShape<3, 128, false>::IMAGE_BYTES;
+    case 3: return TcShape<4, 256, true>::IMAGE_BYTES;
     case 4: return TcShape<8, 256, true>::IMAGE_BYTES;
     default: return 16;
   }
@@ -893,6 +683,7 @@ cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev) {
     case 0: return launch_prep_variant<2, 64, false>(h, params_dev);
     case 1: return launch_prep_variant<2, 128, false>(h, params_dev);
     case 2: return launch_prep_variant<3, 128, false>(h, params_dev);
+    case 3: return launch_prep_variant<4, 256, true, true>(h, params_dev);
     case 4: return launch_prep_variant<8, 256, true>(h, params_dev);
     default: return cudaErrorNotSupported;
   }
@@ -904,6 +695,7 @@ cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args) {
     case 0: return tm ? launch_tc_variant<2, 2, 64, true>(h, args) : launch_tc_variant<2, 2, 64, false>(h, args);
     case 1: return tm ? launch_tc_variant<2, 2, 128, true>(h, args) : launch_tc_variant<2, 2, 128, false>(h, args);
     case 2: return tm ? launch_tc_variant<3, 3, 128, true>(h, args) : launch_tc_variant<3, 3, 128, false>(h, args);
+    case 3: return launch_tc_variant<4, 5, 256, true>(h, args);
     case 4: return launch_tc_variant<8, 8, 256, true>(h, args);
     default: return cudaErrorNotSupported;
   }
