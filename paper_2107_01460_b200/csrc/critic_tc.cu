@@ -27,7 +27,8 @@ struct CriticShape {
   static constexpr int K1 = (KJ + 2 + 15) / 16 * 16;      // + two ones columns that carry c1
   static constexpr int CHUNK = 48;                        // K columns per A buffer (3 MMA K steps)
   static constexpr int NCHUNK = K1 / CHUNK;
-  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0, "chunking assumes float4 rows and whole chunks");
+  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0 && (kTileRows * (CHUNK / 4)) % kGroupThreads == 0,
+                "chunking assumes float4 rows, whole chunks and an even split of a chunk over the group");
   static constexpr uint32_t C1_BYTES = kCH * K1 * 2;
   static constexpr uint32_t A_BUF_BYTES = kTileRows * CHUNK * 2;
   static constexpr uint32_t A_SBO = (CHUNK / 8) * 128;
@@ -137,15 +138,27 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
   };
 
   for (int tile = blockIdx.x * 2 + g; tile < n_tiles && !timed_out; tile += gridDim.x * 2) {
-    const long long r_idx = static_cast<long long>(tile) * kTileRows + row;
-    const bool valid = r_idx < rows_total;
-    const float *src = obs;
-    if (valid) src = r_idx < rows_main ? obs + r_idx * KJ : obs_last + (r_idx - rows_main) * KJ;
+    // Coalesced loading: float4 number i = row + 128 q of a chunk is (tile row i / V, float4 i % V
+    // of that row's CHUNK columns), so consecutive threads read consecutive 16 bytes of a row.
+    const float *ptr[V];  // address of that float4 in chunk 0 (nullptr: the row is past the end)
+    uint32_t soff[V];     // its place in an A buffer
+#pragma unroll
+    for (int q = 0; q < V; ++q) {
+      const int i = row + kGroupThreads * q, r = i / V, v = i - r * V;
+      const long long r_idx = static_cast<long long>(tile) * kTileRows + r;
+      ptr[q] = nullptr;
+      if (r_idx < rows_total) ptr[q] = (r_idx < rows_main ? obs + r_idx * KJ : obs_last + (r_idx - rows_main) * KJ) + 4 * v;
+      soff[q] = static_cast<uint32_t>((r >> 3) * S::A_SBO + ((4 * v) >> 3) * 128 + (r & 7) * 16 + ((4 * v) & 7) * 2);
+    }
     auto load_chunk = [&](int c, float4 *dst) {
 #pragma unroll
-      for (int v = 0; v < V; ++v) {
-        const int k = c * CHUNK + 4 * v;
-        dst[v] = (valid && k < KJ) ? __ldg(reinterpret_cast<const float4 *>(src + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int q = 0; q < V; ++q) {
+        const int v = (row + kGroupThreads * q) % V, k = c * CHUNK + 4 * v;
+        dst[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ptr[q] != nullptr) {
+          if (k < KJ) dst[q] = __ldg(reinterpret_cast<const float4 *>(ptr[q] + c * CHUNK));
+          else if (k == KJ) dst[q] = make_float4(1.f, 1.f, 0.f, 0.f);  // the two ones columns that pick up c1
+        }
       }
     };
     float4 cur[V], nxt[V];
@@ -156,18 +169,11 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
       const int b = c & 1;
       const uint32_t abuf = abuf0 + static_cast<uint32_t>(b) * S::A_BUF_BYTES;
       if (c >= 2) timed_out |= !wait_buffer(b);  // the MMAs of chunk c-2 have finished reading this buffer
-      if (valid && c == NCHUNK - 1) {  // the two ones columns that pick up c1
-        constexpr int o = KJ - (NCHUNK - 1) * CHUNK;
-        static_assert(o % 4 == 0 && o + 1 < CHUNK, "ones columns inside the last chunk, at the start of a float4");
-        cur[o / 4].x = 1.0f;
-        cur[o / 4].y = 1.0f;
-      }
 #pragma unroll
-      for (int kc = 0; kc < CHUNK / 8; ++kc) {
-        const float4 lo = cur[2 * kc], hi = cur[2 * kc + 1];
-        sts_v4(abuf + (row >> 3) * S::A_SBO + kc * 128 + (row & 7) * 16, pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w),
-               pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
-      }
+      for (int q = 0; q < V; ++q)
+        asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(abuf + soff[q]), "r"(pack_bf16(cur[q].x, cur[q].y)),
+                     "r"(pack_bf16(cur[q].z, cur[q].w))
+                     : "memory");
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
@@ -181,7 +187,7 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
         mma_commit(bar0 + 8u * b);
       }
 #pragma unroll
-      for (int v = 0; v < V; ++v) cur[v] = nxt[v];
+      for (int q = 0; q < V; ++q) cur[q] = nxt[q];
     }
     // the last two chunks are still outstanding, one per buffer
     timed_out |= !wait_buffer(NCHUNK & 1);
