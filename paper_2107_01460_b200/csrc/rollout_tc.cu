@@ -467,8 +467,8 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       tc_fence_before();
       group_sync(g);
       if (PP) pair_sync(kBarTmem + g);  // the other group has read its heads out of tensor memory
-      // 2. layer 1 runs while the uniform of this step's action draw is computed and (when the
-      //    block is not needed later) the observation block goes to obs[t]
+      // 2. layer 1 runs while the previous step's per-row outputs and (when the block is not needed
+      //    later) the observation block go to global memory
       if (row == 0) {
         tc_fence_after();
         issue_layer<K1, H, !S::FOLD1, false, kALbo>(acc_col, a_addr, w_addr + S::W1_OFF, w_addr + S::ONES_OFF,
@@ -494,8 +494,6 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
           __syncwarp();
         }
       }
-      float u = 0.0f;
-      if (active && !last) u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag));
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       if (!TM) {  // every read of the block is done before the epilogue reuses its memory
@@ -504,21 +502,24 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       }
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, stage_addr, row);
-      // layer 1 is done with A: zero it for the next step (ping-pong: the next user does that)
-      if (TM && !PP) {  // own row only, its readers are in this warp
-#pragma unroll
-        for (int kc = 0; kc < K1 / 8; ++kc)
-          sts_zero16(a_addr + a_offset<K1>(row, kc * 8));
-      } else if (!TM) {
-        for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads) sts_zero16(a_addr + 16u * i);
-      }
-      fence_async_smem();
+      if (!TM) fence_async_smem();  // the hidden activations just written feed the next MMA
       tc_fence_before();
       group_sync(g);
       // 3. layer 2; in ping-pong mode its (long) run time hides the observation block's way out
       if (row == 0) {
         tc_fence_after();
         issue_layer<H, H, true, TM>(acc_col, h_addr, w_addr + S::W2_OFF, w_addr + S::ONES_OFF, w_addr + S::B2_OFF, bar);
+      }
+      // while layer 2 runs: the uniform of this step's action draw, and the A tile (layer 1 is done
+      // with it) is zeroed for the next step (ping-pong: the next user of the tile does that)
+      float u = 0.0f;
+      if (active && !last) u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag));
+      if (TM && !PP) {  // own row only, its readers are in this warp
+#pragma unroll
+        for (int kc = 0; kc < K1 / 8; ++kc)
+          sts_zero16(a_addr + a_offset<K1>(row, kc * 8));
+      } else if (!TM) {
+        for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads) sts_zero16(a_addr + 16u * i);
       }
       if (PP) {
         if (!last || a.obs_last != nullptr) {  // the observation after the last step feeds a centralised critic

@@ -21,7 +21,7 @@ N_ACTIONS = 6
 WORKLOADS = {
     "cfg0_tiny_8x8_2p2f_h64": dict(
         grid=8, n_agents=2, n_food=2, max_agent_level=2, view_radius=2, episode_cap=50,
-        hidden=64, net_kind=0, n_envs=16, T=32, seed=0, precision="fp32"),
+        hidden=64, net_kind=0, n_envs=16, T=32, seed=0, precision="bf16"),
     "cfg1_8x8_2p2f_h128": dict(
         grid=8, n_agents=2, n_food=2, max_agent_level=2, view_radius=2, episode_cap=50,
         hidden=128, net_kind=0, n_envs=1024, T=128, seed=1, precision="bf16"),
