@@ -203,7 +203,7 @@ def test_capacity_and_argument_errors():
 # ---- GAE on arbitrary data, odd shapes ------------------------------------------------------------
 
 @pytest.mark.parametrize("idx,n_envs,T", [(0, 16, 1), (0, 5, 13), (2, 47, 37), (4, 33, 64), (1, 300, 128), (3, 9, 250),
-                                              (4, 2100, 37), (2, 5464, 100)]  # the last two take the float4 variant)
+                                              (4, 2100, 37), (2, 5464, 100)])  # the last two take the float4 variant
 def test_gae_on_random_trajectories(idx, n_envs, T):
     import torch
 
