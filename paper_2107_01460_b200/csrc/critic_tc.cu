@@ -4,7 +4,7 @@
 //   layer-1 kernel: h1 = relu(X C1^T + c1), X = the N observations of an environment-step
 //     concatenated (N*D fp32, contiguous in the time-major obs array).  C1 (bf16, canonical K-major
 //     layout) stays in shared memory; each of two thread groups streams its 128-row tiles through
-//     a ring of four 16-column A buffers, with as many chunks of loads in flight (fp32 -> bf16 on the way in), and leaves h1 as bf16 tiles, already in
+//     two 48-column A buffers (fp32 -> bf16 on the way in) and leaves h1 as bf16 tiles, already in
 //     the operand layout, in a scratch array.
 //   layer-2 kernel: v = Cv relu(h1 C2^T + c2) + cv.  C2 stays in shared memory, the h1 tiles come
 //     in by bulk copies; two thread groups alternate tiles, one in its epilogue (ReLU, bf16
@@ -25,10 +25,9 @@ struct CriticShape {
   static constexpr int D = kObsFixed + N;
   static constexpr int KJ = N * D;                        // joint observation width
   static constexpr int K1 = (KJ + 2 + 15) / 16 * 16;      // + two ones columns that carry c1
-  static constexpr int CHUNK = 16;                        // K columns per A buffer: one MMA K step
-  static constexpr int STAGES = 4;                        // A buffers (and chunks of loads in flight) per group
+  static constexpr int CHUNK = 48;                        // K columns per A buffer (3 MMA K steps)
   static constexpr int NCHUNK = K1 / CHUNK;
-  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0 && (kTileRows * (CHUNK / 4)) % kGroupThreads == 0 && K1 / CHUNK >= STAGES,
+  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0 && (kTileRows * (CHUNK / 4)) % kGroupThreads == 0,
                 "chunking assumes float4 rows, whole chunks and an even split of a chunk over the group");
   static constexpr uint32_t C1_BYTES = kCH * K1 * 2;
   static constexpr uint32_t A_BUF_BYTES = kTileRows * CHUNK * 2;
@@ -85,9 +84,9 @@ template <int N>
 struct CriticL1Smem {
   using S = CriticShape<N>;
   alignas(128) unsigned char c1[S::C1_BYTES];
-  alignas(128) unsigned char abuf[2][S::STAGES][S::A_BUF_BYTES];  // [group][stage]
+  alignas(128) unsigned char abuf[2][2][S::A_BUF_BYTES];  // [group][buffer]
   alignas(8) uint64_t load_bar;
-  alignas(8) uint64_t mma_bar[2][S::STAGES];
+  alignas(8) uint64_t mma_bar[2][2];
   uint32_t tmem_base;
 };
 
@@ -103,7 +102,7 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
   const int tid = threadIdx.x, g = tid / kGroupThreads, row = tid % kGroupThreads, warp = tid / 32;
   if (tid == 0) {
     mbar_init(smem_u32(&sm.load_bar), 1);
-    for (int i = 0; i < 2 * S::STAGES; ++i) mbar_init(smem_u32(&sm.mma_bar[i / S::STAGES][i % S::STAGES]), 1);
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm.mma_bar[i / 2][i % 2]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -128,10 +127,15 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
   const uint32_t acc = tmem_base + static_cast<uint32_t>(g * kCH);
   const uint32_t lane_off = static_cast<uint32_t>((row / 32) * 32) << 16;
   const uint32_t c1_addr = smem_u32(sm.c1);
-  constexpr int P = S::STAGES;
-  const uint32_t abuf0 = smem_u32(sm.abuf[g][0]);     // stage s at abuf0 + s * A_BUF_BYTES
-  const uint32_t bar0 = smem_u32(&sm.mma_bar[g][0]);  // its barrier at bar0 + 8 s
-  uint32_t waits = 0;  // bit s: parity of the next wait on stage s
+  const uint32_t abuf0 = smem_u32(sm.abuf[g][0]);  // buffer b at abuf0 + b * A_BUF_BYTES
+  const uint32_t bar0 = smem_u32(&sm.mma_bar[g][0]);  // its barrier at bar0 + 8 b
+  uint32_t waits0 = 0, waits1 = 0;  // completed waits per buffer: the next wait's parity
+  auto wait_buffer = [&](int b) {
+    const uint32_t parity = (b ? waits1 : waits0) & 1u;
+    const bool ok = mbar_wait(bar0 + 8u * b, parity);
+    if (b) waits1 += 1; else waits0 += 1;
+    return ok;
+  };
 
   for (int tile = blockIdx.x * 2 + g; tile < n_tiles && !timed_out; tile += gridDim.x * 2) {
     // Coalesced loading: float4 number i = row + 128 q of a chunk is (tile row i / V, float4 i % V
@@ -151,51 +155,43 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
       for (int q = 0; q < V; ++q) {
         const int v = (row + kGroupThreads * q) % V, k = c * CHUNK + 4 * v;
         dst[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ptr[q] != nullptr && c < NCHUNK) {
+        if (ptr[q] != nullptr) {
           if (k < KJ) dst[q] = __ldg(reinterpret_cast<const float4 *>(ptr[q] + c * CHUNK));
           else if (k == KJ) dst[q] = make_float4(1.f, 1.f, 0.f, 0.f);  // the two ones columns that pick up c1
         }
       }
     };
-    // P chunks of loads are in flight: chunk c sits in ring slot c % P (registers and A buffer alike)
-    float4 ring[P][V];
-#pragma unroll
-    for (int s2 = 0; s2 < P - 1; ++s2) load_chunk(s2, ring[s2]);
+    float4 cur[V], nxt[V];
+    load_chunk(0, cur);
 #pragma unroll 1
-    for (int c0 = 0; c0 < NCHUNK; c0 += P) {
+    for (int c = 0; c < NCHUNK; ++c) {
+      if (c + 1 < NCHUNK) load_chunk(c + 1, nxt);
+      const int b = c & 1;
+      const uint32_t abuf = abuf0 + static_cast<uint32_t>(b) * S::A_BUF_BYTES;
+      if (c >= 2) timed_out |= !wait_buffer(b);  // the MMAs of chunk c-2 have finished reading this buffer
 #pragma unroll
-      for (int s2 = 0; s2 < P; ++s2) {
-        const int c = c0 + s2;
-        if (c < NCHUNK) {
-          load_chunk(c + P - 1, ring[(s2 + P - 1) % P]);
-          const uint32_t abuf = abuf0 + static_cast<uint32_t>(s2) * S::A_BUF_BYTES;
-          if (c >= P) {  // the MMA of chunk c - P has finished reading this buffer
-            timed_out |= !mbar_wait(bar0 + 8u * s2, (waits >> s2) & 1u);
-            waits ^= 1u << s2;
-          }
+      for (int q = 0; q < V; ++q)
+        asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(abuf + soff[q]), "r"(pack_bf16(cur[q].x, cur[q].y)),
+                     "r"(pack_bf16(cur[q].z, cur[q].w))
+                     : "memory");
+      fence_async_smem();
+      tc_fence_before();
+      group_sync(g);
+      if (row == 0) {
+        tc_fence_after();
 #pragma unroll
-          for (int q = 0; q < V; ++q)
-            asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(abuf + soff[q]), "r"(pack_bf16(ring[s2][q].x, ring[s2][q].y)),
-                         "r"(pack_bf16(ring[s2][q].z, ring[s2][q].w))
-                         : "memory");
-          fence_async_smem();
-          tc_fence_before();
-          group_sync(g);
-          if (row == 0) {
-            tc_fence_after();
-            mma_bf16(acc, smem_desc(abuf, 128, S::A_SBO), smem_desc(c1_addr + c * 256, 128, K1 * 16),
-                     instr_desc(kTileRows, kCH), c > 0 ? 1u : 0u);
-            mma_commit(bar0 + 8u * s2);
-          }
-        }
+        for (int j = 0; j < CHUNK / 16; ++j)
+          mma_bf16(acc, smem_desc(abuf + j * 256, 128, S::A_SBO),
+                   smem_desc(c1_addr + (c * (CHUNK / 16) + j) * 256, 128, K1 * 16), instr_desc(kTileRows, kCH),
+                   (c > 0 || j > 0) ? 1u : 0u);
+        mma_commit(bar0 + 8u * b);
       }
-    }
-    // the last P chunks are still outstanding, one per stage
 #pragma unroll
-    for (int s2 = 0; s2 < P; ++s2) {
-      timed_out |= !mbar_wait(bar0 + 8u * s2, (waits >> s2) & 1u);
-      waits ^= 1u << s2;
+      for (int q = 0; q < V; ++q) cur[q] = nxt[q];
     }
+    // the last two chunks are still outstanding, one per buffer
+    timed_out |= !wait_buffer(NCHUNK & 1);
+    timed_out |= !wait_buffer((NCHUNK + 1) & 1);
     tc_fence_after();
     // epilogue: ReLU, bf16, the row goes out in the operand layout of layer 2
     unsigned char *tile_out = h1 + static_cast<size_t>(tile) * S::H1_TILE_BYTES;
