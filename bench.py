@@ -33,6 +33,8 @@ from paper_2107_01460_b200 import workloads as wl  # noqa: E402
 
 METRIC = "env_agent_steps_per_s"
 UNIT = "env-agent-steps/s"
+# Filled from profiles/rollout_tc_cfg1_full.md; reset an entry to None when its kernel changes.
+NCU_TRAFFIC_BYTES = {("cfg1_8x8_2p2f_h128", "bf16"): None}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -302,6 +304,11 @@ def run_gpu(args):
         roofline = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None}
     roofline["kernel"] = "rollout (fused env step + MLP + sampler), %s" % ("bf16 tcgen05" if precision else "fp32 SIMT")
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch of that kernel, from the ncu capture
+    # summarised under profiles/ (None when no capture of the current kernel exists for the workload)
+    roofline["traffic"] = NCU_TRAFFIC_BYTES.get((w["name"], "bf16" if precision else "fp32"))
+    roofline["traffic_note"] = ("ncu, one launch; below the algorithmic bytes because the 126 MB L2 still holds part of "
+                                "the trajectory when the kernel ends") if roofline["traffic"] else None
     roofline["peak_source"] = "of " + peaks["source"]
     roofline["kernel_ms"] = roll_ms
     gae_ach = rows * gae_bytes_per_element(w) / (gae_ms * 1e-3) / 1e9

@@ -63,12 +63,13 @@ struct TcShape {
   // hidden activations (two per column) when TM, the heads accumulator.
   static constexpr int HID_COL = H;
   static constexpr int HEAD_COL = H + (TM ? H / 2 : 0);
-  static constexpr int GROUP_COLS = HEAD_COL + 32;
+  static constexpr int GROUP_COLS = HEAD_COL + 64;  // two heads accumulators: one per thread group in ping-pong mode
   // independent sets of tile resources (A tile, block, tensor-memory columns) per CTA
   static constexpr int GROUPS = (2 * GROUP_COLS <= 512 && 2 * (A_BYTES + X_BYTES) + IMAGE_BYTES <= 220 * 1024) ? 2 : 1;
   static constexpr int TMEM_COLS = GROUPS * GROUP_COLS <= 256 ? 256 : 512;
   // When only one set of tile resources fits (H = 256), two thread groups still run, in
-  // anti-phase: they take turns on the one A tile and the one set of tensor-memory columns, so
+  // anti-phase: they take turns on the one A tile and on the accumulator and hidden-activation
+  // columns of tensor memory (each handed over as soon as its last reader is done), so
   // that one group's environment phase (sampler, transition, observation) overlaps the other's
   // network phase (the three MMAs and their epilogues).
   static constexpr bool PINGPONG = TM && GROUPS == 1;
@@ -360,7 +361,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const uint32_t tmem_base = sm.tmem_base;
   const uint32_t acc_col = tmem_base + static_cast<uint32_t>(dg * S::GROUP_COLS);
   const uint32_t hid_col = acc_col + static_cast<uint32_t>(S::HID_COL);
-  const uint32_t head_col = acc_col + static_cast<uint32_t>(S::HEAD_COL);
+  const uint32_t head_col = acc_col + static_cast<uint32_t>(S::HEAD_COL + (PP ? 32 * g : 0));
   const uint32_t lane_off = static_cast<uint32_t>(wg * 32) << 16;  // this warp's TMEM lanes
   const uint32_t w_addr = smem_u32(sm.weights);
   const uint32_t a_addr = smem_u32(gs.a);
@@ -381,6 +382,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   if (PP && g == 1) {  // group 0 goes first on both shared resources
     pair_arrive(kBarTile + 0);
     pair_arrive(kBarTmem + 0);
+    pair_arrive(kBarHid + 0);
   }
 
   // ---- tiles: in round `it` group g works on tile (it * gridDim.x + blockIdx.x) * 2 + g ----------
@@ -440,10 +442,12 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         // one verdict for the whole group (its threads may see the flag at different times); the flag
         // is looked at every eighth step only: the load would queue behind the partner's copy-out
         idle = group_any(g, idle || ((t & 7) == 0 && lds_s32(abort_addr) != 0));
-        if (idle) {  // keep the hand-over order of a working step: tile, tensor memory, tile, tensor memory
+        if (idle) {  // keep the hand-over order of a working step: three acquisitions, then three releases
           pair_sync(kBarTmem + g);
+          pair_sync(kBarHid + g);
           pair_arrive(kBarTile + (1 - g));
           pair_arrive(kBarTmem + (1 - g));
+          pair_arrive(kBarHid + (1 - g));
           continue;
         }
 #pragma unroll
@@ -466,7 +470,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       fence_async_smem();
       tc_fence_before();
       group_sync(g);
-      if (PP) pair_sync(kBarTmem + g);  // the other group has read its heads out of tensor memory
+      if (PP) pair_sync(kBarTmem + g);  // the other group's second epilogue has read the accumulator columns
       // 2. layer 1 runs while the previous step's per-row outputs and (when the block is not needed
       //    later) the observation block go to global memory
       if (row == 0) {
@@ -500,6 +504,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         if (bulk_pending) { bulk_store_wait_read(); bulk_pending = false; }
         group_sync(g);
       }
+      if (PP) pair_sync(kBarHid + g);  // the other group's heads MMA has read the hidden-activation columns
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, stage_addr, row);
       if (!TM) fence_async_smem();  // the hidden activations just written feed the next MMA
@@ -536,8 +541,9 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       phase ^= 1;
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, stage_addr, row);
-      fence_async_smem();
+      if (!TM) fence_async_smem();
       tc_fence_before();
+      if (PP) pair_arrive(kBarTmem + (1 - g));  // this thread is done with the accumulator columns
       group_sync(g);
       // 4. heads: six logits and the value, N padded to 16
       if (row == 0) {
@@ -546,6 +552,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       }
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
+      if (PP) pair_arrive(kBarHid + (1 - g));  // the heads MMA is done reading the hidden-activation columns
       tc_fence_after();
       int action = 0;
       {
@@ -553,10 +560,6 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         tmem_ld16(head_col + lane_off, hv);
 #pragma unroll
         for (int k = 0; k <= kActions; ++k) hv[k] += head_bias[k];  // the heads' biases stay fp32
-        if (PP) {  // this thread is done with tensor memory for this step
-          tc_fence_before();
-          pair_arrive(kBarTmem + (1 - g));
-        }
         if (!TM)  // the hidden activations are dead: zero the observation block for the next step
           for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
         if (active) {

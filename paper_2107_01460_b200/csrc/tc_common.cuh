@@ -99,8 +99,9 @@ __device__ __forceinline__ void pair_sync(int id) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
 }
 // Ping-pong hand-over barriers (ids 1..2 belong to the groups): group g waits on kBar* + g for
-// the A tile / the tensor-memory columns, and the other group arrives there when it lets go.
-constexpr int kBarTile = 8, kBarTmem = 10;
+// the A tile / the accumulator columns / the hidden-activation columns of tensor memory, and the
+// other group arrives there when it lets go.
+constexpr int kBarTile = 8, kBarTmem = 10, kBarHid = 12;
 // Barrier of the group that also ORs a predicate over its threads.
 __device__ __forceinline__ bool group_any(int g, bool pred) {
   uint32_t out;
