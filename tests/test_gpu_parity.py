@@ -222,3 +222,78 @@ def test_gae_on_random_trajectories(idx, n_envs, T):
         ga, gr = ro.adv.cpu().numpy(), ro.ret.cpu().numpy()
         assert np.max(np.abs(ga - adv) / np.maximum(1, np.abs(adv))) <= 1e-5
         assert np.max(np.abs(gr - ret) / np.maximum(1, np.abs(ret))) <= 1e-5
+
+
+# ---- tensor-core path: determinism, continuation, sharding, forcing, degenerate sizes ----------
+
+@pytest.mark.parametrize("idx,n_envs", [(1, 150), (4, 50), (3, 40)])
+def test_bf16_two_calls_continue_like_one_and_runs_repeat(idx, n_envs):
+    import torch
+
+    w = wl.workload(idx)
+    cfg = binding.make_config(w, precision=BF16, max_T=50, n_envs=n_envs)
+    params = torch.from_numpy(wl.make_params(w, bias_scale=0.1)).cuda()
+    a = binding.Rollout(cfg)
+    a.run(params, 50)
+    whole = [t.clone() for t in (a.obs, a.actions, a.logp, a.values, a.rewards, a.dones)]
+    a.reset(w["seed"])
+    a.run(params, 50)
+    for x, y in zip(whole, (a.obs, a.actions, a.logp, a.values, a.rewards, a.dones)):
+        assert torch.equal(x, y)  # same seed, same bytes
+    b = binding.Rollout(cfg)
+    b.run(params, 20)
+    first = [t[:20].clone() for t in (b.obs, b.actions, b.logp, b.rewards, b.dones)]
+    b.run(params, 30)
+    for x, y, z in zip(first, (b.obs, b.actions, b.logp, b.rewards, b.dones), (a.obs, a.actions, a.logp, a.rewards, a.dones)):
+        assert torch.equal(z[:20], x) and torch.equal(z[20:50], y[:30])
+    assert torch.equal(a.values[50], b.values[30]) and np.array_equal(a.get_state(), b.get_state())
+    assert a.status() == 0 and b.status() == 0
+
+
+@pytest.mark.parametrize("idx", [2, 4])
+def test_env_shards_reproduce_the_whole_batch_on_the_gpu(idx):
+    """Two handles with first_env offsets give the bytes of one handle over all environments."""
+    import torch
+
+    w = wl.workload(idx)
+    T, n = 30, 90
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    whole = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=n))
+    whole.run(params, T)
+    cut = 37
+    lo = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=cut))
+    hi = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=n - cut, first_env=cut))
+    lo.run(params, T)
+    hi.run(params, T)
+    for name in ("obs", "actions", "rewards", "dones", "logp", "values"):
+        full = getattr(whole, name)
+        assert torch.equal(full[:, :cut], getattr(lo, name)) and torch.equal(full[:, cut:], getattr(hi, name)), name
+
+
+@pytest.mark.parametrize("precision", [FP32, BF16])
+@pytest.mark.parametrize("idx,n_envs,T", [(0, 1, 1), (2, 1, 3), (4, 1, 2), (3, 2, 1)])
+def test_degenerate_sizes(idx, n_envs, T, precision):
+    w = wl.workload(idx)
+    params = wl.make_params(w)
+    ro, _ = run_gpu(w, precision, T, n_envs=n_envs, params=params)
+    check_against_oracle(w, ro, params, T, precision, np.arange(n_envs))
+
+
+def test_forced_actions_on_the_tensor_path():
+    """Teacher forcing in bf16: the oracle's own free-running actions, replayed on the GPU."""
+    import torch
+
+    w = wl.workload(1)
+    T, n = 40, 70
+    params = wl.make_params(w)
+    ocfg = oracle.make_config(w)
+    free = oracle.rollout(ocfg, w["seed"], params, T, np.arange(n))
+    cfg = binding.make_config(w, precision=BF16, max_T=T, n_envs=n)
+    ro = binding.Rollout(cfg)
+    ro.run_forced(torch.from_numpy(params).cuda(), T, torch.from_numpy(free.actions).cuda())
+    assert ro.status() == 0
+    assert np.array_equal(ro.actions.cpu().numpy(), free.actions)
+    assert np.array_equal(ro.obs.cpu().numpy().view(np.uint32), free.obs.view(np.uint32))
+    assert np.array_equal(ro.rewards.cpu().numpy(), free.rewards) and np.array_equal(ro.dones.cpu().numpy(), free.dones)
+    lp = ro.logp.cpu().numpy()
+    assert np.all(np.abs(lp - free.logp) <= 2e-2 * (1 + np.abs(free.logp)))
