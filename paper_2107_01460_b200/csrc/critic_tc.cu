@@ -3,9 +3,9 @@
 // rollout's serial chain and computed for all (T+1)*E environment-steps at once.
 //   layer-1 kernel: h1 = relu(X C1^T + c1), X = the N observations of an environment-step
 //     concatenated (N*D fp32, contiguous in the time-major obs array).  C1 (bf16, canonical K-major
-//     layout) stays in shared memory; each of two thread groups streams its 128-row tiles through
-//     two 48-column A buffers (fp32 -> bf16 on the way in) and leaves h1 as bf16 tiles, already in
-//     the operand layout, in a scratch array.
+//     layout) stays in shared memory; producer warps stream the 128-row tiles through a ring of
+//     48-column A buffers (fp32 -> bf16 on the way in), one thread issues the MMAs, epilogue warps
+//     leave h1 as bf16 tiles, already in the operand layout, in a scratch array.
 //   layer-2 kernel: v = Cv relu(h1 C2^T + c2) + cv.  C2 stays in shared memory, the h1 tiles come
 //     in by bulk copies; two thread groups alternate tiles, one in its epilogue (ReLU, bf16
 //     rounding, dot product with Cv) while the other's MMAs run.  The value is written to the N
@@ -27,11 +27,13 @@ struct CriticShape {
   static constexpr int K1 = (KJ + 2 + 15) / 16 * 16;      // + two ones columns that carry c1
   static constexpr int CHUNK = 48;                        // K columns per A buffer (3 MMA K steps)
   static constexpr int NCHUNK = K1 / CHUNK;
-  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0 && (kTileRows * (CHUNK / 4)) % kGroupThreads == 0,
-                "chunking assumes float4 rows, whole chunks and an even split of a chunk over the group");
+  static_assert(K1 % CHUNK == 0 && KJ % 4 == 0, "chunking assumes float4 rows and whole chunks");
   static constexpr uint32_t C1_BYTES = kCH * K1 * 2;
-  static constexpr uint32_t A_BUF_BYTES = kTileRows * CHUNK * 2;
-  static constexpr uint32_t A_SBO = (CHUNK / 8) * 128;
+  // A buffers of layer 1: core matrices of a row group 144 bytes apart, so that the twelve 8-byte
+  // stores a row gets from consecutive threads fall into different banks
+  static constexpr uint32_t A_LBO = 144;
+  static constexpr uint32_t A_SBO = (CHUNK / 8) * A_LBO;
+  static constexpr uint32_t A_BUF_BYTES = (kTileRows / 8) * A_SBO;
   // layer-2 image: C2 | c2 bias tile | ones tile | Cv (bf16-rounded, as fp32) | cv
   static constexpr uint32_t C2_OFF = 0, C2_BYTES = kCH * kCH * 2;
   static constexpr uint32_t B2_OFF = C2_OFF + C2_BYTES, B2_BYTES = kCH * 16 * 2;
@@ -80,29 +82,52 @@ __global__ void prep_critic_kernel(const float *__restrict__ params, unsigned ch
 }
 
 // ---- layer 1 -----------------------------------------------------------------------------------
+// Warp-specialised.  Four producer groups of three warps each own one stage of a ring of bf16 A
+// buffers: group g loads item g, g + 4, ... (an item is one 48-column chunk of one 128-row tile)
+// into registers, converts it into its stage and at once starts the loads of its next item, so four
+// items of loads are in flight per SM with a single item per thread.  One thread issues the MMAs as
+// the stages fill and frees them by tcgen05.commit; four epilogue warps drain the two alternating
+// accumulators.  Only mbarriers connect the roles, every wait is bounded.
+constexpr int kL1Stages = 4, kL1GroupThreads = 96, kL1Producers = kL1Stages * kL1GroupThreads;
+constexpr int kL1Threads = kL1Producers + 128 + 32;  // producers, epilogue warps, the issuing warp
+
 template <int N>
 struct CriticL1Smem {
   using S = CriticShape<N>;
   alignas(128) unsigned char c1[S::C1_BYTES];
-  alignas(128) unsigned char abuf[2][2][S::A_BUF_BYTES];  // [group][buffer]
+  alignas(128) unsigned char abuf[kL1Stages][S::A_BUF_BYTES];
   alignas(8) uint64_t load_bar;
-  alignas(8) uint64_t mma_bar[2][2];
+  alignas(8) uint64_t full[kL1Stages], empty[kL1Stages], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
 };
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 template <int N>
-__global__ void __launch_bounds__(2 * kGroupThreads, 1)
+__global__ void __launch_bounds__(kL1Threads, 1)
 critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_last, long long rows_main,
                  long long rows_total, const unsigned char *__restrict__ image, unsigned char *__restrict__ h1, int n_tiles,
                  int *status) {
   using S = CriticShape<N>;
-  constexpr int KJ = S::KJ, K1 = S::K1, CHUNK = S::CHUNK, NCHUNK = S::NCHUNK, V = CHUNK / 4;
+  constexpr int KJ = S::KJ, K1 = S::K1, CHUNK = S::CHUNK, NCHUNK = S::NCHUNK;
+  constexpr int V = CHUNK / 4;        // float4 per row and chunk
+  constexpr int Q = kTileRows / 8;    // float4 per producer thread and item: rows r0, r0 + 8, ...
+  static_assert(V * 8 == kL1GroupThreads, "a group covers eight rows of a chunk per pass");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   CriticL1Smem<N> &sm = *reinterpret_cast<CriticL1Smem<N> *>(smem_raw);
-  const int tid = threadIdx.x, g = tid / kGroupThreads, row = tid % kGroupThreads, warp = tid / 32;
+  const int tid = threadIdx.x, warp = tid / 32;
   if (tid == 0) {
     mbar_init(smem_u32(&sm.load_bar), 1);
-    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm.mma_bar[i / 2][i % 2]), 1);
+    for (int i = 0; i < kL1Stages; ++i) {
+      mbar_init(smem_u32(&sm.full[i]), kL1GroupThreads / 32);  // one arrival per warp of the stage's group
+      mbar_init(smem_u32(&sm.empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&sm.acc_full[i]), 1);
+      mbar_init(smem_u32(&sm.acc_empty[i]), 4);  // one arrival per epilogue warp
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -124,92 +149,121 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
   timed_out = __syncthreads_or(timed_out) != 0;
 
   const uint32_t tmem_base = sm.tmem_base;
-  const uint32_t acc = tmem_base + static_cast<uint32_t>(g * kCH);
-  const uint32_t lane_off = static_cast<uint32_t>((row / 32) * 32) << 16;
-  const uint32_t c1_addr = smem_u32(sm.c1);
-  const uint32_t abuf0 = smem_u32(sm.abuf[g][0]);  // buffer b at abuf0 + b * A_BUF_BYTES
-  const uint32_t bar0 = smem_u32(&sm.mma_bar[g][0]);  // its barrier at bar0 + 8 b
-  uint32_t waits0 = 0, waits1 = 0;  // completed waits per buffer: the next wait's parity
-  auto wait_buffer = [&](int b) {
-    const uint32_t parity = (b ? waits1 : waits0) & 1u;
-    const bool ok = mbar_wait(bar0 + 8u * b, parity);
-    if (b) waits1 += 1; else waits0 += 1;
-    return ok;
-  };
+  const uint32_t full0 = smem_u32(&sm.full[0]), empty0 = smem_u32(&sm.empty[0]);
+  const uint32_t acc_full0 = smem_u32(&sm.acc_full[0]), acc_empty0 = smem_u32(&sm.acc_empty[0]);
+  const uint32_t abuf0 = smem_u32(sm.abuf[0]);
+  // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+  const int my_tiles = (n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  const int n_items = my_tiles * NCHUNK;  // (tile, chunk) pairs in order; item n uses ring stage n % kL1Stages
 
-  for (int tile = blockIdx.x * 2 + g; tile < n_tiles && !timed_out; tile += gridDim.x * 2) {
-    // Coalesced loading: float4 number i = row + 128 q of a chunk is (tile row i / V, float4 i % V
-    // of that row's CHUNK columns), so consecutive threads read consecutive 16 bytes of a row.
-    const float *ptr[V];  // address of that float4 in chunk 0 (nullptr: the row is past the end)
-    uint32_t soff[V];     // its place in an A buffer
+  if (!timed_out && tid < kL1Producers) {
+    // ---- producers --------------------------------------------------------------------------
+    // Thread t of a group takes float4 v = t % 12 of rows r0 + 8 q (r0 = t / 12): consecutive threads
+    // read consecutive 16 bytes of a row, and every address is a per-thread base plus a constant.
+    const int g = tid / kL1GroupThreads, t = tid - g * kL1GroupThreads;
+    const int v = t % V, r0 = t / V;
+    const uint32_t goff = static_cast<uint32_t>(r0 * KJ + 4 * v);  // in floats, within the tile's block of rows
+    const uint32_t sdst = abuf0 + static_cast<uint32_t>(g) * S::A_BUF_BYTES +
+                          static_cast<uint32_t>(((4 * v) >> 3) * S::A_LBO + r0 * 16 + ((4 * v) & 7) * 2);
+    // in the last chunk: the two ones columns that pick up c1, and the zero columns after them
+    const bool ones = (NCHUNK - 1) * CHUNK + 4 * v == KJ, past = (NCHUNK - 1) * CHUNK + 4 * v > KJ;
+    const uint32_t full_bar = full0 + 8u * g, empty_bar = empty0 + 8u * g;
+    int n = g, kt = 0, c = g;  // this group's next item and its (tile, chunk)
+    static_assert(kL1Stages <= S::NCHUNK, "the first items of all groups lie in the first tile");
+    float4 d[Q];
+    auto load_item = [&]() {
+      const long long row0 = (static_cast<long long>(blockIdx.x) + static_cast<long long>(kt) * gridDim.x) * kTileRows;
+      const bool in_main = row0 + kTileRows <= rows_main;
+      const bool in_last = row0 >= rows_main && row0 + kTileRows <= rows_total;
+      const bool last_chunk = c == NCHUNK - 1;
+      if (last_chunk && (ones || past)) {
 #pragma unroll
-    for (int q = 0; q < V; ++q) {
-      const int i = row + kGroupThreads * q, r = i / V, v = i - r * V;
-      const long long r_idx = static_cast<long long>(tile) * kTileRows + r;
-      ptr[q] = nullptr;
-      if (r_idx < rows_total) ptr[q] = (r_idx < rows_main ? obs + r_idx * KJ : obs_last + (r_idx - rows_main) * KJ) + 4 * v;
-      soff[q] = static_cast<uint32_t>((r >> 3) * S::A_SBO + ((4 * v) >> 3) * 128 + (r & 7) * 16 + ((4 * v) & 7) * 2);
-    }
-    auto load_chunk = [&](int c, float4 *dst) {
+        for (int q = 0; q < Q; ++q) d[q] = make_float4(ones ? 1.f : 0.f, ones ? 1.f : 0.f, 0.f, 0.f);
+      } else if (in_main || in_last) {
+        // the tile lies wholly inside one of the two observation arrays: a contiguous block of rows
+        const float *src = (in_main ? obs + row0 * KJ : obs_last + (row0 - rows_main) * KJ) + c * CHUNK + goff;
 #pragma unroll
-      for (int q = 0; q < V; ++q) {
-        const int v = (row + kGroupThreads * q) % V, k = c * CHUNK + 4 * v;
-        dst[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ptr[q] != nullptr) {
-          if (k < KJ) dst[q] = __ldg(reinterpret_cast<const float4 *>(ptr[q] + c * CHUNK));
-          else if (k == KJ) dst[q] = make_float4(1.f, 1.f, 0.f, 0.f);  // the two ones columns that pick up c1
+        for (int q = 0; q < Q; ++q) d[q] = __ldg(reinterpret_cast<const float4 *>(src + q * 8 * KJ));
+      } else {
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+          const long long r_idx = row0 + r0 + 8 * q;
+          d[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (r_idx < rows_total)
+            d[q] = __ldg(reinterpret_cast<const float4 *>(
+                (r_idx < rows_main ? obs + r_idx * KJ : obs_last + (r_idx - rows_main) * KJ) + c * CHUNK + 4 * v));
         }
       }
     };
-    float4 cur[V], nxt[V];
-    load_chunk(0, cur);
+    if (n < n_items) load_item();
 #pragma unroll 1
-    for (int c = 0; c < NCHUNK; ++c) {
-      if (c + 1 < NCHUNK) load_chunk(c + 1, nxt);
-      const int b = c & 1;
-      const uint32_t abuf = abuf0 + static_cast<uint32_t>(b) * S::A_BUF_BYTES;
-      if (c >= 2) timed_out |= !wait_buffer(b);  // the MMAs of chunk c-2 have finished reading this buffer
+    for (uint32_t it = 0; n < n_items && !timed_out; ++it) {
+      timed_out |= !mbar_wait(empty_bar, (it & 1) ^ 1);  // the MMAs that read this stage are done
 #pragma unroll
-      for (int q = 0; q < V; ++q)
-        asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(abuf + soff[q]), "r"(pack_bf16(cur[q].x, cur[q].y)),
-                     "r"(pack_bf16(cur[q].z, cur[q].w))
+      for (int q = 0; q < Q; ++q)
+        asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(sdst + q * S::A_SBO), "r"(pack_bf16(d[q].x, d[q].y)),
+                     "r"(pack_bf16(d[q].z, d[q].w))
                      : "memory");
       fence_async_smem();
-      tc_fence_before();
-      group_sync(g);
-      if (row == 0) {
+      __syncwarp();
+      if ((tid & 31) == 0) mbar_arrive(full_bar);
+      n += kL1Stages;
+      c += kL1Stages;
+      if (c >= NCHUNK) { c -= NCHUNK; ++kt; }
+      if (n < n_items) load_item();
+    }
+  } else if (!timed_out && tid >= kL1Producers + 128) {
+    // ---- the issuing thread -----------------------------------------------------------------
+    if (tid == kL1Producers + 128) {
+      const uint32_t c1_addr = smem_u32(sm.c1);
+      for (int kt = 0; kt < my_tiles && !timed_out; ++kt) {
+        const int a = kt & 1;
+        timed_out |= !mbar_wait(acc_empty0 + 8u * a, ((kt >> 1) & 1) ^ 1);  // the epilogue has drained this accumulator
         tc_fence_after();
+        const uint32_t acc = tmem_base + static_cast<uint32_t>(a * kCH);
+        for (int c = 0; c < NCHUNK && !timed_out; ++c) {
+          const int n = kt * NCHUNK + c, s2 = n % kL1Stages;
+          timed_out |= !mbar_wait(full0 + 8u * s2, (n / kL1Stages) & 1);
+          tc_fence_after();
+          const uint32_t abuf = abuf0 + static_cast<uint32_t>(s2) * S::A_BUF_BYTES;
 #pragma unroll
-        for (int j = 0; j < CHUNK / 16; ++j)
-          mma_bf16(acc, smem_desc(abuf + j * 256, 128, S::A_SBO),
-                   smem_desc(c1_addr + (c * (CHUNK / 16) + j) * 256, 128, K1 * 16), instr_desc(kTileRows, kCH),
-                   (c > 0 || j > 0) ? 1u : 0u);
-        mma_commit(bar0 + 8u * b);
+          for (int j = 0; j < CHUNK / 16; ++j)
+            mma_bf16(acc, smem_desc(abuf + j * 2 * S::A_LBO, S::A_LBO, S::A_SBO),
+                     smem_desc(c1_addr + (c * (CHUNK / 16) + j) * 256, 128, K1 * 16), instr_desc(kTileRows, kCH),
+                     (c > 0 || j > 0) ? 1u : 0u);
+          mma_commit(empty0 + 8u * s2);  // frees the stage when these MMAs have read it
+        }
+        mma_commit(acc_full0 + 8u * a);
       }
-#pragma unroll
-      for (int q = 0; q < V; ++q) cur[q] = nxt[q];
     }
-    // the last two chunks are still outstanding, one per buffer
-    timed_out |= !wait_buffer(NCHUNK & 1);
-    timed_out |= !wait_buffer((NCHUNK + 1) & 1);
-    tc_fence_after();
-    // epilogue: ReLU, bf16, the row goes out in the operand layout of layer 2
-    unsigned char *tile_out = h1 + static_cast<size_t>(tile) * S::H1_TILE_BYTES;
-    uint32_t ra[32], pk[16];
+  } else if (!timed_out) {
+    // ---- epilogue warps: ReLU, bf16, the row goes out in the operand layout of layer 2 -----------
+    const int row = tid - kL1Producers;  // 0..127: tile row and tensor-memory lane
+    const uint32_t lane_off = static_cast<uint32_t>((row / 32) * 32) << 16;
+    for (int kt = 0; kt < my_tiles && !timed_out; ++kt) {
+      const int a = kt & 1;
+      const long long tile = static_cast<long long>(blockIdx.x) + static_cast<long long>(kt) * gridDim.x;
+      timed_out |= !mbar_wait(acc_full0 + 8u * a, (kt >> 1) & 1);
+      tc_fence_after();
+      const uint32_t acc = tmem_base + static_cast<uint32_t>(a * kCH);
+      unsigned char *tile_out = h1 + static_cast<size_t>(tile) * S::H1_TILE_BYTES;
+      uint32_t ra[32], pk[16];
 #pragma unroll 1
-    for (int c0 = 0; c0 < kCH; c0 += 32) {
-      tmem_ld32_nowait(acc + lane_off + static_cast<uint32_t>(c0), ra);
-      tmem_ld_wait();
-      relu_pack32(ra, pk);
+      for (int c0 = 0; c0 < kCH; c0 += 32) {
+        tmem_ld32_nowait(acc + lane_off + static_cast<uint32_t>(c0), ra);
+        tmem_ld_wait();
+        relu_pack32(ra, pk);
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<uint4 *>(tile_out + canon_offset(row, c0 + 8 * q, kCH)) =
-            make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4 *>(tile_out + canon_offset(row, c0 + 8 * q, kCH)) =
+              make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if ((tid & 31) == 0) mbar_arrive(acc_empty0 + 8u * a);
     }
-    tc_fence_before();
-    if (group_any(g, timed_out)) timed_out = true;
   }
-  if (timed_out && row == 0) atomicExch(status, kStatusTimeout);
+  if (timed_out) atomicExch(status, kStatusTimeout);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
@@ -358,9 +412,9 @@ cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T
     const size_t smem = sizeof(CriticL1Smem<4>);
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    const int ctas = (n_tiles + 1) / 2 < sms ? (n_tiles + 1) / 2 : sms;
-    kern<<<ctas, 2 * kGroupThreads, smem, h->stream>>>(h->buf.obs, h->d_obs_last, rows_main, rows_total, image,
-                                                       static_cast<unsigned char *>(h->d_critic_h1), n_tiles, h->d_status);
+    const int ctas = n_tiles < sms ? n_tiles : sms;
+    kern<<<ctas, kL1Threads, smem, h->stream>>>(h->buf.obs, h->d_obs_last, rows_main, rows_total, image,
+                                                static_cast<unsigned char *>(h->d_critic_h1), n_tiles, h->d_status);
     h->launches += 1;
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
