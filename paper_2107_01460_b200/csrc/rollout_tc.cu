@@ -308,7 +308,7 @@ __device__ __forceinline__ void expand_quads(const QuadPlan<D, K1> &p, uint32_t 
 // ---- the rollout kernel ------------------------------------------------------------------------
 template <int N, int F, int H, bool TM>
 __global__ void __launch_bounds__(TcShape<N, H, TM>::THREADS, 1)
-rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles) {
+rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles, int groups) {
   using S = TcShape<N, H, TM>;
   constexpr int D = S::D, K1 = S::K1;
   constexpr bool PP = S::PINGPONG;
@@ -385,12 +385,13 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     pair_arrive(kBarHid + 0);
   }
 
-  // ---- tiles: in round `it` group g works on tile (it * gridDim.x + blockIdx.x) * 2 + g ----------
+  // ---- tiles: in round `it` group g works on tile (it * gridDim.x + blockIdx.x) * groups + g; with
+  // groups == 1 (little work: one group per SM has the tensor pipe to itself) group 1 sits out ------
   for (int it = 0; !timed_out || PP; ++it) {
-    const int tile0 = (it * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x)) * 2;
+    const int tile0 = (it * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x)) * groups;
     if (tile0 >= n_tiles) break;  // same for both groups
     const int tile = tile0 + g;
-    if (!PP && tile >= n_tiles) break;
+    if (!PP && (g >= groups || tile >= n_tiles)) break;
     // ping-pong: a group without a tile (or after a time-out) still walks through the hand-over
     // barriers of every step, so that its partner never waits for it in vain
     bool idle = PP && (tile >= n_tiles || timed_out);
@@ -639,14 +640,17 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   if (err != cudaSuccess) return err;
   // Environments per tile: full tiles when there is enough work for every group of every SM,
   // otherwise smaller tiles so that all groups have one (the per-step chain is latency-bound).
-  const int slots = sms * 2;  // two thread groups per CTA
+  // Two thread groups per CTA, unless one group per SM already holds all environments: alone on
+  // its SM a group does not share the tensor pipe and the barriers' issue slots.
+  const int groups = (!S::PINGPONG && h->cfg.n_envs <= sms * S::EPT_MAX) ? 1 : 2;
+  const int slots = sms * groups;
   int ept = (h->cfg.n_envs + slots - 1) / slots;
   if (ept > S::EPT_MAX) ept = S::EPT_MAX;
   if (ept < 1) ept = 1;
   const int n_tiles = (h->cfg.n_envs + ept - 1) / ept;
-  const int ctas = (n_tiles + 1) / 2;
+  const int ctas = (n_tiles + groups - 1) / groups;
   kern<<<ctas < sms ? ctas : sms, S::THREADS, smem, h->stream>>>(args, static_cast<const unsigned char *>(h->d_wtc), ept,
-                                                                 n_tiles);
+                                                                 n_tiles, groups);
   h->launches += 1;
   return cudaGetLastError();
 }
