@@ -53,6 +53,8 @@ extern "C" {
 #define MAVA_FLAG_WRITE_LOGITS 1 /* also write the six logits of every row to buffers.logits       */
 #define MAVA_FLAG_HIDDEN_IN_TMEM 2 /* bf16 path, H <= 128: keep hidden activations in tensor memory
                                       (the layout H = 256 always uses); results are identical     */
+#define MAVA_FLAG_WIDE_TILES 4 /* bf16 path: always use 128-row tiles, also for batches small
+                                  enough for the few-rows form of the kernel; results are identical */
 
 typedef struct mava_rollout mava_rollout_t; /* opaque, owned by the library */
 

@@ -22,6 +22,7 @@ MAVA_PRECISION_FP32 = 0
 MAVA_PRECISION_BF16 = 1
 MAVA_FLAG_WRITE_LOGITS = 1
 MAVA_FLAG_HIDDEN_IN_TMEM = 2
+MAVA_FLAG_WIDE_TILES = 4
 N_ACTIONS = 6
 
 EXPORTS = [

@@ -628,6 +628,8 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   }
 }
 
+#include "rollout_tc_small.cuh"
+
 template <int N, int F, int H, bool TM>
 cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   using S = TcShape<N, H, TM>;
@@ -638,6 +640,13 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   int sms = 0;
   err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
   if (err != cudaSuccess) return err;
+  // Few rows per SM: the form with the rows as the N operand of the MMA.
+  if constexpr (!TM && H == kTileRows) {
+    if ((h->cfg.flags & MAVA_FLAG_WIDE_TILES) == 0) {
+      if (h->cfg.n_envs <= sms * SmallShape<N, H, 16>::EPT_MAX) return launch_tc_small<N, F, H, 16>(h, args, sms);
+      if (h->cfg.n_envs <= sms * SmallShape<N, H, 32>::EPT_MAX) return launch_tc_small<N, F, H, 32>(h, args, sms);
+    }
+  }
   // Environments per tile: full tiles when there is enough work for every group of every SM,
   // otherwise smaller tiles so that all groups have one (the per-step chain is latency-bound).
   // Two thread groups per CTA, unless one group per SM already holds all environments: alone on

@@ -68,16 +68,20 @@ def test_reduced_configs_fp32(idx, n_envs, T):
     print(idx, out)
 
 
-@pytest.mark.parametrize("idx,n_envs,T,tmem", [(1, 333, 60, False), (2, 300, 110, False), (3, 200, 105, False),
-                                               (4, 150, 40, False), (0, 16, 32, True), (1, 333, 60, True),
-                                               (2, 300, 110, True)])
-def test_reduced_configs_bf16(idx, n_envs, T, tmem):
-    """tmem=True keeps the hidden activations in tensor memory (the layout H = 256 always uses)."""
+@pytest.mark.parametrize("idx,n_envs,T,mode", [(1, 333, 60, ""), (2, 300, 110, ""), (3, 200, 105, ""),
+                                               (4, 150, 40, ""), (0, 16, 32, "tmem"), (1, 333, 60, "tmem"),
+                                               (2, 300, 110, "tmem"), (1, 333, 60, "wide"), (2, 300, 110, "wide"),
+                                               (1, 1500, 40, ""), (2, 1000, 40, ""), (1, 1500, 40, "wide")])
+def test_reduced_configs_bf16(idx, n_envs, T, mode):
+    """mode "tmem" keeps the hidden activations in tensor memory (the layout H = 256 always uses);
+    "wide" forces 128-row tiles where the batch is small enough for the few-rows form of the kernel
+    (H = 128: up to 16 rows per SM at 333 / 300 environments, up to 32 at 1500 / 1000)."""
     w = wl.workload(idx)
     if not _tc_available(w):
         pytest.skip("bf16 tensor-core path not compiled for this shape")
     params = wl.make_params(w, bias_scale=0.1)
-    flags = binding.MAVA_FLAG_WRITE_LOGITS | (binding.MAVA_FLAG_HIDDEN_IN_TMEM if tmem else 0)
+    flags = binding.MAVA_FLAG_WRITE_LOGITS | {"": 0, "tmem": binding.MAVA_FLAG_HIDDEN_IN_TMEM,
+                                              "wide": binding.MAVA_FLAG_WIDE_TILES}[mode]
     ro, _ = run_gpu(w, BF16, T, n_envs=n_envs, params=params, flags=flags)
     ids = wl.sample_env_ids(n_envs, 6, 6, 6, seed=idx)
     out = check_against_oracle(w, ro, params, T, BF16, ids)
@@ -91,6 +95,22 @@ def test_reduced_configs_bf16(idx, n_envs, T, tmem):
     assert np.max(np.abs(lg - ref.logits) / (1 + np.abs(ref.logits))) < 2e-3
     v = ro.values[:T + 1].cpu().numpy()[:, ids]
     assert np.max(np.abs(v - ref.values) / (1 + np.abs(ref.values))) < 2e-3
+
+
+@pytest.mark.parametrize("idx,n_envs", [(1, 1024), (1, 2000), (2, 700), (2, 1400)])
+def test_few_rows_form_equals_wide_tiles(idx, n_envs):
+    """The few-rows form of the bf16 kernel (rows as the N operand of the MMA) forms the same products
+    in the same order as the 128-row form: every output is bit-identical."""
+    w = wl.workload(idx)
+    T = 48
+    params = wl.make_params(w, bias_scale=0.1)
+    outs = []
+    for extra in (0, binding.MAVA_FLAG_WIDE_TILES):
+        ro, _ = run_gpu(w, BF16, T, n_envs=n_envs, params=params, flags=binding.MAVA_FLAG_WRITE_LOGITS | extra)
+        outs.append({k: getattr(ro, k)[:T + (1 if k == "values" else 0)].cpu().numpy().copy()
+                     for k in ("obs", "actions", "logp", "values", "rewards", "dones", "logits", "adv", "ret")})
+    for k in outs[0]:
+        assert np.array_equal(outs[0][k].view(np.uint8), outs[1][k].view(np.uint8)), k
 
 
 # ---- full-size configs in the launch configuration the benchmark times ------------------------
