@@ -347,14 +347,12 @@ __device__ void reset_env(EnvRegs<N, F> &s, const EnvParams &p, uint32_t env, ui
   s.total = total;
 }
 
-// Non-zero observation entries of agent `ag` (see observe_sparse for the element layout).
-template <int N, int F, class Sink>
-__device__ __forceinline__ void observe_env(const EnvRegs<N, F> &s, const EnvParams &p, int ag, Sink sink) {
-  uint32_t me = s.ent[0];
-#pragma unroll
-  for (int m = 1; m < N; ++m) me = (ag == m) ? s.ent[m] : me;
-  const int G = p.grid;
-  const int r0 = me & 0xFF, c0 = (me >> 8) & 0xFF;
+// Non-zero observation entries of one agent (see observe_sparse for the element layout), in three
+// parts that need different pieces of the state, so that different warps can produce them:
+// the wall plane (from the agent's cell), the two level planes (from all entities), and the
+// scalars (own level, step/cap, one-hot id).
+template <class Sink>
+__device__ __forceinline__ void observe_walls(int r0, int c0, int G, Sink sink) {
   bool row_out[kWindow], col_out[kWindow];
 #pragma unroll
   for (int d = 0; d < kWindow; ++d) {
@@ -366,6 +364,9 @@ __device__ __forceinline__ void observe_env(const EnvRegs<N, F> &s, const EnvPar
 #pragma unroll
     for (int dx = 0; dx < kWindow; ++dx)
       if (row_out[dy] || col_out[dx]) sink(2 * kPlane + dy * kWindow + dx, 1.0f);
+}
+template <int N, int F, class Sink>
+__device__ __forceinline__ void observe_levels(const EnvRegs<N, F> &s, int r0, int c0, Sink sink) {
 #pragma unroll
   for (int k = 0; k < N + F; ++k) {
     const uint32_t e = s.ent[k];
@@ -374,9 +375,27 @@ __device__ __forceinline__ void observe_env(const EnvRegs<N, F> &s, const EnvPar
     if (lvl > 0 && dy >= 0 && dy < kWindow && dx >= 0 && dx < kWindow)
       sink((k < N ? 0 : kPlane) + dy * kWindow + dx, static_cast<float>(lvl));
   }
-  sink(3 * kPlane, static_cast<float>(me >> 16));
-  sink(3 * kPlane + 1, __fdiv_rn(static_cast<float>(s.step), static_cast<float>(p.cap)));
+}
+template <class Sink>
+__device__ __forceinline__ void observe_scalars(int level, int step, int cap, int ag, Sink sink) {
+  sink(3 * kPlane, static_cast<float>(level));
+  sink(3 * kPlane + 1, __fdiv_rn(static_cast<float>(step), static_cast<float>(cap)));
   sink(kObsFixed + ag, 1.0f);
+}
+template <int N, int F>
+__device__ __forceinline__ uint32_t own_entity(const EnvRegs<N, F> &s, int ag) {
+  uint32_t me = s.ent[0];
+#pragma unroll
+  for (int m = 1; m < N; ++m) me = (ag == m) ? s.ent[m] : me;
+  return me;
+}
+template <int N, int F, class Sink>
+__device__ __forceinline__ void observe_env(const EnvRegs<N, F> &s, const EnvParams &p, int ag, Sink sink) {
+  const uint32_t me = own_entity(s, ag);
+  const int r0 = me & 0xFF, c0 = (me >> 8) & 0xFF;
+  observe_walls(r0, c0, p.grid, sink);
+  observe_levels<N, F>(s, r0, c0, sink);
+  observe_scalars(static_cast<int>(me >> 16), s.step, p.cap, ag, sink);
 }
 
 // One transition of the environment whose N agent threads occupy lanes [base, base + N) of this

@@ -8,7 +8,10 @@
 // The products and their order of accumulation (bias tile first, then K in ascending steps) are
 // those of the 128-row kernel, and so are the results.
 //   thread j of the CTA: hidden unit j in the epilogues (tensor-memory lane j);
-//   threads 0 .. RB-1 (warp 0): also agent row j of the tile: observation, sampler, transition.
+//   threads 0 .. RB-1 (warp 0): also agent row j of the tile: sampler, transition, level planes of
+//   the observation; after a transition they publish their cell, level and step count in shared
+//   memory, from which lane j of warp 1 writes row j's wall plane and lane j of warp 2 its scalars
+//   (this serial code is bound by instruction latency, so three warps finish it sooner than one).
 // Same weight image as the 128-row kernel; the heads (16 rows there) are copied into a zero-padded
 // 128-row operand once per CTA.
 #pragma once
@@ -39,6 +42,7 @@ struct SmallSmem {
   alignas(128) unsigned char ht[Q::HT_BYTES];       // bf16 hidden activations, N operand of layer 2 and of the heads
   alignas(128) unsigned char stage[Q::STAGE_BYTES]; // fp32 observation block in the global layout
   alignas(16) float logit[RB * 8];                  // heads' outputs, transposed for the row threads
+  alignas(8) uint32_t pub[RB * 2];                  // per row: own entity (cell, level), step count
   alignas(8) uint64_t mma_bar;
   alignas(8) uint64_t load_bar;
   uint32_t tmem_base;
@@ -109,7 +113,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
   }
   const uint32_t w_addr = smem_u32(sm.weights), wh_addr = smem_u32(sm.wh);
   const uint32_t x_addr = smem_u32(sm.x), ht_addr = smem_u32(sm.ht), stage_addr = smem_u32(sm.stage);
-  const uint32_t logit_addr = smem_u32(sm.logit);
+  const uint32_t logit_addr = smem_u32(sm.logit), pub_addr = smem_u32(sm.pub);
   for (int i = row; i < static_cast<int>(Q::X_BYTES / 16); i += kGroupThreads) sts_zero16(x_addr + 16u * i);
   for (int i = row; i < static_cast<int>(Q::HT_BYTES / 16); i += kGroupThreads) sts_zero16(ht_addr + 16u * i);
   for (int i = row; i < static_cast<int>(Q::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
@@ -185,19 +189,39 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
       }
       pend = false;
     };
+    auto publish = [&]() {
+      if (active) {
+        sts_f32(pub_addr + 8u * lane, __uint_as_float(own_entity(env, ag)));
+        sts_f32(pub_addr + 8u * lane + 4u, __int_as_float(env.step));
+      }
+    };
+    publish();
+    group_sync(0);
     for (int t = 0; t <= a.T; ++t) {
       const bool last = (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
-      // 1. non-zero observation entries into the zeroed operand and the zeroed fp32 block
-      if (active) {
-        const uint32_t x_row = x_addr + a_offset<K1>(row, 0);
-        observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
-          sts_f32(stage_addr + 4u * static_cast<uint32_t>(crow * D + j), v);
+      // 1. non-zero observation entries into the zeroed operand and the zeroed fp32 block:
+      //    warp 0 the level planes, warp 1 the walls, warp 2 the scalars of row = lane
+      if (wg < 3 && lane < n_rows) {
+        const uint32_t x_row = x_addr + a_offset<K1>(lane, 0);
+        auto sink = [&](int j, float v) {
+          sts_f32(stage_addr + 4u * static_cast<uint32_t>(lane * D + j), v);
           sts_u16(x_row + a_offset<K1>(0, j), bf16_bits(v));
-        });
-        if (S::FOLD1) {
-          sts_u16(x_row + a_offset<K1>(0, D), 0x3F80);
-          sts_u16(x_row + a_offset<K1>(0, D + 1), 0x3F80);
+        };
+        if (wg == 0) {
+          const uint32_t me = own_entity(env, ag);
+          observe_levels<N, F>(env, me & 0xFF, (me >> 8) & 0xFF, sink);
+        } else {
+          const uint32_t me = static_cast<uint32_t>(lds_s32(pub_addr + 8u * lane));
+          if (wg == 1) {
+            observe_walls(me & 0xFF, (me >> 8) & 0xFF, a.env.grid, sink);
+          } else {
+            observe_scalars(static_cast<int>(me >> 16), lds_s32(pub_addr + 8u * lane + 4u), a.env.cap, ag, sink);
+            if (S::FOLD1) {
+              sts_u16(x_row + a_offset<K1>(0, D), 0x3F80);
+              sts_u16(x_row + a_offset<K1>(0, D + 1), 0x3F80);
+            }
+          }
         }
       }
       fence_async_smem();
@@ -300,21 +324,22 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
           }
         }
       }
-      tc_fence_before();
-      if (group_any(0, timed_out)) {
-        timed_out = true;
-        break;
-      }
-      if (last) break;
-      // 5. transition and auto-reset, inside warp 0
-      if (wg == 0) {
+      // 5. transition and auto-reset, inside warp 0, which then publishes what warps 1 and 2 need
+      if (wg == 0 && !last) {
         float reward;
         bool done;
         step_env_warp<N, F>(env, a.env, env_id, ag, base, active, action, reward, done);
         pend_reward = reward;
         pend_done = done;
         pend_done_idx = static_cast<size_t>(t) * a.env.n_envs + e0 + le;
+        publish();
       }
+      tc_fence_before();
+      if (group_any(0, timed_out)) {  // also the barrier between publishing and the next observation
+        timed_out = true;
+        break;
+      }
+      if (last) break;
     }
     flush_outputs();
     if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
