@@ -13,8 +13,12 @@
 //   memory, from which lane j of warp 1 writes row j's wall plane and lane j of warp 2 its scalars
 //   (this serial code is bound by instruction latency, so three warps finish it sooner than one).
 // Same weight image as the 128-row kernel; the heads (16 rows there) are copied into a zero-padded
-// 128-row operand once per CTA.
+// 64-row operand once per CTA.
 #pragma once
+
+// The heads are an M = 64 operand (the smallest M): their seven rows come out in lanes 0..6; the
+// time of an MMA here is the time to stream its M operand from shared memory.
+constexpr int kHeadM = 64;
 
 template <int N, int H, int RB>
 struct SmallShape {
@@ -28,7 +32,7 @@ struct SmallShape {
   static constexpr uint32_t X_BYTES = (RB / 8) * (K1 / 8) * kALbo;
   static constexpr uint32_t HT_BYTES = (RB / 8) * (H / 8) * kALbo;
   static constexpr uint32_t STAGE_BYTES = (ROWS * D * 4 + 15) / 16 * 16;
-  static constexpr uint32_t WH_BYTES = kTileRows * H * 2;
+  static constexpr uint32_t WH_BYTES = kHeadM * H * 2;
   static constexpr int ACC_COL = 0, HEAD_COL = 32, TMEM_COLS = 64;
 };
 
@@ -37,12 +41,13 @@ struct SmallSmem {
   using S = TcShape<N, H, false>;
   using Q = SmallShape<N, H, RB>;
   alignas(128) unsigned char weights[S::IMAGE_BYTES];
-  alignas(128) unsigned char wh[Q::WH_BYTES];       // heads as a 128-row operand, rows 16.. zero
+  alignas(128) unsigned char wh[Q::WH_BYTES];       // heads as a 64-row operand, rows 16.. zero
   alignas(128) unsigned char x[Q::X_BYTES];         // bf16 observations, N operand of layer 1
   alignas(128) unsigned char ht[Q::HT_BYTES];       // bf16 hidden activations, N operand of layer 2 and of the heads
   alignas(128) unsigned char stage[Q::STAGE_BYTES]; // fp32 observation block in the global layout
   alignas(16) float logit[RB * 8];                  // heads' outputs, transposed for the row threads
   alignas(8) uint32_t pub[RB * 2];                  // per row: own entity (cell, level), step count
+  float uniform[RB];                                // per row: the uniform of this step's action draw
   alignas(8) uint64_t mma_bar;
   alignas(8) uint64_t load_bar;
   uint32_t tmem_base;
@@ -76,10 +81,10 @@ __device__ __forceinline__ void small_epilogue(uint32_t acc_taddr, uint32_t ht_a
 }
 
 // One dense layer, weights as the M operand: accumulator[unit][row] = bias[unit] + sum_k W[unit][k] x[row][k].
-template <int K, int RB, bool BIAS_TILE>
+template <int K, int RB, bool BIAS_TILE, int MROWS = kTileRows>
 __device__ __forceinline__ void small_issue_layer(uint32_t d_tmem, uint32_t w_addr, uint32_t x_addr, uint32_t bias_addr,
                                                   uint32_t ones_addr, uint32_t bar) {
-  constexpr uint32_t idesc = instr_desc(kTileRows, RB);
+  constexpr uint32_t idesc = instr_desc(MROWS, RB);
   if (BIAS_TILE) mma_bf16(d_tmem, smem_desc(bias_addr, 128, 256), smem_desc(ones_addr, 128, 256), idesc, 0);
 #pragma unroll
   for (int k = 0; k < K / 16; ++k)
@@ -87,6 +92,11 @@ __device__ __forceinline__ void small_issue_layer(uint32_t d_tmem, uint32_t w_ad
              idesc, (BIAS_TILE || k > 0) ? 1u : 0u);
   mma_commit(bar);
 }
+
+// The thread that issues the MMAs sits in the last warp: warp 0 has the rows' serial work to do
+// (stores of the previous step, the step's uniform) while a layer is being issued.
+constexpr int kIssuer = kGroupThreads - 32;
+constexpr int kCopier = 32;  // the thread that sends the observation block out (bulk copy)
 
 template <int N, int F, int H, int RB>
 __global__ void __launch_bounds__(kGroupThreads, 1)
@@ -113,7 +123,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
   }
   const uint32_t w_addr = smem_u32(sm.weights), wh_addr = smem_u32(sm.wh);
   const uint32_t x_addr = smem_u32(sm.x), ht_addr = smem_u32(sm.ht), stage_addr = smem_u32(sm.stage);
-  const uint32_t logit_addr = smem_u32(sm.logit), pub_addr = smem_u32(sm.pub);
+  const uint32_t logit_addr = smem_u32(sm.logit), pub_addr = smem_u32(sm.pub), uni_addr = smem_u32(sm.uniform);
   for (int i = row; i < static_cast<int>(Q::X_BYTES / 16); i += kGroupThreads) sts_zero16(x_addr + 16u * i);
   for (int i = row; i < static_cast<int>(Q::HT_BYTES / 16); i += kGroupThreads) sts_zero16(ht_addr + 16u * i);
   for (int i = row; i < static_cast<int>(Q::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
@@ -133,7 +143,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
   }
   timed_out = !mbar_wait(smem_u32(&sm.load_bar), 0);
   timed_out = __syncthreads_or(timed_out) != 0;
-  // the 16 head rows are the first two 8-row groups of the 128-row operand (same pitch)
+  // the 16 head rows are the first two 8-row groups of the 64-row operand (same pitch)
   for (int i = row; i < static_cast<int>(S::WH_BYTES / 16); i += kGroupThreads)
     *reinterpret_cast<uint4 *>(sm.wh + 16 * i) = *reinterpret_cast<const uint4 *>(sm.weights + S::WH_OFF + 16 * i);
   fence_async_smem();
@@ -228,17 +238,20 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
       tc_fence_before();
       group_sync(0);
       // 2. layer 1; meanwhile the previous step's outputs and the observation block leave
-      if (row == 0) {
-        tc_fence_after();
-        small_issue_layer<K1, RB, !S::FOLD1>(acc_col, w_addr + S::W1_OFF, x_addr, w_addr + S::B1_OFF, w_addr + S::ONES_OFF,
-                                             bar);
+      if (wg == kIssuer / 32) {  // its other lanes wait here rather than spin beside the issuing one
+        if (row == kIssuer) {
+          tc_fence_after();
+          small_issue_layer<K1, RB, !S::FOLD1>(acc_col, w_addr + S::W1_OFF, x_addr, w_addr + S::B1_OFF, w_addr + S::ONES_OFF,
+                                               bar);
+        }
+        __syncwarp();
       }
       flush_outputs();
       if (!last) {
         float *obs_dst = a.buf.obs + row0 * D;
         const int count = n_rows * D;
         if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
-          if (row == 0) {
+          if (row == kCopier) {
             bulk_store(obs_dst, stage_addr, static_cast<uint32_t>(count) * 4u);
             bulk_pending = true;
           }
@@ -254,12 +267,16 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
       tc_fence_before();
       group_sync(0);
       // 3. layer 2; meanwhile the uniform of this step's draw, and the observation operand is zeroed
-      if (row == 0) {
-        tc_fence_after();
-        small_issue_layer<H, RB, true>(acc_col, w_addr + S::W2_OFF, ht_addr, w_addr + S::B2_OFF, w_addr + S::ONES_OFF, bar);
+      if (wg == kIssuer / 32) {  // its other lanes wait here rather than spin beside the issuing one
+        if (row == kIssuer) {
+          tc_fence_after();
+          small_issue_layer<H, RB, true>(acc_col, w_addr + S::W2_OFF, ht_addr, w_addr + S::B2_OFF, w_addr + S::ONES_OFF, bar);
+        }
+        __syncwarp();
       }
-      float u = 0.0f;
-      if (active && !last) u = action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag));
+      if (wg == 2 && lane < n_rows && !last)  // the uniform of row = lane, for the sampler in warp 0
+        sts_f32(uni_addr + 4u * lane,
+                action_uniform(a.env, a.t_global0 + static_cast<uint32_t>(t), env_id, static_cast<uint32_t>(ag)));
       for (int i = row; i < static_cast<int>(Q::X_BYTES / 16); i += kGroupThreads) sts_zero16(x_addr + 16u * i);
       if (bulk_pending) { bulk_store_wait_read(); bulk_pending = false; }  // the block may be zeroed after the next barrier
       timed_out |= !mbar_wait(bar, phase);
@@ -270,9 +287,12 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
       tc_fence_before();
       group_sync(0);
       // 4. heads: lanes 0..5 the logits, lane 6 the value, one column per row
-      if (row == 0) {
-        tc_fence_after();
-        small_issue_layer<H, RB, false>(head_col, wh_addr, ht_addr, 0u, 0u, bar);
+      if (wg == kIssuer / 32) {  // its other lanes wait here rather than spin beside the issuing one
+        if (row == kIssuer) {
+          tc_fence_after();
+          small_issue_layer<H, RB, false, kHeadM>(head_col, wh_addr, ht_addr, 0u, 0u, bar);
+        }
+        __syncwarp();
       }
       for (int i = row; i < static_cast<int>(Q::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
       timed_out |= !mbar_wait(bar, phase);
@@ -294,6 +314,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
           for (int k = 0; k <= kActions; ++k) hv[k] = lds_f32(logit_addr + 4u * static_cast<uint32_t>(lane * 8 + k));
           pend = true; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
           if (!last) {
+            const float u = lds_f32(uni_addr + 4u * lane);
             float e[kActions];
             float m = hv[0];
 #pragma unroll
