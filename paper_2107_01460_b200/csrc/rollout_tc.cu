@@ -656,6 +656,10 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   int ept = (h->cfg.n_envs + slots - 1) / slots;
   if (ept > S::EPT_MAX) ept = S::EPT_MAX;
   if (ept < 1) ept = 1;
+  if (!TM) {  // tiles whose observation block is a whole number of 16-byte pieces leave as one bulk copy
+    for (int e = ept; e <= S::EPT_MAX; ++e)
+      if ((e * N * S::D) % 4 == 0) { ept = e; break; }
+  }
   const int n_tiles = (h->cfg.n_envs + ept - 1) / ept;
   const int ctas = (n_tiles + groups - 1) / groups;
   kern<<<ctas < sms ? ctas : sms, S::THREADS, smem, h->stream>>>(args, static_cast<const unsigned char *>(h->d_wtc), ept,

@@ -385,6 +385,10 @@ cudaError_t launch_tc_small(mava_rollout *h, const RolloutArgs &args, int sms) {
   int ept = (h->cfg.n_envs + sms - 1) / sms;  // the caller made sure this fits a tile
   if (ept > Q::EPT_MAX) ept = Q::EPT_MAX;
   if (ept < 1) ept = 1;
+  // A tile's observation block leaves as one bulk copy when it is a whole number of 16-byte pieces
+  // (every tile then also starts on such a boundary): take the next such size if the tile has room.
+  for (int e = ept; e <= Q::EPT_MAX; ++e)
+    if ((e * N * Q::D) % 4 == 0) { ept = e; break; }
   const int n_tiles = (h->cfg.n_envs + ept - 1) / ept;
   kern<<<n_tiles < sms ? n_tiles : sms, kGroupThreads, smem, h->stream>>>(args, static_cast<const unsigned char *>(h->d_wtc),
                                                                          ept, n_tiles);
