@@ -106,6 +106,11 @@ def lib():
             C.c_void_p,
         ]
         L.orc_rollout.restype = C.c_int
+        L.orc_evaluate.argtypes = [
+            C.POINTER(Config), C.c_uint64, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int32, C.c_uint32,
+            C.POINTER(EnvState), C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+        ]
+        L.orc_evaluate.restype = C.c_int
         L.orc_gae.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_double,
                               C.c_double, C.c_void_p, C.c_void_p]
         L.orc_gae.restype = None
@@ -232,6 +237,44 @@ def rollout(cfg: Config, seed: int, params, T: int, env_ids, *, forced_actions=N
     if rc != 0:
         raise ValueError("orc_rollout rejected its arguments")
     return Rollout(obs, actions, own, logp, values, rewards, dones, logits, margin, list(st))
+
+
+@dataclass
+class Evaluation:
+    ep_count: np.ndarray   # [n] int32
+    ret_sum: np.ndarray    # [n] float32
+    len_sum: np.ndarray    # [n] int32
+    actions: np.ndarray    # [T][n][N] int32
+    logits: np.ndarray     # [T][n][N][6] float64
+    states: list
+
+
+def evaluate(cfg: Config, seed: int, params, T: int, env_ids, *, greedy: bool = True, forced_actions=None,
+             states=None, t_global0: int = 0, emulate_bf16: bool = False) -> Evaluation:
+    """An evaluation block of T steps over the listed environments (see orc_evaluate)."""
+    env_ids = np.ascontiguousarray(env_ids, dtype=np.int32)
+    n = int(env_ids.size)
+    N = cfg.n_agents
+    if states is None:
+        states = [env_reset(cfg, seed, int(e), 0) for e in env_ids]
+    st = (EnvState * n)(*states)
+    fa = None
+    if forced_actions is not None:
+        fa = np.ascontiguousarray(forced_actions, dtype=np.int32)
+        assert fa.shape == (T, n, N)
+    p = np.ascontiguousarray(params, dtype=np.float32)
+    assert p.size == params_count(cfg)
+    ep = np.empty(n, dtype=np.int32)
+    rs = np.empty(n, dtype=np.float32)
+    ls = np.empty(n, dtype=np.int32)
+    actions = np.empty((T, n, N), dtype=np.int32)
+    logits = np.empty((T, n, N, N_ACTIONS), dtype=np.float64)
+    rc = lib().orc_evaluate(C.byref(cfg), C.c_uint64(seed), _ptr(p), int(emulate_bf16), n, _ptr(env_ids), T,
+                            t_global0, st, _ptr(fa), int(greedy), _ptr(ep), _ptr(rs), _ptr(ls), _ptr(actions),
+                            _ptr(logits))
+    if rc != 0:
+        raise ValueError("orc_evaluate rejected its arguments")
+    return Evaluation(ep, rs, ls, actions, logits, list(st))
 
 
 def gae(values, rewards, dones, gamma: float, lam: float):

@@ -4,8 +4,8 @@
  * TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, obviously-correct
  * restatement of what the rollout computes: the foraging gridworld
  * (reset, observation, transition, reward, done), the shared actor-critic MLP,
- * the Philox4x32-10 inverse-CDF categorical sampler, and generalised advantage
- * estimation.  It shares no code with the CUDA library and is used only by the
+ * the Philox4x32-10 inverse-CDF categorical sampler, generalised advantage
+ * estimation, and the evaluation block (greedy or sampled episodes, returns).  It shares no code with the CUDA library and is used only by the
  * tests, by the smoke check and by the benchmark's CPU-baseline leg.
  *
  * The technical report this follows describes the loop only in words
@@ -429,6 +429,81 @@ int orc_rollout(const orc_config_t *cfg, uint64_t seed, const float *params, int
       if (rewards) for (int n = 0; n < N; ++n) rewards[row0 + n] = reward;
       if (dones) dones[(size_t)t * E_arr + p] = done;
       if (done) orc_env_reset(cfg, seed, env, s->episode + 1, s);
+    }
+  }
+  free(o);
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Evaluation block (Section 2, "Multi-device training with easy checkpointing */
+/* and logging": training is interleaved with blocks that run the current      */
+/* policy and report how its episodes went).  The report gives no more than    */
+/* that; the reading taken here: T steps of the same loop as the rollout       */
+/* (observe, actor forward, act, transition, auto-reset) with no trajectory    */
+/* kept.  The action is the arg max of the six logits (lowest index on a tie)  */
+/* when `greedy`, else the rollout's Philox inverse-CDF draw.  Per environment */
+/* three sums over the episodes that END inside the block:                     */
+/*   ep_count  how many ended,                                                 */
+/*   ret_sum   the sum of their returns; an episode's return is the sum of its */
+/*             (shared) step rewards received inside the block, accumulated in */
+/*             binary32 in step order, and the returns are added to ret_sum in */
+/*             binary32 in the order the episodes end,                         */
+/*   len_sum   the sum of their lengths in steps inside the block.             */
+/* An episode still running when the block ends is not counted.  Arrays are    */
+/* indexed by position in env_ids; forced_actions / actions / logits are       */
+/* [T][n_local][N](x6), any of them may be NULL.                               */
+/* ------------------------------------------------------------------------- */
+int orc_evaluate(const orc_config_t *cfg, uint64_t seed, const float *params, int emulate_bf16,
+                 int32_t n_local, const int32_t *env_ids, int32_t T, uint32_t t_global0,
+                 orc_env_state_t *states, const int32_t *forced_actions, int greedy,
+                 int32_t *ep_count, float *ret_sum, int32_t *len_sum, int32_t *actions,
+                 double *logits) {
+  const int N = cfg->n_agents, D = orc_obs_dim(cfg);
+  if (N > ORC_MAX_AGENTS || cfg->n_food > ORC_MAX_FOOD || !params) return -1;
+  float *o = (float *)malloc(sizeof(float) * (size_t)N * D);
+  double lg[ORC_MAX_AGENTS * ORC_N_ACTIONS], val[ORC_MAX_AGENTS], lp[ORC_N_ACTIONS];
+  int32_t act[ORC_MAX_AGENTS];
+  for (int i = 0; i < n_local; ++i) {
+    const int32_t env = env_ids[i];
+    orc_env_state_t *s = &states[i];
+    float running = 0.0f; /* return of the episode in progress */
+    int32_t length = 0;   /* its steps so far                  */
+    ep_count[i] = 0; ret_sum[i] = 0.0f; len_sum[i] = 0;
+    for (int t = 0; t < T; ++t) {
+      const size_t row0 = ((size_t)t * n_local + (size_t)i) * N;
+      for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
+      orc_mlp_forward_env(cfg, params, o, emulate_bf16, lg, val);
+      for (int n = 0; n < N; ++n) {
+        const double *l = lg + n * ORC_N_ACTIONS;
+        int32_t own = 0;
+        if (greedy) {
+          for (int k = 1; k < ORC_N_ACTIONS; ++k)
+            if (l[k] > l[own]) own = k;
+        } else {
+          double mg;
+          const float u = orc_action_uniform(seed, t_global0 + (uint32_t)t, (uint32_t)env, (uint32_t)n);
+          orc_sample(l, u, &own, lp, &mg);
+        }
+        act[n] = forced_actions ? forced_actions[row0 + n] : own;
+        if (act[n] < 0 || act[n] >= ORC_N_ACTIONS) { free(o); return -1; }
+        if (actions) actions[row0 + n] = act[n];
+        if (logits)
+          for (int k = 0; k < ORC_N_ACTIONS; ++k) logits[(row0 + n) * ORC_N_ACTIONS + k] = l[k];
+      }
+      float reward;
+      uint8_t done;
+      orc_env_step(cfg, s, act, &reward, &done);
+      running += reward;
+      length += 1;
+      if (done) {
+        ep_count[i] += 1;
+        ret_sum[i] += running;
+        len_sum[i] += length;
+        running = 0.0f;
+        length = 0;
+        orc_env_reset(cfg, seed, env, s->episode + 1, s);
+      }
     }
   }
   free(o);
