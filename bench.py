@@ -224,6 +224,21 @@ def time_workload(torch, binding, w, precision, steps, warmup, first_env=0, flus
     return ro, params, t_roll, t_gae, launches
 
 
+def time_evaluate(torch, ro, params, w, steps, warmup, flush):
+    """Device timing of greedy evaluation blocks of the workload's T steps (ms per block)."""
+    times = []
+    for i in range(warmup + steps):
+        flush.add_(1.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ro.evaluate(params, w["T"], greedy=True)
+        e1.record()
+        e1.synchronize()
+        if i >= warmup:
+            times.append(e0.elapsed_time(e1))
+    return sum(times) / len(times)
+
+
 def time_e2e(torch, binding, ro, w, steps, warmup):
     T, E, N, D = w["T"], w["n_envs"], w["n_agents"], wl.obs_dim(w)
     pin = lambda shape, dt: torch.empty(shape, dtype=dt).pin_memory()  # noqa: E731
@@ -282,6 +297,7 @@ def run_gpu(args):
         dist.barrier()
     step_ms = (sum(t_roll) + sum(t_gae)) / args.steps
     e2e_s, h2d, d2h = time_e2e(torch, binding, ro, w, max(3, args.steps // 4), 2)
+    eval_ms = time_evaluate(torch, ro, params, w, max(3, args.steps // 4), 3, flush)  # rank-local, reported by rank 0
     if dist is not None:
         t = torch.tensor([step_ms, e2e_s], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -355,6 +371,8 @@ def run_gpu(args):
         "gpu_launches": launches,
         "roofline": roofline,
         "gae": gae,
+        "evaluate": {"value": rows / (eval_ms * 1e-3), "unit": UNIT, "ms_per_block": eval_ms,
+                     "block": f"greedy, T={T} steps, no trajectory stored (mava_rollout_evaluate), one GPU"},
         "cpu_baseline": {"value": cpu_rows / cpu_s, "unit": UNIT, "cores": used, "kind": "oracle",
                          "sample": f"first {n_sample} of {E} envs x full T={T} (rollout + GAE), {passes} pass(es), {cpu_s:.1f} s wall"},
         "workloads": sweep,

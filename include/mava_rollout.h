@@ -129,6 +129,22 @@ int mava_rollout_run(mava_rollout_t *h, const float *params_dev, int32_t T);
 int mava_rollout_run_forced(mava_rollout_t *h, const float *params_dev, int32_t T,
                             const int32_t *actions_dev);
 
+/* Evaluation block (Section 2, "Multi-device training with easy checkpointing and logging":
+ * training is interleaved with blocks that run the current policy to report how it does).  The
+ * same loop as the rollout for T >= 1 steps (not limited by max_T), continuing from the handle's
+ * environment states and step counter and advancing both, but nothing of the trajectory is stored
+ * and the caller's buffers are not touched.  greedy != 0: every action is the arg max of its six
+ * logits, the lowest index on a tie; greedy == 0: the rollout's Philox draw.  Outputs, device
+ * pointers to n_envs elements each, written by the call's kernels, over the episodes that END
+ * inside the block: ep_count how many, ret_sum the sum of their returns (an episode's return is
+ * the sum of its shared step rewards received inside the block; fp32 sums in step order), len_sum
+ * the sum of their lengths in steps inside the block.  An episode still running at the end of the
+ * block is not counted.  actions_dev: NULL, or [T][E][N] int32 that receives the actions taken.
+ * The centralised critic is not evaluated.  Asynchronous.  Errors: INVALID_ARG, CUDA. */
+int mava_rollout_evaluate(mava_rollout_t *h, const float *params_dev, int32_t T, int32_t greedy,
+                          int32_t *ep_count_dev, float *ret_sum_dev, int32_t *len_sum_dev,
+                          int32_t *actions_dev);
+
 /* Generalised advantage estimation over the rows of the last run (multi-agent PPO, Section 2):
  *   delta_t = r_t + gamma V_{t+1} (1-d_t) - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1},
  *   A_T = 0;  Ret_t = A_t + V_t.

@@ -29,7 +29,7 @@ EXPORTS = [
     "mava_params_count", "mava_rollout_create", "mava_rollout_run", "mava_rollout_run_forced", "mava_gae",
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
-    "mava_strerror", "mava_rollout_run_static",
+    "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate",
 ]
 
 
@@ -67,6 +67,8 @@ def lib():
         L.mava_rollout_create.argtypes = [cfgp, bufp, vp, C.POINTER(vp)]; L.mava_rollout_create.restype = C.c_int
         L.mava_rollout_run.argtypes = [vp, vp, C.c_int32]; L.mava_rollout_run.restype = C.c_int
         L.mava_rollout_run_forced.argtypes = [vp, vp, C.c_int32, vp]; L.mava_rollout_run_forced.restype = C.c_int
+        L.mava_rollout_evaluate.argtypes = [vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp]
+        L.mava_rollout_evaluate.restype = C.c_int
         L.mava_gae.argtypes = [vp, C.c_float, C.c_float]; L.mava_gae.restype = C.c_int
         L.mava_rollout_reset.argtypes = [vp, C.c_uint64]; L.mava_rollout_reset.restype = C.c_int
         L.mava_rollout_status.argtypes = [vp]; L.mava_rollout_status.restype = C.c_int
@@ -157,6 +159,22 @@ class Rollout:
         assert params.is_cuda and params.numel() == self.n_params
         _check(lib().mava_rollout_run_forced(self.handle, params.data_ptr(), T, actions.data_ptr()),
                "mava_rollout_run_forced")
+
+    def evaluate(self, params, T: int, greedy: bool = True, want_actions: bool = False):
+        """An evaluation block of T steps (mava_rollout_evaluate): returns device tensors
+        (ep_count [E] int32, ret_sum [E] float32, len_sum [E] int32, actions [T][E][N] int32 or None)."""
+        t = self.torch
+        assert params.is_cuda and params.dtype == t.float32 and params.numel() == self.n_params
+        E, N = self.cfg.n_envs, self.cfg.n_agents
+        dev = params.device
+        ep_count = t.empty(E, dtype=t.int32, device=dev)
+        ret_sum = t.empty(E, dtype=t.float32, device=dev)
+        len_sum = t.empty(E, dtype=t.int32, device=dev)
+        actions = t.empty((T, E, N), dtype=t.int32, device=dev) if want_actions else None
+        _check(lib().mava_rollout_evaluate(self.handle, params.data_ptr(), T, int(greedy), ep_count.data_ptr(),
+                                           ret_sum.data_ptr(), len_sum.data_ptr(),
+                                           actions.data_ptr() if want_actions else None), "mava_rollout_evaluate")
+        return ep_count, ret_sum, len_sum, actions
 
     def gae(self, gamma: float, lam: float):
         _check(lib().mava_gae(self.handle, gamma, lam), "mava_gae")

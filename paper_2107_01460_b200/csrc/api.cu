@@ -37,10 +37,19 @@ struct DeviceGuard {  // makes the handle's device current for the duration of a
   }
 };
 
-int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_t *forced) {
+// What an evaluation block adds to a launch (nullptr: a rollout).
+struct EvalRequest {
+  int32_t greedy;
+  int32_t *count;
+  float *ret;
+  int32_t *len;
+  int32_t *actions;
+};
+
+int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_t *forced, const EvalRequest *ev = nullptr) {
   if (!h || !params_dev) return MAVA_ERR_INVALID_ARG;
   if (T < 1) return MAVA_ERR_INVALID_ARG;
-  if (T > h->cfg.max_T) return MAVA_ERR_CAPACITY;
+  if (!ev && T > h->cfg.max_T) return MAVA_ERR_CAPACITY;  // an evaluation block stores no trajectory
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
   RolloutArgs args{};
@@ -53,18 +62,24 @@ int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_
   args.write_logits = (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) ? 1 : 0;
   args.status = h->d_status;
   args.obs_last = h->d_obs_last;
+  if (ev) {
+    args.eval = 1;
+    args.greedy = ev->greedy;
+    args.ev_count = ev->count; args.ev_ret = ev->ret; args.ev_len = ev->len; args.ev_actions = ev->actions;
+    args.obs_last = nullptr;
+  }
   cudaError_t err;
   if (h->cfg.precision == MAVA_PRECISION_BF16) {
     err = launch_prep_tc(h, params_dev);
     if (err == cudaSuccess) err = launch_rollout_tc(h, args);
-    if (err == cudaSuccess && h->cfg.net_kind == MAVA_NET_CENTRAL_CRITIC) err = launch_critic_tc(h, params_dev, T);
+    if (err == cudaSuccess && !ev && h->cfg.net_kind == MAVA_NET_CENTRAL_CRITIC) err = launch_critic_tc(h, params_dev, T);
   } else {
     err = launch_prep_simt(h, params_dev);
     if (err == cudaSuccess) err = launch_rollout_simt(h, args);
   }
   if (err != cudaSuccess) return MAVA_ERR_CUDA;
   h->t_global += static_cast<uint32_t>(T);
-  h->last_T = T;
+  if (!ev) h->last_T = T;
   return MAVA_OK;
 }
 
@@ -141,6 +156,13 @@ int mava_rollout_run(mava_rollout_t *h, const float *params_dev, int32_t T) {
 int mava_rollout_run_forced(mava_rollout_t *h, const float *params_dev, int32_t T, const int32_t *actions_dev) {
   if (!actions_dev) return MAVA_ERR_INVALID_ARG;
   return run_common(h, params_dev, T, actions_dev);
+}
+
+int mava_rollout_evaluate(mava_rollout_t *h, const float *params_dev, int32_t T, int32_t greedy, int32_t *ep_count_dev,
+                          float *ret_sum_dev, int32_t *len_sum_dev, int32_t *actions_dev) {
+  if (!ep_count_dev || !ret_sum_dev || !len_sum_dev) return MAVA_ERR_INVALID_ARG;
+  const EvalRequest ev{greedy ? 1 : 0, ep_count_dev, ret_sum_dev, len_sum_dev, actions_dev};
+  return run_common(h, params_dev, T, nullptr, &ev);
 }
 
 int mava_gae(mava_rollout_t *h, float gamma, float lambda) {

@@ -47,7 +47,39 @@ struct RolloutArgs {
   int32_t write_logits;
   int *status;
   float *obs_last;  // bf16 path with a centralised critic: where the observation after the last step goes
+  // Evaluation block: no trajectory is stored; per environment the episodes ending inside the block
+  // are counted and their returns and lengths summed.
+  int32_t eval;         // 0: rollout, 1: evaluation block
+  int32_t greedy;       // evaluation: arg max of the logits (lowest index on a tie) instead of the draw
+  int32_t *ev_count;    // [E]
+  float *ev_ret;        // [E]
+  int32_t *ev_len;      // [E]
+  int32_t *ev_actions;  // [T][E][N] or nullptr
 };
+
+// Episode bookkeeping of one environment inside an evaluation block (all in step order, fp32 sums).
+struct EvalSums {
+  float running = 0.0f, ret = 0.0f;  // return of the episode in progress; sum over the finished ones
+  int32_t length = 0, len = 0, count = 0;
+  __device__ __forceinline__ void step(float reward, bool done) {
+    running += reward;
+    length += 1;
+    if (done) {
+      count += 1; ret += running; len += length;
+      running = 0.0f; length = 0;
+    }
+  }
+};
+
+// Index of the largest of the six logits, the lowest index on a tie.
+__device__ __forceinline__ int greedy_action(const float *l) {
+  int best = 0;
+  float top = l[0];
+#pragma unroll
+  for (int k = 1; k < kActions; ++k)
+    if (l[k] > top) { top = l[k]; best = k; }
+  return best;
+}
 
 // Re-laid-out fp32 weights of the SIMT path: every dense layer transposed to [in][out].
 struct SimtWeights {

@@ -84,8 +84,10 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
   for (int i = tid; i < kSimtRows * D; i += kSimtThreads) sm.obs[i] = 0.0f;
   __syncthreads();
 
-  for (int t = 0; t <= a.T; ++t) {
-    const bool last = (t == a.T);
+  const bool ev = a.eval != 0;
+  EvalSums sums;  // thread tid < n_env: environment e0 + tid
+  for (int t = 0; t <= (ev ? a.T - 1 : a.T); ++t) {
+    const bool last = !ev && (t == a.T);
     const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
     auto sink = [&](int row, int j, float v) { sm.obs[row * D + j] = v; };
     observe_fill<N>(sm.st, a.env, n_rows, tid, kSimtThreads, sink);
@@ -93,7 +95,7 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
     observe_scatter<N, F>(sm.st, n_rows, tid, kSimtThreads, sink);
     __syncthreads();
 
-    if (!last) {  // the tile's rows are one contiguous block of the time-major obs array
+    if (!last && !ev) {  // the tile's rows are one contiguous block of the time-major obs array
       float *dst = a.buf.obs + row0 * D;
       const int count = n_rows * D;
       if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
@@ -134,7 +136,7 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
     }
 
     if (tid < n_rows) {
-      a.buf.values[row0 + tid] = sm.value[tid];
+      if (!ev) a.buf.values[row0 + tid] = sm.value[tid];
       if (!last) {
         const int le = tid / N, ag = tid - le * N;
         float l[kActions], e[kActions];
@@ -159,15 +161,20 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
           action = a.forced[row0 + tid];
           if (action < 0 || action >= kActions) action = 0;
         }
+        if (ev && a.greedy) action = greedy_action(l);
         float la = l[0];
 #pragma unroll
         for (int k = 1; k < kActions; ++k) la = (action == k) ? l[k] : la;
         sm.act[tid] = action;
-        a.buf.actions[row0 + tid] = action;
-        a.buf.logp[row0 + tid] = la - m - logf(sum);
-        if (a.write_logits) {
+        if (ev) {
+          if (a.ev_actions) a.ev_actions[row0 + tid] = action;
+        } else {
+          a.buf.actions[row0 + tid] = action;
+          a.buf.logp[row0 + tid] = la - m - logf(sum);
+          if (a.write_logits) {
 #pragma unroll
-          for (int k = 0; k < kActions; ++k) a.buf.logits[(row0 + tid) * kActions + k] = l[k];
+            for (int k = 0; k < kActions; ++k) a.buf.logits[(row0 + tid) * kActions + k] = l[k];
+          }
         }
       }
     }
@@ -181,10 +188,17 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
       bool done;
       step_apply<N, F>(sm.st[tid], a.env, static_cast<uint32_t>(a.env.first_env + e0 + tid), sm.new_r, sm.new_c,
                        sm.collected, tid, reward, done);
-      for (int n = 0; n < N; ++n) a.buf.rewards[row0 + tid * N + n] = reward;
-      a.buf.dones[static_cast<size_t>(t) * a.env.n_envs + e0 + tid] = done ? 1 : 0;
+      if (ev) {
+        sums.step(reward, done);
+      } else {
+        for (int n = 0; n < N; ++n) a.buf.rewards[row0 + tid * N + n] = reward;
+        a.buf.dones[static_cast<size_t>(t) * a.env.n_envs + e0 + tid] = done ? 1 : 0;
+      }
     }
     __syncthreads();
+  }
+  if (ev && tid < n_env) {
+    a.ev_count[e0 + tid] = sums.count; a.ev_ret[e0 + tid] = sums.ret; a.ev_len[e0 + tid] = sums.len;
   }
 
   for (int i = tid; i < n_env * static_cast<int>(sizeof(EnvRec) / 4); i += kSimtThreads)

@@ -306,7 +306,7 @@ __device__ __forceinline__ void expand_quads(const QuadPlan<D, K1> &p, uint32_t 
 }
 
 // ---- the rollout kernel ------------------------------------------------------------------------
-template <int N, int F, int H, bool TM>
+template <int N, int F, int H, bool TM, bool EVAL>
 __global__ void __launch_bounds__(TcShape<N, H, TM>::THREADS, 1)
 rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles, int groups) {
   using S = TcShape<N, H, TM>;
@@ -435,8 +435,10 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       }
       pend = false;
     };
-    for (int t = 0; t <= a.T; ++t) {
-      const bool last = (t == a.T);
+    constexpr bool ev = EVAL;     // evaluation block: nothing of the trajectory is stored
+    EvalSums sums;                // lanes with ag == 0: their environment
+    for (int t = 0; t <= (ev ? a.T - 1 : a.T); ++t) {
+      const bool last = !ev && (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
       if (PP) {
         pair_sync(kBarTile + g);  // the other group is done with the A tile
@@ -481,7 +483,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       }
       flush_outputs();  // the previous step's rows
       float *obs_dst = a.buf.obs + row0 * D;
-      if (!last && !PP) {
+      if (!last && !PP && !ev) {
         if (!TM) {  // one contiguous piece of the time-major array
           // by the bulk-copy engine when alignment allows: it leaves the load/store pipe to the
           // other group; the block was fenced for the async proxy together with the A tile
@@ -528,7 +530,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads) sts_zero16(a_addr + 16u * i);
       }
       if (PP) {
-        if (!last || a.obs_last != nullptr) {  // the observation after the last step feeds a centralised critic
+        if (!ev && (!last || a.obs_last != nullptr)) {  // the observation after the last step feeds a centralised critic
           float *dst = last ? a.obs_last + static_cast<size_t>(e0) * N * D : obs_dst;
           if constexpr (N % 4 == 0)
             expand_quads<D, K1>(quad_plan, a_addr, frac_addr, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32,
@@ -564,7 +566,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         if (!TM)  // the hidden activations are dead: zero the observation block for the next step
           for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
         if (active) {
-          pend = true; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
+          pend = !ev; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
           if (!last) {
             float e[kActions];
             float m = hv[0];
@@ -585,6 +587,10 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
             if (a.forced) {
               action = a.forced[row0 + crow];
               if (action < 0 || action >= kActions) action = 0;
+            }
+            if (ev) {
+              if (a.greedy) action = greedy_action(hv);
+              if (a.ev_actions) a.ev_actions[row0 + crow] = action;
             }
             float la = hv[0];
 #pragma unroll
@@ -612,9 +618,13 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       pend_reward = reward;
       pend_done = done;
       pend_done_idx = static_cast<size_t>(t) * a.env.n_envs + e0 + le;
+      if (ev) sums.step(reward, done);
     }
     flush_outputs();  // the last step's rows (the bootstrap values among them)
-    if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
+    if (!timed_out && active && ag == 0) {
+      store_env(env, a.state[e0 + le]);
+      if (ev) { a.ev_count[e0 + le] = sums.count; a.ev_ret[e0 + le] = sums.ret; a.ev_len[e0 + le] = sums.len; }
+    }
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
 
@@ -633,7 +643,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
 template <int N, int F, int H, bool TM>
 cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   using S = TcShape<N, H, TM>;
-  auto kern = rollout_tc_kernel<N, F, H, TM>;
+  auto kern = args.eval ? rollout_tc_kernel<N, F, H, TM, true> : rollout_tc_kernel<N, F, H, TM, false>;
   const size_t smem = sizeof(TcSmem<N, F, H, TM>);
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (err != cudaSuccess) return err;

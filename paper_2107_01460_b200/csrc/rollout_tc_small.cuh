@@ -98,7 +98,7 @@ __device__ __forceinline__ void small_issue_layer(uint32_t d_tmem, uint32_t w_ad
 constexpr int kIssuer = kGroupThreads - 32;
 constexpr int kCopier = 32;  // the thread that sends the observation block out (bulk copy)
 
-template <int N, int F, int H, int RB>
+template <int N, int F, int H, int RB, bool EVAL>
 __global__ void __launch_bounds__(kGroupThreads, 1)
 rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles) {
   using S = TcShape<N, H, false>;
@@ -207,8 +207,10 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
     };
     publish();
     group_sync(0);
-    for (int t = 0; t <= a.T; ++t) {
-      const bool last = (t == a.T);
+    constexpr bool ev = EVAL;     // evaluation block: nothing of the trajectory is stored
+    EvalSums sums;                // lanes with ag == 0: their environment
+    for (int t = 0; t <= (ev ? a.T - 1 : a.T); ++t) {
+      const bool last = !ev && (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
       // 1. non-zero observation entries into the zeroed operand and the zeroed fp32 block:
       //    warp 0 the level planes, warp 1 the walls, warp 2 the scalars of row = lane
@@ -247,7 +249,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
         __syncwarp();
       }
       flush_outputs();
-      if (!last) {
+      if (!last && !ev) {
         float *obs_dst = a.buf.obs + row0 * D;
         const int count = n_rows * D;
         if (((row0 * D) & 3) == 0 && (count & 3) == 0) {
@@ -312,7 +314,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
           float hv[kActions + 1];
 #pragma unroll
           for (int k = 0; k <= kActions; ++k) hv[k] = lds_f32(logit_addr + 4u * static_cast<uint32_t>(lane * 8 + k));
-          pend = true; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
+          pend = !ev; pend_step = !last; pend_row0 = row0; pend_value = hv[kActions];
           if (!last) {
             const float u = lds_f32(uni_addr + 4u * lane);
             float e[kActions];
@@ -335,6 +337,10 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
               action = a.forced[row0 + crow];
               if (action < 0 || action >= kActions) action = 0;
             }
+            if (ev) {
+              if (a.greedy) action = greedy_action(hv);
+              if (a.ev_actions) a.ev_actions[row0 + crow] = action;
+            }
             float la = hv[0];
 #pragma unroll
             for (int k = 1; k < kActions; ++k) la = (action == k) ? hv[k] : la;
@@ -353,6 +359,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
         pend_reward = reward;
         pend_done = done;
         pend_done_idx = static_cast<size_t>(t) * a.env.n_envs + e0 + le;
+        if (ev) sums.step(reward, done);
         publish();
       }
       tc_fence_before();
@@ -363,7 +370,10 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
       if (last) break;
     }
     flush_outputs();
-    if (!timed_out && active && ag == 0) store_env(env, a.state[e0 + le]);
+    if (!timed_out && active && ag == 0) {
+      store_env(env, a.state[e0 + le]);
+      if (ev) { a.ev_count[e0 + le] = sums.count; a.ev_ret[e0 + le] = sums.ret; a.ev_len[e0 + le] = sums.len; }
+    }
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
   bulk_store_wait_all();
@@ -378,7 +388,7 @@ rollout_tc_small_kernel(RolloutArgs a, const unsigned char *__restrict__ image, 
 template <int N, int F, int H, int RB>
 cudaError_t launch_tc_small(mava_rollout *h, const RolloutArgs &args, int sms) {
   using Q = SmallShape<N, H, RB>;
-  auto kern = rollout_tc_small_kernel<N, F, H, RB>;
+  auto kern = args.eval ? rollout_tc_small_kernel<N, F, H, RB, true> : rollout_tc_small_kernel<N, F, H, RB, false>;
   const size_t smem = sizeof(SmallSmem<N, F, H, RB>);
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (err != cudaSuccess) return err;
