@@ -46,15 +46,24 @@ struct EvalRequest {
   int32_t *actions;
 };
 
-int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_t *forced, const EvalRequest *ev = nullptr) {
+// `t_first`: the time row of the caller's buffers that step 0 of this launch writes (collect_host
+// rolls a trajectory out in pieces).
+int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_t *forced, const EvalRequest *ev = nullptr,
+               int32_t t_first = 0) {
   if (!h || !params_dev) return MAVA_ERR_INVALID_ARG;
-  if (T < 1) return MAVA_ERR_INVALID_ARG;
-  if (!ev && T > h->cfg.max_T) return MAVA_ERR_CAPACITY;  // an evaluation block stores no trajectory
+  if (T < 1 || t_first < 0) return MAVA_ERR_INVALID_ARG;
+  if (!ev && t_first + T > h->cfg.max_T) return MAVA_ERR_CAPACITY;  // an evaluation block stores no trajectory
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
   RolloutArgs args{};
   args.env = env_params(h);
   args.buf = h->buf;
+  if (t_first > 0) {  // rows t_first.. of every time-major array
+    const size_t E = static_cast<size_t>(h->cfg.n_envs), M = E * h->cfg.n_agents, r0 = M * t_first;
+    args.buf.obs += r0 * h->D; args.buf.actions += r0; args.buf.logp += r0; args.buf.values += r0;
+    args.buf.rewards += r0; args.buf.dones += E * t_first;
+    if (args.buf.logits) args.buf.logits += r0 * kActions;
+  }
   args.state = h->d_state;
   args.forced = forced;
   args.T = T;
@@ -79,7 +88,7 @@ int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_
   }
   if (err != cudaSuccess) return MAVA_ERR_CUDA;
   h->t_global += static_cast<uint32_t>(T);
-  if (!ev) h->last_T = T;
+  if (!ev) h->last_T = t_first + T;
   return MAVA_OK;
 }
 
@@ -258,28 +267,56 @@ int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32
   if (cudaMemcpyAsync(h->d_params_stage, params_host, np * sizeof(float), cudaMemcpyHostToDevice, h->stream) !=
       cudaSuccess)
     return MAVA_ERR_CUDA;
-  int rc = run_common(h, h->d_params_stage, T, nullptr);
-  if (rc != MAVA_OK) return rc;
-  if (h->buf.adv && h->buf.ret) {
-    rc = mava_gae(h, gamma, lambda);
-    if (rc != MAVA_OK) return rc;
+  if (T < 1) return MAVA_ERR_INVALID_ARG;
+  if (T > h->cfg.max_T) return MAVA_ERR_CAPACITY;
+  if (!h->copy_ready) {
+    bool made = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; made && i <= kCollectChunks; ++i)
+      made = cudaEventCreateWithFlags(&h->chunk_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!made) return MAVA_ERR_CUDA;
+    h->copy_ready = true;
   }
-  const size_t E = static_cast<size_t>(h->cfg.n_envs), M = E * h->cfg.n_agents, rows = M * T;
+  // The copies are bound by the host link and take several times as long as the kernels, so the
+  // rollout is cut into pieces in time (two calls continue like one) and the rows of a finished
+  // piece travel while the next piece runs.  The centralised critic works on the whole trajectory
+  // at once and is not cut.
+  const int chunks = (h->cfg.net_kind == MAVA_NET_CENTRAL_CRITIC || T < 2 * kCollectChunks) ? 1 : kCollectChunks;
+  const size_t E = static_cast<size_t>(h->cfg.n_envs), M = E * h->cfg.n_agents;
   bool ok = true;
-  auto back = [&](void *dst, const void *src, size_t bytes) {
+  auto back = [&](void *dst, const void *src, size_t offset, size_t bytes) {
     if (dst && src && ok)
-      ok = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, h->stream) == cudaSuccess;
+      ok = cudaMemcpyAsync(static_cast<unsigned char *>(dst) + offset, static_cast<const unsigned char *>(src) + offset, bytes,
+                           cudaMemcpyDeviceToHost, h->copy_stream) == cudaSuccess;
   };
-  back(out->obs, h->buf.obs, rows * h->D * sizeof(float));
-  back(out->actions, h->buf.actions, rows * sizeof(int32_t));
-  back(out->logp, h->buf.logp, rows * sizeof(float));
-  back(out->values, h->buf.values, (rows + M) * sizeof(float));
-  back(out->rewards, h->buf.rewards, rows * sizeof(float));
-  back(out->dones, h->buf.dones, E * T);
-  back(out->adv, h->buf.adv, rows * sizeof(float));
-  back(out->ret, h->buf.ret, rows * sizeof(float));
-  if (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) back(out->logits, h->buf.logits, rows * kActions * sizeof(float));
-  if (!ok || cudaStreamSynchronize(h->stream) != cudaSuccess) return MAVA_ERR_CUDA;
+  for (int c = 0; c < chunks; ++c) {
+    const int32_t t0 = static_cast<int32_t>(static_cast<int64_t>(T) * c / chunks);
+    const int32_t t1 = static_cast<int32_t>(static_cast<int64_t>(T) * (c + 1) / chunks);
+    const int rc = run_common(h, h->d_params_stage, t1 - t0, nullptr, nullptr, t0);
+    if (rc != MAVA_OK) return rc;
+    if (cudaEventRecord(h->chunk_done[c], h->stream) != cudaSuccess ||
+        cudaStreamWaitEvent(h->copy_stream, h->chunk_done[c], 0) != cudaSuccess)
+      return MAVA_ERR_CUDA;
+    const size_t r0 = M * t0, rn = M * (t1 - t0);
+    back(out->obs, h->buf.obs, r0 * h->D * sizeof(float), rn * h->D * sizeof(float));
+    back(out->actions, h->buf.actions, r0 * sizeof(int32_t), rn * sizeof(int32_t));
+    back(out->logp, h->buf.logp, r0 * sizeof(float), rn * sizeof(float));
+    back(out->values, h->buf.values, r0 * sizeof(float), (rn + (c == chunks - 1 ? M : 0)) * sizeof(float));
+    back(out->rewards, h->buf.rewards, r0 * sizeof(float), rn * sizeof(float));
+    back(out->dones, h->buf.dones, E * t0, E * (t1 - t0));
+    if (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS)
+      back(out->logits, h->buf.logits, r0 * kActions * sizeof(float), rn * kActions * sizeof(float));
+  }
+  if (h->buf.adv && h->buf.ret) {
+    const int rc = mava_gae(h, gamma, lambda);
+    if (rc != MAVA_OK) return rc;
+    if (cudaEventRecord(h->chunk_done[kCollectChunks], h->stream) != cudaSuccess ||
+        cudaStreamWaitEvent(h->copy_stream, h->chunk_done[kCollectChunks], 0) != cudaSuccess)
+      return MAVA_ERR_CUDA;
+    back(out->adv, h->buf.adv, 0, M * T * sizeof(float));
+    back(out->ret, h->buf.ret, 0, M * T * sizeof(float));
+  }
+  if (!ok || cudaStreamSynchronize(h->copy_stream) != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return MAVA_ERR_CUDA;
   return MAVA_OK;
 }
 
@@ -381,6 +418,11 @@ void mava_rollout_destroy(mava_rollout_t *h) {
   cudaFree(h->d_critic);
   cudaFree(h->d_critic_h1);
   cudaFree(h->d_obs_last);
+  if (h->copy_ready) {
+    cudaStreamSynchronize(h->copy_stream);
+    for (int i = 0; i <= kCollectChunks; ++i) cudaEventDestroy(h->chunk_done[i]);
+    cudaStreamDestroy(h->copy_stream);
+  }
   delete h;
 }
 

@@ -7,6 +7,7 @@
 
 namespace mava {
 
+constexpr int kCollectChunks = 4;  // pieces (in time) a host-collected rollout is cut into
 constexpr int kMaxAgents = 8;
 constexpr int kMaxFood = 8;
 constexpr int kActions = MAVA_N_ACTIONS;
@@ -107,6 +108,11 @@ struct mava_rollout {
   uint32_t t_global;
   int32_t last_T;
   int64_t launches;
+  // collect_host: a second stream carries the device-to-host copies of the steps already rolled
+  // out while the rest of the rollout runs (created on first use)
+  cudaStream_t copy_stream;
+  cudaEvent_t chunk_done[mava::kCollectChunks + 1];
+  bool copy_ready;
 };
 
 namespace mava {

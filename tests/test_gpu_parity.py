@@ -317,3 +317,28 @@ def test_forced_actions_on_the_tensor_path():
     assert np.array_equal(ro.rewards.cpu().numpy(), free.rewards) and np.array_equal(ro.dones.cpu().numpy(), free.dones)
     lp = ro.logp.cpu().numpy()
     assert np.all(np.abs(lp - free.logp) <= 2e-2 * (1 + np.abs(free.logp)))
+
+
+@pytest.mark.parametrize("idx,n_envs,T", [(1, 200, 41), (2, 900, 64), (3, 60, 33), (0, 16, 5), (4, 80, 24)])
+def test_collect_host_delivers_the_bytes_of_run_and_gae(idx, n_envs, T):
+    """The host-buffer call (parameters in, whole trajectory out, rolled out in pieces whose copies
+    overlap the kernels) against run + gae on a second handle: every array bit for bit, twice in a row."""
+    import torch
+
+    w = wl.workload(idx)
+    flags = binding.MAVA_FLAG_WRITE_LOGITS
+    params = torch.from_numpy(wl.make_params(w, bias_scale=0.1))
+    a = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=n_envs, flags=flags))
+    b = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=n_envs, flags=flags))
+    names = ("obs", "actions", "logp", "values", "rewards", "dones", "adv", "ret", "logits")
+    out = {n: torch.empty_like(getattr(b, n), device="cpu").pin_memory() for n in names}
+    p_dev = params.cuda()
+    for _ in range(2):
+        a.run(p_dev, T)
+        a.gae(wl.GAMMA, wl.LAMBDA)
+        b.collect_host(params.pin_memory(), T, wl.GAMMA, wl.LAMBDA, out)
+        for n in names:
+            rows = T + 1 if n == "values" else T
+            assert torch.equal(out[n][:rows], getattr(a, n)[:rows].cpu()), n
+    assert np.array_equal(a.get_state(), b.get_state())
+    assert a.status() == 0 and b.status() == 0
