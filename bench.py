@@ -34,7 +34,7 @@ from paper_2107_01460_b200 import workloads as wl  # noqa: E402
 METRIC = "env_agent_steps_per_s"
 UNIT = "env-agent-steps/s"
 # Filled from profiles/rollout_tc_cfg1_full.md; reset an entry to None when its kernel changes.
-NCU_TRAFFIC_BYTES = {("cfg1_8x8_2p2f_h128", "bf16"): 28870912 + 206592}
+NCU_TRAFFIC_BYTES = {("cfg1_8x8_2p2f_h128", "bf16"): 28624384 + 179968}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
