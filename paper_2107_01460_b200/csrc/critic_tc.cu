@@ -11,6 +11,8 @@
 //     rounding, dot product with Cv) while the other's MMAs run.  The value is written to the N
 //     slots of its environment-step.
 // Every mbarrier wait is bounded; a group that gives up records kStatusTimeout and leaves.
+#include <cuda.h>  // CUtensorMap and its enums (types only: nothing of the driver library is linked)
+
 #include "common.cuh"
 #include "layout.h"
 #include "tc_common.cuh"
@@ -82,47 +84,69 @@ __global__ void prep_critic_kernel(const float *__restrict__ params, unsigned ch
 }
 
 // ---- layer 1 -----------------------------------------------------------------------------------
-// Warp-specialised.  Four producer groups of three warps each own one stage of a ring of bf16 A
-// buffers: group g loads item g, g + 4, ... (an item is one 48-column chunk of one 128-row tile)
-// into registers, converts it into its stage and at once starts the loads of its next item, so four
-// items of loads are in flight per SM with a single item per thread.  One thread issues the MMAs as
-// the stages fill and frees them by tcgen05.commit; four epilogue warps drain the two alternating
-// accumulators.  Only mbarriers connect the roles, every wait is bounded.
-constexpr int kL1Stages = 4, kL1GroupThreads = 96, kL1Producers = kL1Stages * kL1GroupThreads;
-constexpr int kL1Threads = kL1Producers + 128 + 32;  // producers, epilogue warps, the issuing warp
+// Warp-specialised, fed by the tensor-map copy engine.  An item is one K step (16 columns) of one
+// 128-row tile.  One thread issues a tiled copy per item: 128 rows x 64 bytes of fp32 observations
+// into a ring of shared-memory stages (64-byte swizzle, so that a thread reading its own row does
+// not collide with its neighbours), never touching L1 or registers on the way.  Two converter
+// groups of 128 threads (thread r = tile row r) alternate items: fp32 -> bf16 into a ring of
+// operand buffers in the MMA's canonical K-major layout.  One thread issues the MMAs as the
+// operand buffers fill and frees them by tcgen05.commit; four epilogue warps drain the two
+// alternating accumulators.  Only mbarriers connect the roles, every wait is bounded.
+// Rows are tiled per array (the T*E rows of `obs`, then the E rows of the last observation), so a
+// tile never straddles the two; rows past an array's end come in as zeros and are never stored.
+constexpr int kL1F32Stages = 5, kL1Bf16Stages = 3;
+constexpr int kL1ConvGroups = 2, kL1ConvThreads = kL1ConvGroups * 128;
+constexpr int kL1Threads = kL1ConvThreads + 128 + 64;  // converters, epilogue warps, copy warp, MMA warp
+constexpr uint32_t kL1F32StageBytes = kTileRows * 16 * 4, kL1Bf16StageBytes = kTileRows * 16 * 2;
 
 template <int N>
 struct CriticL1Smem {
   using S = CriticShape<N>;
-  alignas(128) unsigned char c1[S::C1_BYTES];
-  alignas(128) unsigned char abuf[kL1Stages][S::A_BUF_BYTES];
+  alignas(1024) unsigned char c1[S::C1_BYTES];
+  alignas(1024) unsigned char xf[kL1F32Stages][kL1F32StageBytes];
+  alignas(128) unsigned char xb[kL1Bf16Stages][kL1Bf16StageBytes];
   alignas(8) uint64_t load_bar;
-  alignas(8) uint64_t full[kL1Stages], empty[kL1Stages], acc_full[2], acc_empty[2];
+  alignas(8) uint64_t xf_full[kL1F32Stages], xf_empty[kL1F32Stages], xb_full[kL1Bf16Stages], xb_empty[kL1Bf16Stages];
+  alignas(8) uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
 };
+static_assert(CriticShape<4>::C1_BYTES % 1024 == 0, "the fp32 stages follow C1 on a swizzle-pattern boundary");
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Tiled 2-D copy global -> shared through a tensor map; x (innermost, in elements) must be a multiple of 4 floats.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ float4 lds_f32x4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
 
 template <int N>
 __global__ void __launch_bounds__(kL1Threads, 1)
-critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_last, long long rows_main,
-                 long long rows_total, const unsigned char *__restrict__ image, unsigned char *__restrict__ h1, int n_tiles,
-                 int *status) {
+critic_l1_kernel(const __grid_constant__ CUtensorMap map_main, const __grid_constant__ CUtensorMap map_last, int tiles_main,
+                 const unsigned char *__restrict__ image, unsigned char *__restrict__ h1, int n_tiles, int *status) {
   using S = CriticShape<N>;
-  constexpr int KJ = S::KJ, K1 = S::K1, CHUNK = S::CHUNK, NCHUNK = S::NCHUNK;
-  constexpr int V = CHUNK / 4;        // float4 per row and chunk
-  constexpr int Q = kTileRows / 8;    // float4 per producer thread and item: rows r0, r0 + 8, ...
-  static_assert(V * 8 == kL1GroupThreads, "a group covers eight rows of a chunk per pass");
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  CriticL1Smem<N> &sm = *reinterpret_cast<CriticL1Smem<N> *>(smem_raw);
+  constexpr int KJ = S::KJ, K1 = S::K1, KS = K1 / 16;  // K steps per tile
+  static_assert(KJ / 16 == KS - 1 && KJ % 16 == 4, "the ones columns open the second float4 of the last K step");
+  extern __shared__ unsigned char smem_raw[];
+  // the swizzle pattern of the fp32 stages repeats every 512 bytes of shared address: align by hand
+  CriticL1Smem<N> &sm = *reinterpret_cast<CriticL1Smem<N> *>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
   const int tid = threadIdx.x, warp = tid / 32;
   if (tid == 0) {
     mbar_init(smem_u32(&sm.load_bar), 1);
-    for (int i = 0; i < kL1Stages; ++i) {
-      mbar_init(smem_u32(&sm.full[i]), kL1GroupThreads / 32);  // one arrival per warp of the stage's group
-      mbar_init(smem_u32(&sm.empty[i]), 1);
+    for (int i = 0; i < kL1F32Stages; ++i) {
+      mbar_init(smem_u32(&sm.xf_full[i]), 1);
+      mbar_init(smem_u32(&sm.xf_empty[i]), 4);  // one arrival per warp of the converting group
+    }
+    for (int i = 0; i < kL1Bf16Stages; ++i) {
+      mbar_init(smem_u32(&sm.xb_full[i]), 4);
+      mbar_init(smem_u32(&sm.xb_empty[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&sm.acc_full[i]), 1);
@@ -149,96 +173,48 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
   timed_out = __syncthreads_or(timed_out) != 0;
 
   const uint32_t tmem_base = sm.tmem_base;
-  const uint32_t full0 = smem_u32(&sm.full[0]), empty0 = smem_u32(&sm.empty[0]);
+  const uint32_t xf_full0 = smem_u32(&sm.xf_full[0]), xf_empty0 = smem_u32(&sm.xf_empty[0]);
+  const uint32_t xb_full0 = smem_u32(&sm.xb_full[0]), xb_empty0 = smem_u32(&sm.xb_empty[0]);
   const uint32_t acc_full0 = smem_u32(&sm.acc_full[0]), acc_empty0 = smem_u32(&sm.acc_empty[0]);
-  const uint32_t abuf0 = smem_u32(sm.abuf[0]);
+  const uint32_t xf0 = smem_u32(sm.xf[0]), xb0 = smem_u32(sm.xb[0]);
   // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
   const int my_tiles = (n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
-  const int n_items = my_tiles * NCHUNK;  // (tile, chunk) pairs in order; item n uses ring stage n % kL1Stages
+  const int n_items = my_tiles * KS;  // (tile, K step) pairs in order; item n uses fp32 stage n % 5, operand buffer n % 3
 
-  if (!timed_out && tid < kL1Producers) {
-    // ---- producers --------------------------------------------------------------------------
-    // Thread t of a group takes float4 v = t % 12 of rows r0 + 8 q (r0 = t / 12): consecutive threads
-    // read consecutive 16 bytes of a row, and every address is a per-thread base plus a constant.
-    const int g = tid / kL1GroupThreads, t = tid - g * kL1GroupThreads;
-    const int v = t % V, r0 = t / V;
-    const uint32_t goff = static_cast<uint32_t>(r0 * KJ + 4 * v);  // in floats, within the tile's block of rows
-    const uint32_t sdst = abuf0 + static_cast<uint32_t>(g) * S::A_BUF_BYTES +
-                          static_cast<uint32_t>(((4 * v) >> 3) * S::A_LBO + r0 * 16 + ((4 * v) & 7) * 2);
-    // in the last chunk: the two ones columns that pick up c1, and the zero columns after them
-    const bool ones = (NCHUNK - 1) * CHUNK + 4 * v == KJ, past = (NCHUNK - 1) * CHUNK + 4 * v > KJ;
-    const uint32_t full_bar = full0 + 8u * g, empty_bar = empty0 + 8u * g;
-    int n = g, kt = 0, c = g;  // this group's next item and its (tile, chunk)
-    static_assert(kL1Stages <= S::NCHUNK, "the first items of all groups lie in the first tile");
-    float4 d[Q];
-    auto load_item = [&]() {
-      const long long row0 = (static_cast<long long>(blockIdx.x) + static_cast<long long>(kt) * gridDim.x) * kTileRows;
-      const bool in_main = row0 + kTileRows <= rows_main;
-      const bool in_last = row0 >= rows_main && row0 + kTileRows <= rows_total;
-      const bool last_chunk = c == NCHUNK - 1;
-      if (last_chunk && (ones || past)) {
-#pragma unroll
-        for (int q = 0; q < Q; ++q) d[q] = make_float4(ones ? 1.f : 0.f, ones ? 1.f : 0.f, 0.f, 0.f);
-      } else if (in_main || in_last) {
-        // the tile lies wholly inside one of the two observation arrays: a contiguous block of rows
-        const float *src = (in_main ? obs + row0 * KJ : obs_last + (row0 - rows_main) * KJ) + c * CHUNK + goff;
-#pragma unroll
-        for (int q = 0; q < Q; ++q) d[q] = __ldg(reinterpret_cast<const float4 *>(src + q * 8 * KJ));
-      } else {
-#pragma unroll
-        for (int q = 0; q < Q; ++q) {
-          const long long r_idx = row0 + r0 + 8 * q;
-          d[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (r_idx < rows_total)
-            d[q] = __ldg(reinterpret_cast<const float4 *>(
-                (r_idx < rows_main ? obs + r_idx * KJ : obs_last + (r_idx - rows_main) * KJ) + c * CHUNK + 4 * v));
-        }
-      }
-    };
-    if (n < n_items) load_item();
+  if (timed_out) {
+    // nothing was started
+  } else if (tid < kL1ConvThreads) {
+    // ---- converters: thread r of a group turns row r of an item into bf16 ---------------------
+    const int g = tid / 128, r = tid % 128;
+    const uint32_t src_row = static_cast<uint32_t>(r) * 64u, sw = static_cast<uint32_t>((r >> 1) & 3);  // 64-byte swizzle
+    const uint32_t dst_row = static_cast<uint32_t>((r >> 3) * 256 + (r & 7) * 16);
 #pragma unroll 1
-    for (uint32_t it = 0; n < n_items && !timed_out; ++it) {
-      timed_out |= !mbar_wait(empty_bar, (it & 1) ^ 1);  // the MMAs that read this stage are done
-#pragma unroll
-      for (int q = 0; q < Q; ++q)
-        asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(sdst + q * S::A_SBO), "r"(pack_bf16(d[q].x, d[q].y)),
-                     "r"(pack_bf16(d[q].z, d[q].w))
-                     : "memory");
+    for (int n = g; n < n_items && !timed_out; n += kL1ConvGroups) {
+      const int s = n % kL1F32Stages, b = n % kL1Bf16Stages;
+      const bool last_step = n % KS == KS - 1;
+      timed_out |= !mbar_wait(xf_full0 + 8u * s, (n / kL1F32Stages) & 1);
+      const uint32_t src = xf0 + static_cast<uint32_t>(s) * kL1F32StageBytes + src_row;
+      const float4 f0 = lds_f32x4(src + ((0u ^ sw) << 4));
+      float4 f1 = lds_f32x4(src + ((1u ^ sw) << 4));
+      const float4 f2 = lds_f32x4(src + ((2u ^ sw) << 4));
+      const float4 f3 = lds_f32x4(src + ((3u ^ sw) << 4));
+      if (last_step) f1 = make_float4(1.f, 1.f, 0.f, 0.f);  // the two ones columns that pick up c1 (the copy filled zeros)
+      timed_out |= !mbar_wait(xb_empty0 + 8u * b, ((n / kL1Bf16Stages) & 1) ^ 1);  // the MMA that read this buffer is done
+      timed_out = __any_sync(0xFFFFFFFFu, timed_out);  // the warp leaves together
+      if (timed_out) break;
+      const uint32_t dst = xb0 + static_cast<uint32_t>(b) * kL1Bf16StageBytes + dst_row;
+      sts_v4(dst, pack_bf16(f0.x, f0.y), pack_bf16(f0.z, f0.w), pack_bf16(f1.x, f1.y), pack_bf16(f1.z, f1.w));
+      sts_v4(dst + 128, pack_bf16(f2.x, f2.y), pack_bf16(f2.z, f2.w), pack_bf16(f3.x, f3.y), pack_bf16(f3.z, f3.w));
       fence_async_smem();
       __syncwarp();
-      if ((tid & 31) == 0) mbar_arrive(full_bar);
-      n += kL1Stages;
-      c += kL1Stages;
-      if (c >= NCHUNK) { c -= NCHUNK; ++kt; }
-      if (n < n_items) load_item();
-    }
-  } else if (!timed_out && tid >= kL1Producers + 128) {
-    // ---- the issuing thread -----------------------------------------------------------------
-    if (tid == kL1Producers + 128) {
-      const uint32_t c1_addr = smem_u32(sm.c1);
-      for (int kt = 0; kt < my_tiles && !timed_out; ++kt) {
-        const int a = kt & 1;
-        timed_out |= !mbar_wait(acc_empty0 + 8u * a, ((kt >> 1) & 1) ^ 1);  // the epilogue has drained this accumulator
-        tc_fence_after();
-        const uint32_t acc = tmem_base + static_cast<uint32_t>(a * kCH);
-        for (int c = 0; c < NCHUNK && !timed_out; ++c) {
-          const int n = kt * NCHUNK + c, s2 = n % kL1Stages;
-          timed_out |= !mbar_wait(full0 + 8u * s2, (n / kL1Stages) & 1);
-          tc_fence_after();
-          const uint32_t abuf = abuf0 + static_cast<uint32_t>(s2) * S::A_BUF_BYTES;
-#pragma unroll
-          for (int j = 0; j < CHUNK / 16; ++j)
-            mma_bf16(acc, smem_desc(abuf + j * 2 * S::A_LBO, S::A_LBO, S::A_SBO),
-                     smem_desc(c1_addr + (c * (CHUNK / 16) + j) * 256, 128, K1 * 16), instr_desc(kTileRows, kCH),
-                     (c > 0 || j > 0) ? 1u : 0u);
-          mma_commit(empty0 + 8u * s2);  // frees the stage when these MMAs have read it
-        }
-        mma_commit(acc_full0 + 8u * a);
+      if ((tid & 31) == 0) {
+        mbar_arrive(xb_full0 + 8u * b);
+        mbar_arrive(xf_empty0 + 8u * s);  // after the stores, which needed the loaded values: the stage has been read
       }
     }
-  } else if (!timed_out) {
+  } else if (tid < kL1ConvThreads + 128) {
     // ---- epilogue warps: ReLU, bf16, the row goes out in the operand layout of layer 2 -----------
-    const int row = tid - kL1Producers;  // 0..127: tile row and tensor-memory lane
+    const int row = tid - kL1ConvThreads;  // 0..127: tile row and tensor-memory lane
     const uint32_t lane_off = static_cast<uint32_t>((row / 32) * 32) << 16;
     for (int kt = 0; kt < my_tiles && !timed_out; ++kt) {
       const int a = kt & 1;
@@ -261,6 +237,45 @@ critic_l1_kernel(const float *__restrict__ obs, const float *__restrict__ obs_la
       tc_fence_before();
       __syncwarp();
       if ((tid & 31) == 0) mbar_arrive(acc_empty0 + 8u * a);
+    }
+  } else if (tid == kL1ConvThreads + 128) {
+    // ---- the copy thread ----------------------------------------------------------------------
+    int n = 0;
+    for (int kt = 0; kt < my_tiles && !timed_out; ++kt) {
+      const int tile = static_cast<int>(blockIdx.x) + kt * static_cast<int>(gridDim.x);
+      const bool in_main = tile < tiles_main;
+      const CUtensorMap *map = in_main ? &map_main : &map_last;
+      const int y = (in_main ? tile : tile - tiles_main) * kTileRows;
+      for (int ks = 0; ks < KS && !timed_out; ++ks, ++n) {
+        const int s = n % kL1F32Stages;
+        timed_out |= !mbar_wait(xf_empty0 + 8u * s, ((n / kL1F32Stages) & 1) ^ 1);
+        if (timed_out) break;
+        mbar_expect_tx(xf_full0 + 8u * s, kL1F32StageBytes);
+        tma_load_2d(xf0 + static_cast<uint32_t>(s) * kL1F32StageBytes, map, ks * 16, y, xf_full0 + 8u * s);
+      }
+    }
+    if (timed_out)  // let the copies still in flight land before the block goes away
+      for (int j = n > kL1F32Stages ? n - kL1F32Stages : 0; j < n; ++j)
+        mbar_wait(xf_full0 + 8u * (j % kL1F32Stages), (j / kL1F32Stages) & 1);
+  } else if (tid == kL1ConvThreads + 128 + 32) {
+    // ---- the MMA-issuing thread -----------------------------------------------------------------
+    const uint32_t c1_addr = smem_u32(sm.c1);
+    int n = 0;
+    for (int kt = 0; kt < my_tiles && !timed_out; ++kt) {
+      const int a = kt & 1;
+      timed_out |= !mbar_wait(acc_empty0 + 8u * a, ((kt >> 1) & 1) ^ 1);  // the epilogue has drained this accumulator
+      tc_fence_after();
+      const uint32_t acc = tmem_base + static_cast<uint32_t>(a * kCH);
+      for (int ks = 0; ks < KS && !timed_out; ++ks, ++n) {
+        const int b = n % kL1Bf16Stages;
+        timed_out |= !mbar_wait(xb_full0 + 8u * b, (n / kL1Bf16Stages) & 1);
+        if (timed_out) break;
+        tc_fence_after();
+        mma_bf16(acc, smem_desc(xb0 + static_cast<uint32_t>(b) * kL1Bf16StageBytes, 128, 256),
+                 smem_desc(c1_addr + static_cast<uint32_t>(ks) * 256, 128, K1 * 16), instr_desc(kTileRows, kCH), ks > 0 ? 1u : 0u);
+        mma_commit(xb_empty0 + 8u * b);  // frees the buffer when this MMA has read it
+      }
+      if (!timed_out) mma_commit(acc_full0 + 8u * a);
     }
   }
   if (timed_out) atomicExch(status, kStatusTimeout);
@@ -287,7 +302,7 @@ struct CriticL2Smem {
 template <int N>
 __global__ void __launch_bounds__(2 * kGroupThreads, 1)
 critic_l2_kernel(const unsigned char *__restrict__ h1, const unsigned char *__restrict__ image, float *__restrict__ values,
-                 long long rows_total, int n_tiles, int *status) {
+                 long long rows_main, long long rows_total, int tiles_main, int n_tiles, int *status) {
   using S = CriticShape<N>;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   CriticL2Smem<N> &sm = *reinterpret_cast<CriticL2Smem<N> *>(smem_raw);
@@ -364,8 +379,11 @@ critic_l2_kernel(const unsigned char *__restrict__ h1, const unsigned char *__re
       }
     }
     v += lds_f32(cv_addr + 4u * kCH);
-    const long long r_idx = static_cast<long long>(tile) * kTileRows + row;
-    if (r_idx < rows_total && !timed_out) {
+    // layer 1 tiles the two observation arrays separately: main tiles first, then those of the last observation
+    const bool in_main = tile < tiles_main;
+    const long long r_loc = static_cast<long long>(in_main ? tile : tile - tiles_main) * kTileRows + row;
+    const long long r_idx = in_main ? r_loc : rows_main + r_loc;
+    if (r_loc < (in_main ? rows_main : rows_total - rows_main) && !timed_out) {
       float *out = values + r_idx * N;
 #pragma unroll
       for (int n = 0; n < N; ++n) out[n] = v;
@@ -382,6 +400,28 @@ critic_l2_kernel(const unsigned char *__restrict__ h1, const unsigned char *__re
   }
 }
 
+// Tensor map of a row-major fp32 matrix [rows][width] for boxes of 128 rows x 16 columns (64 bytes, 64-byte swizzle);
+// elements outside the matrix read as zero.  The encoder is a driver entry point fetched through the runtime.
+bool encode_obs_map(CUtensorMap *map, const float *base, long long rows, int width) {
+  using Fn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                          const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                          CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static Fn encode = [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<Fn>(p);
+  }();
+  if (!encode || rows < 1 || reinterpret_cast<uintptr_t>(base) % 16 != 0 || (width * sizeof(float)) % 16 != 0) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(width), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(width) * sizeof(float)};
+  const cuuint32_t box[2] = {16, kTileRows}, elem[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, elem,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 size_t critic_weight_bytes(const mava_config_t &cfg) {
@@ -390,8 +430,9 @@ size_t critic_weight_bytes(const mava_config_t &cfg) {
 
 size_t critic_hidden_bytes(const mava_config_t &cfg) {
   if (find_variant(cfg) != 3) return 16;
-  const long long rows = static_cast<long long>(cfg.max_T + 1) * cfg.n_envs;
-  return static_cast<size_t>((rows + kTileRows - 1) / kTileRows) * CriticShape<4>::H1_TILE_BYTES;
+  const long long rows = static_cast<long long>(cfg.max_T) * cfg.n_envs;
+  const long long tiles = (rows + kTileRows - 1) / kTileRows + (cfg.n_envs + kTileRows - 1) / kTileRows;
+  return static_cast<size_t>(tiles) * CriticShape<4>::H1_TILE_BYTES;
 }
 
 cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T) {
@@ -406,15 +447,19 @@ cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T
   err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
   if (err != cudaSuccess) return err;
   const long long rows_main = static_cast<long long>(T) * h->cfg.n_envs, rows_total = rows_main + h->cfg.n_envs;
-  const int n_tiles = static_cast<int>((rows_total + kTileRows - 1) / kTileRows);
+  const int tiles_main = static_cast<int>((rows_main + kTileRows - 1) / kTileRows);
+  const int n_tiles = tiles_main + (h->cfg.n_envs + kTileRows - 1) / kTileRows;
   {
+    CUtensorMap map_main, map_last;
+    if (!encode_obs_map(&map_main, h->buf.obs, rows_main, S::KJ) || !encode_obs_map(&map_last, h->d_obs_last, h->cfg.n_envs, S::KJ))
+      return cudaErrorInvalidValue;
     auto kern = critic_l1_kernel<4>;
-    const size_t smem = sizeof(CriticL1Smem<4>);
+    const size_t smem = sizeof(CriticL1Smem<4>) + 1024;  // room to align the struct by hand
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     const int ctas = n_tiles < sms ? n_tiles : sms;
-    kern<<<ctas, kL1Threads, smem, h->stream>>>(h->buf.obs, h->d_obs_last, rows_main, rows_total, image,
-                                                static_cast<unsigned char *>(h->d_critic_h1), n_tiles, h->d_status);
+    kern<<<ctas, kL1Threads, smem, h->stream>>>(map_main, map_last, tiles_main, image, static_cast<unsigned char *>(h->d_critic_h1),
+                                                n_tiles, h->d_status);
     h->launches += 1;
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
@@ -426,7 +471,7 @@ cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T
     if (err != cudaSuccess) return err;
     const int ctas = n_tiles < sms ? n_tiles : sms;
     kern<<<ctas, 2 * kGroupThreads, smem, h->stream>>>(static_cast<const unsigned char *>(h->d_critic_h1), image + S::C1_BYTES,
-                                                       h->buf.values, rows_total, n_tiles, h->d_status);
+                                                       h->buf.values, rows_main, rows_total, tiles_main, n_tiles, h->d_status);
     h->launches += 1;
     err = cudaGetLastError();
   }
