@@ -144,7 +144,6 @@ int mava_rollout_create(const mava_config_t *cfg, const mava_buffers_t *buffers,
     ok = cudaMalloc(&h->d_wtc, tc_weight_bytes(*cfg, h->D)) == cudaSuccess;
   if (ok && cfg->precision == MAVA_PRECISION_BF16 && cfg->net_kind == MAVA_NET_CENTRAL_CRITIC)
     ok = cudaMalloc(&h->d_critic, critic_weight_bytes(*cfg)) == cudaSuccess &&
-         cudaMalloc(&h->d_critic_h1, critic_hidden_bytes(*cfg)) == cudaSuccess &&
          cudaMalloc(&h->d_obs_last, sizeof(float) * static_cast<size_t>(cfg->n_envs) * cfg->n_agents * h->D) == cudaSuccess;
   if (ok) ok = cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream) == cudaSuccess;
   if (ok) ok = launch_env_init(h) == cudaSuccess;
@@ -416,7 +415,6 @@ void mava_rollout_destroy(mava_rollout_t *h) {
   cudaFree(h->d_wtc);
   cudaFree(h->d_params_stage);
   cudaFree(h->d_critic);
-  cudaFree(h->d_critic_h1);
   cudaFree(h->d_obs_last);
   if (h->copy_ready) {
     cudaStreamSynchronize(h->copy_stream);

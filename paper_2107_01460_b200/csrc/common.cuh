@@ -102,8 +102,7 @@ struct mava_rollout {
   float *d_wsimt;   // transposed fp32 weights (SIMT path)
   void *d_wtc;      // bf16 weights in tensor-core layout (bf16 path)
   float *d_params_stage;  // device copy of host params (collect_host)
-  void *d_critic;      // centralised critic on the bf16 path: weight images,
-  void *d_critic_h1;   //   hidden activations of all environment-steps (bf16 tiles),
+  void *d_critic;      // centralised critic on the bf16 path: weight images
   float *d_obs_last;   //   and the observations after the last step [E][N][D]
   uint32_t t_global;
   int32_t last_T;
@@ -133,7 +132,6 @@ cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev);
 cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args);
 bool tc_supported(const mava_config_t &cfg);
 size_t critic_weight_bytes(const mava_config_t &cfg);
-size_t critic_hidden_bytes(const mava_config_t &cfg);
 cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T);
 
 }  // namespace mava
