@@ -6,11 +6,10 @@
 //   v  = Cv relu(h1 C2^T + c2) + cv, h1 and h2 rounded to bf16 as the operands of the next layer are.
 // Pairs of SMs share the two weight matrices (tcgen05 cta_group::2), h1 stays in tensor memory.
 // Every mbarrier wait is bounded; a role that gives up records kStatusTimeout and leaves.
-#include <cuda.h>  // CUtensorMap and its enums (types only: nothing of the driver library is linked)
-
 #include "common.cuh"
 #include "layout.h"
 #include "tc_common.cuh"
+#include "tmap.cuh"
 
 namespace mava {
 namespace {
@@ -113,17 +112,6 @@ static_assert((CriticShape<4>::C1_BYTES / 2) % 1024 == 0, "the fp32 stages follo
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// Tiled 2-D copy global -> shared through a tensor map; x (innermost, in elements) must be a multiple of 4 floats.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-               "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
-               : "memory");
-}
-// The same box, but only as far as L2: nothing to wait for, nothing lands in shared memory.
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *map, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y)
-               : "memory");
 }
 __device__ __forceinline__ float4 lds_f32x4(uint32_t addr) {
   float4 v;
@@ -459,28 +447,6 @@ critic_kernel(const __grid_constant__ CUtensorMap map_main, const __grid_constan
   }
 }
 
-// Tensor map of a row-major fp32 matrix [rows][width] for boxes of 128 rows x 16 columns (64 bytes, 64-byte swizzle);
-// elements outside the matrix read as zero.  The encoder is a driver entry point fetched through the runtime.
-bool encode_obs_map(CUtensorMap *map, const float *base, long long rows, int width) {
-  using Fn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                          const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                          CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static Fn encode = [] {
-    void *p = nullptr;
-    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<Fn>(p);
-  }();
-  if (!encode || rows < 1 || reinterpret_cast<uintptr_t>(base) % 16 != 0 || (width * sizeof(float)) % 16 != 0) return false;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(width), static_cast<cuuint64_t>(rows)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(width) * sizeof(float)};
-  const cuuint32_t box[2] = {16, kTileRows}, elem[2] = {1, 1};
-  return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, elem,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 size_t critic_weight_bytes(const mava_config_t &cfg) {
@@ -502,7 +468,9 @@ cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T
   const int tiles_main = static_cast<int>((rows_main + kTileRows - 1) / kTileRows);
   const int n_tiles = tiles_main + (h->cfg.n_envs + kTileRows - 1) / kTileRows;
   CUtensorMap map_main, map_last;
-  if (!encode_obs_map(&map_main, h->buf.obs, rows_main, S::KJ) || !encode_obs_map(&map_last, h->d_obs_last, h->cfg.n_envs, S::KJ))
+  // boxes of 128 rows x 16 columns (64 bytes, 64-byte swizzle): one K step of one tile
+  if (!encode_f32_map(&map_main, h->buf.obs, S::KJ, rows_main, 16, kTileRows, CU_TENSOR_MAP_SWIZZLE_64B) ||
+      !encode_f32_map(&map_last, h->d_obs_last, S::KJ, h->cfg.n_envs, 16, kTileRows, CU_TENSOR_MAP_SWIZZLE_64B))
     return cudaErrorInvalidValue;
   const int pair_tiles = (n_tiles + 1) / 2, pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
   auto go = [&](auto kern, size_t smem) {

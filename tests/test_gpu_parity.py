@@ -223,7 +223,12 @@ def test_capacity_and_argument_errors():
 # ---- GAE on arbitrary data, odd shapes ------------------------------------------------------------
 
 @pytest.mark.parametrize("idx,n_envs,T", [(0, 16, 1), (0, 5, 13), (2, 47, 37), (4, 33, 64), (1, 300, 128), (3, 9, 250),
-                                              (4, 2100, 37), (2, 5464, 100)])  # the last two take the float4 variant
+                                              (4, 2100, 37), (2, 5464, 100),  # these two take the float4 variant
+                                              # the copy-engine variant (E a multiple of 16): environments that straddle
+                                              # a thread's four columns and a ragged last tile, single-step last chunk,
+                                              # two agents and more chunks than a warp has lanes, a long T
+                                              (2, 5488, 101), (4, 2112, 37), (1, 8208, 130), (0, 8192, 200),
+                                              (0, 8192, 255)])  # too long for three stages: back to the plain scan
 def test_gae_on_random_trajectories(idx, n_envs, T):
     import torch
 
