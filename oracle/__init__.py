@@ -4,8 +4,9 @@ TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
 benchmark's CPU-baseline leg; the CUDA library and its Python binding never
 import this package, and this package never imports them.
 
-All arithmetic lives in the C file; this module only builds the shared object
-(``gcc``) and marshals numpy arrays.
+All arithmetic of the rollout, the evaluation block and GAE lives in the C file; this
+module only builds the shared object (``gcc``) and marshals numpy arrays.  The update
+block (multi-agent PPO loss, its gradient, Adam) is ``oracle/ppo.py``, plain numpy in float64.
 """
 from __future__ import annotations
 
