@@ -152,6 +152,38 @@ int mava_rollout_evaluate(mava_rollout_t *h, const float *params_dev, int32_t T,
  * Errors: INVALID_ARG (no run yet, adv/ret NULL), CUDA. */
 int mava_gae(mava_rollout_t *h, float gamma, float lambda);
 
+/* Update block (Section 2: each update function minimises the multi-agent PPO loss on the rolled-out experience;
+ * the report prints no formula, so the clipped-surrogate objective of Schulman et al. 2017 is taken, see below).
+ * Coefficients of the loss and of the optimiser; mava_ppo_defaults fills in 0.2, 0.01, 0.5, 2.5e-4, 0.9, 0.999,
+ * 1e-5, 0.5. */
+typedef struct {
+  float clip_eps, ent_coef, vf_coef;          /* loss */
+  float lr, beta1, beta2, adam_eps;           /* Adam */
+  float max_grad_norm;                        /* global 2-norm the gradient is scaled down to */
+} mava_ppo_hyper_t;
+void mava_ppo_defaults(mava_ppo_hyper_t *hp);
+
+/* Loss and gradient of one minibatch made of ALL rows of the last run (T steps; mava_gae must have run), under
+ * `params_dev` (same layout as for run):
+ *   rho = exp(logp_new(a) - logp);  Ahat = (adv - mean adv) / (std adv + 1e-8)   (population std over the rows)
+ *   L = -mean min(rho Ahat, clip(rho, 1 - eps, 1 + eps) Ahat) - ent_coef * mean H
+ *       + vf_coef * 0.5 * mean max((V - ret)^2, (values + clip(V - values, -eps, eps) - ret)^2)
+ * With the centralised critic a value row is an environment-step (slot 0 of `values` and `ret`, its input the
+ * agents' observations concatenated).  Reads obs, actions, logp, values, adv, ret of the caller's buffers; writes
+ * grad_dev [mava_params_count] (dL/dparams, parameter order) and, if not NULL, terms_dev [4] = L, actor term,
+ * mean entropy, value term (device pointers).  fp32 arithmetic on either precision of the handle; the library
+ * allocates its scratch (one gradient slice per SM) on the first call.  Asynchronous.
+ * Errors: INVALID_ARG (NULL pointers, no run yet, adv/ret NULL), CUDA. */
+int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, float *grad_dev, float *terms_dev);
+
+/* One Adam step in place (Kingma & Ba 2015, bias-corrected; `step` counts from 1) after the gradient has been
+ * scaled to a global 2-norm of at most max_grad_norm:  m = b1 m + (1 - b1) g;  v = b2 v + (1 - b2) g^2;
+ * params -= lr * (m / (1 - b1^step)) / (sqrt(v / (1 - b2^step)) + adam_eps).  All arrays are device pointers of
+ * mava_params_count floats; m and v start at zero and belong to the caller.  Asynchronous.
+ * Errors: INVALID_ARG (NULL pointers, step < 1), CUDA. */
+int mava_adam_step(mava_rollout_t *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
+                   const mava_ppo_hyper_t *hp);
+
 /* Back to episode 0 and global step 0 under a new seed.  Asynchronous. */
 int mava_rollout_reset(mava_rollout_t *h, uint64_t seed);
 

@@ -29,8 +29,13 @@ EXPORTS = [
     "mava_params_count", "mava_rollout_create", "mava_rollout_run", "mava_rollout_run_forced", "mava_gae",
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
-    "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate",
+    "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate", "mava_ppo_defaults", "mava_ppo_grad",
+    "mava_adam_step",
 ]
+
+
+class mava_ppo_hyper_t(C.Structure):
+    _fields_ = [(n, C.c_float) for n in ("clip_eps", "ent_coef", "vf_coef", "lr", "beta1", "beta2", "adam_eps", "max_grad_norm")]
 
 
 class mava_config_t(C.Structure):
@@ -81,6 +86,10 @@ def lib():
         L.mava_strerror.argtypes = [C.c_int]; L.mava_strerror.restype = C.c_char_p
         L.mava_rollout_run_static.argtypes = [cfgp, bufp, vp, C.c_int32, vp]
         L.mava_rollout_run_static.restype = C.c_int
+        hpp = C.POINTER(mava_ppo_hyper_t)
+        L.mava_ppo_defaults.argtypes = [hpp]; L.mava_ppo_defaults.restype = None
+        L.mava_ppo_grad.argtypes = [vp, vp, hpp, vp, vp]; L.mava_ppo_grad.restype = C.c_int
+        L.mava_adam_step.argtypes = [vp, vp, vp, vp, vp, C.c_int32, hpp]; L.mava_adam_step.restype = C.c_int
         _lib = L
     return _lib
 
@@ -99,6 +108,12 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
         view_radius=w["view_radius"], episode_cap=w["episode_cap"], n_envs=w["n_envs"] if n_envs is None else n_envs,
         max_T=w["T"] if max_T is None else max_T, hidden=w["hidden"], net_kind=w["net_kind"], precision=precision,
         flags=flags, first_env=first_env, reserved=0, seed=w["seed"] if seed is None else seed)
+
+
+def ppo_defaults() -> mava_ppo_hyper_t:
+    hp = mava_ppo_hyper_t()
+    lib().mava_ppo_defaults(C.byref(hp))
+    return hp
 
 
 def _check(code: int, where: str):
@@ -178,6 +193,22 @@ class Rollout:
 
     def gae(self, gamma: float, lam: float):
         _check(lib().mava_gae(self.handle, gamma, lam), "mava_gae")
+
+    def ppo_grad(self, params, hp: "mava_ppo_hyper_t | None" = None):
+        """Loss terms [4] (total, actor, entropy, value) and dL/dparams of the last run's rows; device tensors."""
+        import torch
+
+        hp = ppo_defaults() if hp is None else hp
+        grad = torch.empty_like(params)
+        terms = torch.empty(4, dtype=torch.float32, device=params.device)
+        _check(lib().mava_ppo_grad(self.handle, params.data_ptr(), C.byref(hp), grad.data_ptr(), terms.data_ptr()), "mava_ppo_grad")
+        return terms, grad
+
+    def adam_step(self, params, grad, m, v, step: int, hp: "mava_ppo_hyper_t | None" = None):
+        """One clipped Adam step on `params` in place (m, v: the caller's moment tensors, zero at first)."""
+        hp = ppo_defaults() if hp is None else hp
+        _check(lib().mava_adam_step(self.handle, params.data_ptr(), grad.data_ptr(), m.data_ptr(), v.data_ptr(), step,
+                                    C.byref(hp)), "mava_adam_step")
 
     def reset(self, seed: int):
         _check(lib().mava_rollout_reset(self.handle, seed), "mava_rollout_reset")

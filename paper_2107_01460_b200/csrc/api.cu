@@ -181,6 +181,29 @@ int mava_gae(mava_rollout_t *h, float gamma, float lambda) {
   return launch_gae(h, gamma, lambda) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
 }
 
+void mava_ppo_defaults(mava_ppo_hyper_t *hp) {
+  if (!hp) return;
+  hp->clip_eps = 0.2f; hp->ent_coef = 0.01f; hp->vf_coef = 0.5f;
+  hp->lr = 2.5e-4f; hp->beta1 = 0.9f; hp->beta2 = 0.999f; hp->adam_eps = 1e-5f;
+  hp->max_grad_norm = 0.5f;
+}
+
+int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, float *grad_dev, float *terms_dev) {
+  if (!h || !params_dev || !hp || !grad_dev || h->last_T < 1 || !h->buf.adv || !h->buf.ret) return MAVA_ERR_INVALID_ARG;
+  if (!(hp->clip_eps > 0.0f)) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  return launch_ppo_grad(h, params_dev, *hp, grad_dev, terms_dev) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+}
+
+int mava_adam_step(mava_rollout_t *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
+                   const mava_ppo_hyper_t *hp) {
+  if (!h || !params_dev || !grad_dev || !m_dev || !v_dev || !hp || step < 1) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  return launch_adam_step(h, params_dev, grad_dev, m_dev, v_dev, step, *hp) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+}
+
 int mava_rollout_reset(mava_rollout_t *h, uint64_t seed) {
   if (!h) return MAVA_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
@@ -416,6 +439,7 @@ void mava_rollout_destroy(mava_rollout_t *h) {
   cudaFree(h->d_params_stage);
   cudaFree(h->d_critic);
   cudaFree(h->d_obs_last);
+  cudaFree(h->d_upd);
   if (h->copy_ready) {
     cudaStreamSynchronize(h->copy_stream);
     for (int i = 0; i <= kCollectChunks; ++i) cudaEventDestroy(h->chunk_done[i]);

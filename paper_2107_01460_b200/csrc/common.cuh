@@ -104,6 +104,8 @@ struct mava_rollout {
   float *d_params_stage;  // device copy of host params (collect_host)
   void *d_critic;      // centralised critic on the bf16 path: weight images
   float *d_obs_last;   //   and the observations after the last step [E][N][D]
+  void *d_upd;         // scratch of the update block (made on its first call)
+  size_t upd_bytes;
   uint32_t t_global;
   int32_t last_T;
   int64_t launches;
@@ -133,5 +135,10 @@ cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args);
 bool tc_supported(const mava_config_t &cfg);
 size_t critic_weight_bytes(const mava_config_t &cfg);
 cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T);
+
+// Update block (fp32).
+cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava_ppo_hyper_t &hp, float *grad_dev, float *terms_dev);
+cudaError_t launch_adam_step(mava_rollout *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
+                             const mava_ppo_hyper_t &hp);
 
 }  // namespace mava

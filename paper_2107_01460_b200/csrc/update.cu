@@ -1,0 +1,417 @@
+// Update block, first correct path (fp32 on the plain ALUs): the multi-agent PPO loss of one minibatch (all rows
+// of the last rollout), its gradient with respect to every parameter, and the Adam step.
+//   loss:  rho = exp(logp_new(a) - logp_old);  Ahat = (A - mean A) / (std A + 1e-8);
+//          L = -mean min(rho Ahat, clip(rho, 1 +- eps) Ahat) - c_ent mean H
+//              + c_val 0.5 mean max((V - R)^2, (Vold + clip(V - Vold, +-eps) - R)^2)
+// A CTA of H threads (thread j = hidden unit j) walks over tiles of 32 rows: forward through the two hidden
+// layers with the activations of the tile in shared memory, heads and per-row loss derivatives by one warp per
+// row, backward through the layers, and the tile's contribution to every weight gradient added into the CTA's
+// own slice of a partial-gradient array (no atomics; a last kernel adds the slices in a fixed order, so the
+// result does not depend on scheduling).  Sums that decide a mean are kept in double.
+// This is the validation path of the update block, as rollout_simt.cu is the rollout's; a tensor-core path
+// (the weight gradients are GEMMs over millions of rows) is not built yet.
+#include "common.cuh"
+#include "layout.h"
+
+namespace mava {
+namespace {
+
+constexpr int kUpdRows = 32;       // rows per tile
+constexpr int kStatBlocks = 256;   // partial sums of the two reductions
+
+struct UpdNet {
+  const float *W1, *b1, *W2, *b2;  // caller layout [out][in]
+  const float *W1t, *W2t;          // [in][out] copies
+  const float *Wa, *ba, *Wv, *bv;  // heads (nullptr when the net has none of that kind)
+  int Din, H;
+  size_t oW1, ob1, oW2, ob2, oWa, oba, oWv, obv;  // offsets of the gradients in the flat array
+};
+struct UpdRows {
+  const float *x;                  // [n][Din]
+  const int32_t *actions;          // [n]          (actor)
+  const float *logp_old, *adv;     // [n]          (actor)
+  const float *value_old, *ret;    // [n * vstride] (value), element r at r * vstride
+  int vstride;
+  long long n;
+};
+
+__global__ void transpose_kernel(const float *__restrict__ W, float *__restrict__ Wt, int out, int in) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < out * in; i += gridDim.x * blockDim.x) {
+    const int o = i / in, k = i - o * in;
+    Wt[static_cast<size_t>(k) * out + o] = W[i];
+  }
+}
+
+// Block partial sums of x and x^2 (double), then one block turns them into mean and population std.
+__global__ void stat_partial_kernel(const float *__restrict__ x, long long n, double *__restrict__ part) {
+  __shared__ double s0[256], s1[256];
+  double a = 0.0, b = 0.0;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const double v = x[i];
+    a += v; b += v * v;
+  }
+  s0[threadIdx.x] = a; s1[threadIdx.x] = b;
+  __syncthreads();
+  for (int k = blockDim.x / 2; k > 0; k /= 2) {
+    if (threadIdx.x < k) { s0[threadIdx.x] += s0[threadIdx.x + k]; s1[threadIdx.x] += s1[threadIdx.x + k]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { part[2 * blockIdx.x] = s0[0]; part[2 * blockIdx.x + 1] = s1[0]; }
+}
+__global__ void stat_final_kernel(const double *__restrict__ part, int nb, long long n, double *__restrict__ out) {
+  double a = 0.0, b = 0.0;
+  for (int i = 0; i < nb; ++i) { a += part[2 * i]; b += part[2 * i + 1]; }
+  const double mean = a / static_cast<double>(n);
+  const double var = fmax(b / static_cast<double>(n) - mean * mean, 0.0);
+  out[0] = mean; out[1] = sqrt(var); out[2] = sqrt(b);  // [2]: the 2-norm, for the gradient clipping
+}
+
+struct UpdHyper { float clip_eps, ent_coef, vf_coef; };
+
+__global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const double *__restrict__ adv_stats,
+                               float *__restrict__ partial, size_t n_params, double *__restrict__ term_partial) {
+  extern __shared__ __align__(16) float smf[];
+  const int H = net.H, Din = net.Din, j = threadIdx.x, lane = j & 31, warp = j >> 5, n_warps = H >> 5;
+  float *xs = smf, *h1s = xs + kUpdRows * Din, *h2s = h1s + kUpdRows * H, *dz2s = h2s + kUpdRows * H,
+        *dz1s = dz2s + kUpdRows * H, *dl = dz1s + kUpdRows * H;  // dl [32][8]: d logits (6), d value, unused
+  float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
+  const bool has_actor = net.Wa != nullptr, has_value = net.Wv != nullptr;
+  const float mean = has_actor ? static_cast<float>(adv_stats[0]) : 0.0f;
+  const float inv_std = has_actor ? 1.0f / (static_cast<float>(adv_stats[1]) + 1e-8f) : 0.0f;
+  const float inv_n = 1.0f / static_cast<float>(rows.n);
+  float gWa[kActions], gWv = 0.0f, gb1 = 0.0f, gb2 = 0.0f, gbh = 0.0f;
+#pragma unroll
+  for (int k = 0; k < kActions; ++k) gWa[k] = 0.0f;
+  double t_actor = 0.0, t_ent = 0.0, t_value = 0.0;  // lane 0 of every warp
+  const long long n_tiles = (rows.n + kUpdRows - 1) / kUpdRows;
+  for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const long long row0 = tile * kUpdRows;
+    const int n_valid = static_cast<int>(min(static_cast<long long>(kUpdRows), rows.n - row0));
+    for (int i = j; i < kUpdRows * Din; i += H) xs[i] = i < n_valid * Din ? rows.x[row0 * Din + i] : 0.0f;
+    __syncthreads();
+    float acc[kUpdRows];
+    // hidden layer 1 and 2: thread j computes unit j of all rows of the tile
+#pragma unroll
+    for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
+    for (int k = 0; k < Din; ++k) {
+      const float w = net.W1t[static_cast<size_t>(k) * H + j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) acc[r] = fmaf(xs[r * Din + k], w, acc[r]);
+    }
+    {
+      const float b = net.b1[j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) h1s[r * H + j] = fmaxf(acc[r] + b, 0.0f);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
+    for (int k = 0; k < H; ++k) {
+      const float w = net.W2t[static_cast<size_t>(k) * H + j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) acc[r] = fmaf(h1s[r * H + k], w, acc[r]);
+    }
+    {
+      const float b = net.b2[j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) h2s[r * H + j] = fmaxf(acc[r] + b, 0.0f);
+    }
+    __syncthreads();
+    // heads and the per-row derivatives of the loss: one warp per row
+    for (int r = warp; r < kUpdRows; r += n_warps) {
+      float s[kActions + 1];
+#pragma unroll
+      for (int k = 0; k <= kActions; ++k) s[k] = 0.0f;
+      for (int i = lane; i < H; i += 32) {
+        const float hv = h2s[r * H + i];
+        if (has_actor) {
+#pragma unroll
+          for (int k = 0; k < kActions; ++k) s[k] = fmaf(hv, net.Wa[k * H + i], s[k]);
+        }
+        if (has_value) s[kActions] = fmaf(hv, net.Wv[i], s[kActions]);
+      }
+#pragma unroll
+      for (int k = 0; k <= kActions; ++k)
+        for (int o = 16; o > 0; o >>= 1) s[k] += __shfl_xor_sync(0xFFFFFFFFu, s[k], o);
+      if (lane == 0) {
+        float d[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) d[k] = 0.0f;
+        if (r < n_valid) {
+          const long long row = row0 + r;
+          if (has_actor) {
+            float l[kActions], m = -INFINITY, sum = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kActions; ++k) { l[k] = s[k] + net.ba[k]; m = fmaxf(m, l[k]); }
+#pragma unroll
+            for (int k = 0; k < kActions; ++k) sum += expf(l[k] - m);
+            const float lse = m + logf(sum);
+            const int a = rows.actions[row];
+            float ent = 0.0f, p[kActions], lp[kActions], lpa = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kActions; ++k) {
+              lp[k] = l[k] - lse; p[k] = expf(lp[k]); ent -= p[k] * lp[k];
+              if (k == a) lpa = lp[k];
+            }
+            const float rho = expf(lpa - rows.logp_old[row]);
+            const float ahat = (rows.adv[row] - mean) * inv_std;
+            const float clipped = fminf(fmaxf(rho, 1.0f - hp.clip_eps), 1.0f + hp.clip_eps);
+            const float s1 = rho * ahat, s2 = clipped * ahat;
+            const bool inside = rho >= 1.0f - hp.clip_eps && rho <= 1.0f + hp.clip_eps;
+            const float d_logp = (inside || s1 < s2) ? -s1 * inv_n : 0.0f;  // the clipped branch is constant in rho
+#pragma unroll
+            for (int k = 0; k < kActions; ++k)
+              d[k] = d_logp * ((k == a ? 1.0f : 0.0f) - p[k]) + hp.ent_coef * inv_n * p[k] * (lp[k] + ent);
+            t_actor += fminf(s1, s2);
+            t_ent += ent;
+          }
+          if (has_value) {
+            const float v = s[kActions] + net.bv[0], vo = rows.value_old[row * rows.vstride], rt = rows.ret[row * rows.vstride];
+            const float u = v - rt, uc = vo + fminf(fmaxf(v - vo, -hp.clip_eps), hp.clip_eps) - rt;
+            const bool in_range = fabsf(v - vo) <= hp.clip_eps;
+            d[kActions] = (in_range || u * u > uc * uc) ? hp.vf_coef * u * inv_n : 0.0f;
+            t_value += 0.5 * fmaxf(u * u, uc * uc);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) dl[r * 8 + k] = d[k];
+      }
+    }
+    __syncthreads();
+    // back through the heads: d h2, head gradients (kept in registers over all tiles), d z2
+    for (int r = 0; r < kUpdRows; ++r) {
+      const float hv = h2s[r * H + j];
+      float dh = 0.0f;
+      if (has_actor) {
+#pragma unroll
+        for (int k = 0; k < kActions; ++k) {
+          const float dk = dl[r * 8 + k];
+          dh = fmaf(dk, net.Wa[k * H + j], dh);
+          gWa[k] = fmaf(dk, hv, gWa[k]);
+        }
+      }
+      if (has_value) {
+        const float dv = dl[r * 8 + kActions];
+        dh = fmaf(dv, net.Wv[j], dh);
+        gWv = fmaf(dv, hv, gWv);
+      }
+      const float dz = hv > 0.0f ? dh : 0.0f;
+      dz2s[r * H + j] = dz;
+      gb2 += dz;
+      if (j < 8) gbh += dl[r * 8 + j];  // threads 0..6: the heads' biases
+    }
+    __syncthreads();
+    // d h1 = d z2 . W2 (rows of W2 are contiguous in j), d z1
+#pragma unroll
+    for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
+    for (int i = 0; i < H; ++i) {
+      const float w = net.W2[static_cast<size_t>(i) * H + j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) acc[r] = fmaf(dz2s[r * H + i], w, acc[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < kUpdRows; ++r) {
+      const float dz = h1s[r * H + j] > 0.0f ? acc[r] : 0.0f;
+      dz1s[r * H + j] = dz;
+      gb1 += dz;
+    }
+    __syncthreads();
+    // d W2[i][j] += sum_r d z2[r][i] h1[r][j]   (thread j, coalesced over j)
+    {
+      float hcol[kUpdRows];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) hcol[r] = h1s[r * H + j];
+      for (int i = 0; i < H; ++i) {
+        float sacc = 0.0f;
+#pragma unroll
+        for (int r = 0; r < kUpdRows; ++r) sacc = fmaf(dz2s[r * H + i], hcol[r], sacc);
+        part[net.oW2 + static_cast<size_t>(i) * H + j] += sacc;
+      }
+    }
+    // d W1[i][k] += sum_r d z1[r][i] x[r][k]    (thread k, coalesced over k)
+    for (int k = j; k < Din; k += H) {
+      float xcol[kUpdRows];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) xcol[r] = xs[r * Din + k];
+      for (int i = 0; i < H; ++i) {
+        float sacc = 0.0f;
+#pragma unroll
+        for (int r = 0; r < kUpdRows; ++r) sacc = fmaf(dz1s[r * H + i], xcol[r], sacc);
+        part[net.oW1 + static_cast<size_t>(i) * Din + k] += sacc;
+      }
+    }
+    __syncthreads();
+  }
+  // what was kept in registers over all tiles
+  part[net.ob1 + j] += gb1;
+  part[net.ob2 + j] += gb2;
+  if (has_actor) {
+#pragma unroll
+    for (int k = 0; k < kActions; ++k) part[net.oWa + static_cast<size_t>(k) * H + j] += gWa[k];
+    if (j < kActions) part[net.oba + j] += gbh;
+  }
+  if (has_value) {
+    part[net.oWv + j] += gWv;
+    if (j == kActions) part[net.obv] += gbh;
+  }
+  if (lane == 0) {
+    double *tp = term_partial + (static_cast<size_t>(blockIdx.x) * 8 + warp) * 3;
+    tp[0] += t_actor; tp[1] += t_ent; tp[2] += t_value;
+  }
+}
+
+// grad[p] = sum over the CTAs' slices, in slice order; block 0 also turns the term sums into the loss terms.
+__global__ void reduce_partials_kernel(const float *__restrict__ partial, size_t n_params, int n_slices, float *__restrict__ grad,
+                                       const double *__restrict__ term_partial, int n_term, long long n_actor, long long n_value,
+                                       UpdHyper hp, float *__restrict__ terms) {
+  for (size_t p = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < n_params; p += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    float s = 0.0f;
+    for (int c = 0; c < n_slices; ++c) s += partial[static_cast<size_t>(c) * n_params + p];
+    grad[p] = s;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && terms) {
+    double a = 0.0, e = 0.0, v = 0.0;
+    for (int i = 0; i < n_term; ++i) { a += term_partial[3 * i]; e += term_partial[3 * i + 1]; v += term_partial[3 * i + 2]; }
+    const double actor = -a / static_cast<double>(n_actor), ent = e / static_cast<double>(n_actor), val = v / static_cast<double>(n_value);
+    terms[0] = static_cast<float>(actor - hp.ent_coef * ent + hp.vf_coef * val);
+    terms[1] = static_cast<float>(actor);
+    terms[2] = static_cast<float>(ent);
+    terms[3] = static_cast<float>(val);
+  }
+}
+
+__global__ void adam_kernel(float *__restrict__ params, const float *__restrict__ grad, float *__restrict__ m, float *__restrict__ v,
+                            size_t n, const double *__restrict__ stats, float max_norm, float lr, float beta1, float beta2,
+                            float eps, float corr1, float corr2) {
+  const float norm = static_cast<float>(stats[2]);
+  const float scale = max_norm / fmaxf(norm, max_norm);
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const float g = grad[i] * scale;
+    const float mi = beta1 * m[i] + (1.0f - beta1) * g, vi = beta2 * v[i] + (1.0f - beta2) * g * g;
+    m[i] = mi; v[i] = vi;
+    params[i] -= lr * (mi / corr1) / (sqrtf(vi / corr2) + eps);
+  }
+}
+
+// Scratch of the update block, made on first use: [stats: 3 doubles][stat partials][term partials][transposed
+// weights][partial gradients: one slice per CTA].
+struct UpdScratch {
+  double *stats, *stat_part, *term_part;
+  float *wt, *partial;
+  int slices;
+};
+UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
+  unsigned char *p = static_cast<unsigned char *>(h->d_upd);
+  UpdScratch s{};
+  s.stats = reinterpret_cast<double *>(p); p += 64;
+  s.stat_part = reinterpret_cast<double *>(p); p += sizeof(double) * 2 * kStatBlocks;
+  s.term_part = reinterpret_cast<double *>(p); p += sizeof(double) * 3 * 8 * slices;
+  s.wt = reinterpret_cast<float *>(p); p += sizeof(float) * ((n_params + 3) / 4 * 4);
+  s.partial = reinterpret_cast<float *>(p);
+  s.slices = slices;
+  return s;
+}
+
+}  // namespace
+
+cudaError_t ensure_update_scratch(mava_rollout *h, size_t n_params, int slices) {
+  const size_t bytes = 64 + sizeof(double) * 2 * kStatBlocks + sizeof(double) * 3 * 8 * slices + sizeof(float) * ((n_params + 3) / 4 * 4) +
+                       sizeof(float) * n_params * slices;
+  if (h->d_upd && h->upd_bytes >= bytes) return cudaSuccess;
+  cudaFree(h->d_upd);
+  h->d_upd = nullptr;
+  h->upd_bytes = 0;
+  cudaError_t err = cudaMalloc(&h->d_upd, bytes);
+  if (err == cudaSuccess) h->upd_bytes = bytes;
+  return err;
+}
+
+cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava_ppo_hyper_t &hyper, float *grad_dev,
+                            float *terms_dev) {
+  const mava_config_t &cfg = h->cfg;
+  const int T = h->last_T, E = cfg.n_envs, N = cfg.n_agents, D = h->D, H = cfg.hidden;
+  const ParamLayout L = param_layout(cfg, D, 1);
+  const size_t P = L.total;
+  int sms = 0;
+  cudaError_t err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+  if (err != cudaSuccess) return err;
+  const long long R = static_cast<long long>(T) * E * N, S = static_cast<long long>(T) * E;
+  const long long tiles = (R + kUpdRows - 1) / kUpdRows;
+  const int slices = static_cast<int>(tiles < sms ? tiles : sms);
+  err = ensure_update_scratch(h, P, slices);
+  if (err != cudaSuccess) return err;
+  const UpdScratch sc = carve(h, P, slices);
+  cudaStream_t st = h->stream;
+  const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
+  const int joint = N * D;
+  // transposed copies of the hidden layers' weights, in the parameters' own order
+  auto tr = [&](size_t off, int out, int in) {
+    transpose_kernel<<<64, 256, 0, st>>>(params_dev + off, sc.wt + off, out, in);
+    h->launches += 1;
+  };
+  tr(L.W1, H, D); tr(L.W2, H, H);
+  if (central) { tr(L.C1, H, joint); tr(L.C2, H, H); }
+  stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part);
+  stat_final_kernel<<<1, 1, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
+  h->launches += 2;
+  err = cudaMemsetAsync(sc.term_part, 0, sizeof(double) * 3 * 8 * slices, st);
+  if (err == cudaSuccess) err = cudaMemsetAsync(sc.partial, 0, sizeof(float) * P * slices, st);
+  if (err != cudaSuccess) return err;
+  const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
+  auto run_net = [&](const UpdNet &net, const UpdRows &rows) {
+    const size_t smem = sizeof(float) * (static_cast<size_t>(kUpdRows) * net.Din + 4 * static_cast<size_t>(kUpdRows) * net.H + kUpdRows * 8);
+    cudaError_t e = cudaFuncSetAttribute(ppo_net_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    ppo_net_kernel<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part);
+    h->launches += 1;
+    return cudaGetLastError();
+  };
+  UpdNet actor{};
+  actor.W1 = params_dev + L.W1; actor.b1 = params_dev + L.b1; actor.W2 = params_dev + L.W2; actor.b2 = params_dev + L.b2;
+  actor.W1t = sc.wt + L.W1; actor.W2t = sc.wt + L.W2;
+  actor.Wa = params_dev + L.Wa; actor.ba = params_dev + L.ba;
+  actor.Din = D; actor.H = H;
+  actor.oW1 = L.W1; actor.ob1 = L.b1; actor.oW2 = L.W2; actor.ob2 = L.b2; actor.oWa = L.Wa; actor.oba = L.ba;
+  UpdRows rows{};
+  rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
+  if (!central) {
+    actor.Wv = params_dev + L.Wv; actor.bv = params_dev + L.bv; actor.oWv = L.Wv; actor.obv = L.bv;
+    rows.value_old = h->buf.values; rows.ret = h->buf.ret; rows.vstride = 1;
+    err = run_net(actor, rows);
+  } else {
+    err = run_net(actor, rows);
+    if (err != cudaSuccess) return err;
+    UpdNet critic{};
+    critic.W1 = params_dev + L.C1; critic.b1 = params_dev + L.c1; critic.W2 = params_dev + L.C2; critic.b2 = params_dev + L.c2;
+    critic.W1t = sc.wt + L.C1; critic.W2t = sc.wt + L.C2;
+    critic.Wv = params_dev + L.Cv; critic.bv = params_dev + L.cv;
+    critic.Din = joint; critic.H = H;
+    critic.oW1 = L.C1; critic.ob1 = L.c1; critic.oW2 = L.C2; critic.ob2 = L.c2; critic.oWv = L.Cv; critic.obv = L.cv;
+    UpdRows crows{};
+    crows.x = h->buf.obs; crows.value_old = h->buf.values; crows.ret = h->buf.ret; crows.vstride = N; crows.n = S;
+    err = run_net(critic, crows);
+  }
+  if (err != cudaSuccess) return err;
+  reduce_partials_kernel<<<128, 256, 0, st>>>(sc.partial, P, slices, grad_dev, sc.term_part, 8 * slices, R, central ? S : R, hp,
+                                              terms_dev);
+  h->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_adam_step(mava_rollout *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
+                             const mava_ppo_hyper_t &hp) {
+  const size_t P = param_layout(h->cfg, h->D, 1).total;
+  cudaError_t err = ensure_update_scratch(h, P, 1);
+  if (err != cudaSuccess) return err;
+  const UpdScratch sc = carve(h, P, 1);
+  stat_partial_kernel<<<kStatBlocks, 256, 0, h->stream>>>(grad_dev, static_cast<long long>(P), sc.stat_part);
+  stat_final_kernel<<<1, 1, 0, h->stream>>>(sc.stat_part, kStatBlocks, static_cast<long long>(P), sc.stats);
+  const float corr1 = static_cast<float>(1.0 - pow(static_cast<double>(hp.beta1), step));
+  const float corr2 = static_cast<float>(1.0 - pow(static_cast<double>(hp.beta2), step));
+  adam_kernel<<<128, 256, 0, h->stream>>>(params_dev, grad_dev, m_dev, v_dev, P, sc.stats, hp.max_grad_norm, hp.lr, hp.beta1, hp.beta2,
+                                          hp.adam_eps, corr1, corr2);
+  h->launches += 3;
+  return cudaGetLastError();
+}
+
+}  // namespace mava

@@ -1,0 +1,125 @@
+"""Update block on the GPU (mava_ppo_grad, mava_adam_step) against the float64 oracle (oracle/ppo.py).
+
+The GPU rolls out and runs GAE; the oracle gets the GPU's own trajectory arrays as its minibatch, so the
+comparison is of the update block alone.  The kernels compute in fp32, sums that decide a mean in double.
+Tolerance: a gradient entry is a sum over R rows of products of O(1) factors, rounded in fp32 along the way
+(relative error about sqrt(R) * 2^-24 of the largest partial sums), so entries must agree to
+2e-4 * max|grad| and the loss terms to 1e-5 * (1 + |ref|).
+"""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import ppo
+from paper_2107_01460_b200 import binding, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+FP32, BF16 = binding.MAVA_PRECISION_FP32, binding.MAVA_PRECISION_BF16
+
+
+def _rolled_out(idx, n_envs, T, precision, bias_scale=0.1):
+    import torch
+
+    w = wl.workload(idx)
+    cfg = binding.make_config(w, precision=precision, max_T=T, n_envs=n_envs)
+    ro = binding.Rollout(cfg)
+    params = torch.from_numpy(wl.make_params(w, bias_scale=bias_scale)).cuda()
+    ro.run(params, T)
+    ro.gae(wl.GAMMA, wl.LAMBDA)
+    return w, ro, params
+
+
+def _oracle_batch(w, ro, T):
+    g = lambda name, n: getattr(ro, name)[:n].cpu().numpy().astype(np.float64)
+    return ppo.batch_from_rollout(g("obs", T), ro.actions[:T].cpu().numpy(), g("logp", T), g("values", T + 1), g("adv", T),
+                                  g("ret", T), w["net_kind"])
+
+
+@pytest.mark.parametrize("idx,n_envs,T,precision", [(0, 16, 32, FP32), (1, 77, 20, FP32), (2, 50, 33, BF16), (3, 45, 17, BF16),
+                                                    (3, 9, 5, FP32), (4, 21, 11, FP32)])
+def test_loss_and_gradient_match_the_oracle(idx, n_envs, T, precision):
+    import torch
+
+    w, ro, params = _rolled_out(idx, n_envs, T, precision)
+    # parameters a little away from the rollout's own, so that ratios leave 1 and some rows are clipped
+    g = torch.Generator(device="cuda").manual_seed(idx)
+    new = params + 0.6 * torch.randn(params.shape, generator=g, device="cuda") * params.std()
+    hp = binding.ppo_defaults()
+    terms, grad = ro.ppo_grad(new, hp)
+    assert ro.status() == binding.MAVA_OK
+    shapes = ppo.layer_shapes(wl.obs_dim(w), w["hidden"], w["n_agents"], w["net_kind"])
+    batch = _oracle_batch(w, ro, T)
+    p64 = new.cpu().numpy().astype(np.float64)
+    ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch)
+    ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch)
+    t = terms.cpu().numpy()
+    for k, name in enumerate(("total", "actor", "entropy", "value")):
+        assert abs(t[k] - ref[name]) <= 1e-5 * (1 + abs(ref[name])), (name, t[k], ref[name])
+    assert ref["clip_frac"] > 0.0  # the case exercises the clipped branch
+    gg = grad.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(gg - ref_grad)) <= 2e-4 * np.max(np.abs(ref_grad)), np.max(np.abs(gg - ref_grad)) / np.max(np.abs(ref_grad))
+    # every layer's gradient is there (no segment left at zero)
+    off = 0
+    for _, (o, i) in shapes:
+        assert np.abs(gg[off:off + o * i]).max() > 0 and np.abs(gg[off + o * i:off + o * i + o]).max() > 0
+        off += o * i + o
+    # a second call gives the same bytes (fixed summation order)
+    terms2, grad2 = ro.ppo_grad(new, hp)
+    assert torch.equal(grad, grad2) and torch.equal(terms, terms2)
+    ro.close()
+
+
+def test_at_the_rollouts_own_parameters_every_ratio_is_one():
+    w, ro, params = _rolled_out(0, 16, 32, FP32)
+    terms, grad = ro.ppo_grad(params)
+    t = terms.cpu().numpy()
+    assert abs(t[1]) < 1e-5          # -mean(Ahat) = 0
+    assert 0 < t[2] <= np.log(6.0) + 1e-6
+    ro.close()
+
+
+@pytest.mark.parametrize("idx", [0, 3])
+def test_adam_steps_match_the_oracle_and_lower_the_loss(idx):
+    import torch
+
+    w, ro, params = _rolled_out(idx, 24, 16, FP32)
+    hp = binding.ppo_defaults()
+    hp.lr = 1e-3
+    ohp = ppo.Hyper(lr=1e-3)
+    shapes = ppo.layer_shapes(wl.obs_dim(w), w["hidden"], w["n_agents"], w["net_kind"])
+    batch = _oracle_batch(w, ro, 16)
+    p = params.clone()
+    m, v = torch.zeros_like(p), torch.zeros_like(p)
+    p64 = params.cpu().numpy().astype(np.float64)
+    m64, v64 = np.zeros_like(p64), np.zeros_like(p64)
+    first = None
+    for step in range(1, 4):
+        terms, grad = ro.ppo_grad(p, hp)
+        first = terms[0].item() if first is None else first
+        ro.adam_step(p, grad, m, v, step, hp)
+        p64, m64, v64 = ppo.adam_step(p64, ppo.ppo_grad(p64, shapes, w["net_kind"], batch, ohp), m64, v64, step, ohp)
+        # Adam divides by sqrt(v): entries whose gradient is tiny amplify rounding, so compare in units of the step size
+        assert np.max(np.abs(p.cpu().numpy() - p64)) <= 0.02 * ohp.lr * step, np.max(np.abs(p.cpu().numpy() - p64)) / ohp.lr
+    last, _ = ro.ppo_grad(p, hp)
+    assert ro.status() == binding.MAVA_OK
+    assert last[0].item() < first
+    ro.close()
+
+
+def test_argument_errors():
+    import torch
+
+    w = wl.workload(0)
+    ro = binding.Rollout(binding.make_config(w, precision=FP32))
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    with pytest.raises(binding.MavaError):  # no run yet
+        ro.ppo_grad(params)
+    ro.run(params, 4)
+    ro.gae(wl.GAMMA, wl.LAMBDA)
+    hp = binding.ppo_defaults()
+    grad = torch.zeros_like(params)
+    L = binding.lib()
+    assert L.mava_ppo_grad(ro.handle, None, hp, grad.data_ptr(), None) == binding.MAVA_ERR_INVALID_ARG
+    assert L.mava_adam_step(ro.handle, params.data_ptr(), grad.data_ptr(), grad.data_ptr(), grad.data_ptr(), 0, hp) == binding.MAVA_ERR_INVALID_ARG
+    ro.close()
