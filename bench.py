@@ -239,6 +239,26 @@ def time_evaluate(torch, ro, params, w, steps, warmup, flush):
     return sum(times) / len(times)
 
 
+def time_update(torch, ro, params, w, steps, warmup, flush):
+    """Device timing of the update block on the rows of one rollout: PPO loss + gradient, then one Adam step (ms)."""
+    ro.run(params, w["T"])
+    ro.gae(wl.GAMMA, wl.LAMBDA)
+    p = params.clone()
+    m, v = torch.zeros_like(p), torch.zeros_like(p)
+    times = []
+    for i in range(warmup + steps):
+        flush.add_(1.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        _, grad = ro.ppo_grad(p)
+        ro.adam_step(p, grad, m, v, i + 1)
+        e1.record()
+        e1.synchronize()
+        if i >= warmup:
+            times.append(e0.elapsed_time(e1))
+    return sum(times) / len(times)
+
+
 def time_e2e(torch, binding, ro, w, steps, warmup):
     T, E, N, D = w["T"], w["n_envs"], w["n_agents"], wl.obs_dim(w)
     pin = lambda shape, dt: torch.empty(shape, dtype=dt).pin_memory()  # noqa: E731
@@ -298,6 +318,7 @@ def run_gpu(args):
     step_ms = (sum(t_roll) + sum(t_gae)) / args.steps
     e2e_s, h2d, d2h = time_e2e(torch, binding, ro, w, max(3, args.steps // 4), 2)
     eval_ms = time_evaluate(torch, ro, params, w, max(3, args.steps // 4), 3, flush)  # rank-local, reported by rank 0
+    upd_ms = time_update(torch, ro, params, w, max(3, args.steps // 4), 3, flush) if rank == 0 else 0.0
     if dist is not None:
         t = torch.tensor([step_ms, e2e_s], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -330,6 +351,15 @@ def run_gpu(args):
     gae_ach = rows * gae_bytes_per_element(w) / (gae_ms * 1e-3) / 1e9
     gae = {"elements_per_s": rows / (gae_ms * 1e-3), "kernel_ms": gae_ms, "bound": "hbm", "achieved": gae_ach,
            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gae_ach / peaks["hbm_gbs"]}
+
+    # update block (PPO loss + gradient + Adam over the rollout's rows): forward and the two backward products of every
+    # layer = 3 x the forward FLOPs; its only path so far is fp32 on the plain ALUs, whose peak is
+    # SMs x 128 lanes x 2 FLOP x the SM clock
+    alu_peak = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
+    upd_ach = 3 * rows * flops_per_row(w) / (upd_ms * 1e-3) / 1e12
+    update = {"value": rows / (upd_ms * 1e-3), "unit": "rows/s", "ms": upd_ms, "bound": "alu", "achieved": upd_ach,
+              "peak": alu_peak, "unit_roofline": "TFLOP/s", "frac": upd_ach / alu_peak,
+              "path": "fp32 validation path (mava_ppo_grad + mava_adam_step), all rows as one minibatch; no tensor-core path yet"}
 
     # the other workloads, briefly (reported alongside; the headline stays the workload above)
     sweep = []
@@ -373,6 +403,7 @@ def run_gpu(args):
         "gae": gae,
         "evaluate": {"value": rows / (eval_ms * 1e-3), "unit": UNIT, "ms_per_block": eval_ms,
                      "block": f"greedy, T={T} steps, no trajectory stored (mava_rollout_evaluate), one GPU"},
+        "update": update,
         "cpu_baseline": {"value": cpu_rows / cpu_s, "unit": UNIT, "cores": used, "kind": "oracle",
                          "sample": f"first {n_sample} of {E} envs x full T={T} (rollout + GAE), {passes} pass(es), {cpu_s:.1f} s wall"},
         "workloads": sweep,

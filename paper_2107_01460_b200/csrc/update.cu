@@ -17,6 +17,8 @@ namespace mava {
 namespace {
 
 constexpr int kUpdRows = 32;       // rows per tile
+constexpr int kUpdTS = 36;         // row stride of the transposed d z tiles [unit][row]: 16-byte aligned, and consecutive
+                                   // units' 16-byte stores fall into different banks
 constexpr int kStatBlocks = 256;   // partial sums of the two reductions
 
 struct UpdNet {
@@ -72,8 +74,11 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
                                float *__restrict__ partial, size_t n_params, double *__restrict__ term_partial) {
   extern __shared__ __align__(16) float smf[];
   const int H = net.H, Din = net.Din, j = threadIdx.x, lane = j & 31, warp = j >> 5, n_warps = H >> 5;
-  float *xs = smf, *h1s = xs + kUpdRows * Din, *h2s = h1s + kUpdRows * H, *dz2s = h2s + kUpdRows * H,
-        *dz1s = dz2s + kUpdRows * H, *dl = dz1s + kUpdRows * H;  // dl [32][8]: d logits (6), d value, unused
+  const int Dp = (Din + 3) & ~3;  // row stride of the input tile; the pad columns hold zeros
+  // every inner product below reads four operands per shared-memory access (16-byte broadcast loads)
+  float *xs = smf, *h1s = xs + kUpdRows * Dp, *h2s = h1s + kUpdRows * H, *dz2s = h2s + kUpdRows * H,
+        *dz2t = dz2s + kUpdRows * H, *dz1t = dz2t + H * kUpdTS, *dl = dz1t + H * kUpdTS;  // dl [32][8]: d logits (6), d value
+  auto ld4 = [](const float *p) { return *reinterpret_cast<const float4 *>(p); };
   float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
   const bool has_actor = net.Wa != nullptr, has_value = net.Wv != nullptr;
   const float mean = has_actor ? static_cast<float>(adv_stats[0]) : 0.0f;
@@ -87,16 +92,24 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
   for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     const long long row0 = tile * kUpdRows;
     const int n_valid = static_cast<int>(min(static_cast<long long>(kUpdRows), rows.n - row0));
-    for (int i = j; i < kUpdRows * Din; i += H) xs[i] = i < n_valid * Din ? rows.x[row0 * Din + i] : 0.0f;
+    for (int i = j; i < kUpdRows * Dp; i += H) {
+      const int r = i / Dp, k = i - r * Dp;
+      xs[i] = (r < n_valid && k < Din) ? rows.x[(row0 + r) * Din + k] : 0.0f;
+    }
     __syncthreads();
     float acc[kUpdRows];
     // hidden layer 1 and 2: thread j computes unit j of all rows of the tile
 #pragma unroll
     for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
-    for (int k = 0; k < Din; ++k) {
-      const float w = net.W1t[static_cast<size_t>(k) * H + j];
+    for (int k = 0; k < Dp; k += 4) {
+      float w[4];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) acc[r] = fmaf(xs[r * Din + k], w, acc[r]);
+      for (int q = 0; q < 4; ++q) w[q] = k + q < Din ? net.W1t[static_cast<size_t>(k + q) * H + j] : 0.0f;
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) {
+        const float4 x = ld4(xs + r * Dp + k);
+        acc[r] = fmaf(x.x, w[0], fmaf(x.y, w[1], fmaf(x.z, w[2], fmaf(x.w, w[3], acc[r]))));
+      }
     }
     {
       const float b = net.b1[j];
@@ -106,10 +119,15 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
     __syncthreads();
 #pragma unroll
     for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
-    for (int k = 0; k < H; ++k) {
-      const float w = net.W2t[static_cast<size_t>(k) * H + j];
+    for (int k = 0; k < H; k += 4) {
+      float w[4];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) acc[r] = fmaf(h1s[r * H + k], w, acc[r]);
+      for (int q = 0; q < 4; ++q) w[q] = net.W2t[static_cast<size_t>(k + q) * H + j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) {
+        const float4 x = ld4(h1s + r * H + k);
+        acc[r] = fmaf(x.x, w[0], fmaf(x.y, w[1], fmaf(x.z, w[2], fmaf(x.w, w[3], acc[r]))));
+      }
     }
     {
       const float b = net.b2[j];
@@ -179,6 +197,8 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
     }
     __syncthreads();
     // back through the heads: d h2, head gradients (kept in registers over all tiles), d z2
+    float dzr[kUpdRows];
+#pragma unroll
     for (int r = 0; r < kUpdRows; ++r) {
       const float hv = h2s[r * H + j];
       float dh = 0.0f;
@@ -197,24 +217,35 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
       }
       const float dz = hv > 0.0f ? dh : 0.0f;
       dz2s[r * H + j] = dz;
+      dzr[r] = dz;
       gb2 += dz;
       if (j < 8) gbh += dl[r * 8 + j];  // threads 0..6: the heads' biases
     }
+#pragma unroll
+    for (int r = 0; r < kUpdRows; r += 4)
+      *reinterpret_cast<float4 *>(dz2t + j * kUpdTS + r) = make_float4(dzr[r], dzr[r + 1], dzr[r + 2], dzr[r + 3]);
     __syncthreads();
     // d h1 = d z2 . W2 (rows of W2 are contiguous in j), d z1
 #pragma unroll
     for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
-    for (int i = 0; i < H; ++i) {
-      const float w = net.W2[static_cast<size_t>(i) * H + j];
+    for (int i = 0; i < H; i += 4) {
+      float w[4];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) acc[r] = fmaf(dz2s[r * H + i], w, acc[r]);
+      for (int q = 0; q < 4; ++q) w[q] = net.W2[static_cast<size_t>(i + q) * H + j];
+#pragma unroll
+      for (int r = 0; r < kUpdRows; ++r) {
+        const float4 x = ld4(dz2s + r * H + i);
+        acc[r] = fmaf(x.x, w[0], fmaf(x.y, w[1], fmaf(x.z, w[2], fmaf(x.w, w[3], acc[r]))));
+      }
     }
 #pragma unroll
     for (int r = 0; r < kUpdRows; ++r) {
-      const float dz = h1s[r * H + j] > 0.0f ? acc[r] : 0.0f;
-      dz1s[r * H + j] = dz;
-      gb1 += dz;
+      dzr[r] = h1s[r * H + j] > 0.0f ? acc[r] : 0.0f;
+      gb1 += dzr[r];
     }
+#pragma unroll
+    for (int r = 0; r < kUpdRows; r += 4)
+      *reinterpret_cast<float4 *>(dz1t + j * kUpdTS + r) = make_float4(dzr[r], dzr[r + 1], dzr[r + 2], dzr[r + 3]);
     __syncthreads();
     // d W2[i][j] += sum_r d z2[r][i] h1[r][j]   (thread j, coalesced over j)
     {
@@ -224,7 +255,10 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
       for (int i = 0; i < H; ++i) {
         float sacc = 0.0f;
 #pragma unroll
-        for (int r = 0; r < kUpdRows; ++r) sacc = fmaf(dz2s[r * H + i], hcol[r], sacc);
+        for (int r = 0; r < kUpdRows; r += 4) {
+          const float4 d = ld4(dz2t + i * kUpdTS + r);
+          sacc = fmaf(d.x, hcol[r], fmaf(d.y, hcol[r + 1], fmaf(d.z, hcol[r + 2], fmaf(d.w, hcol[r + 3], sacc))));
+        }
         part[net.oW2 + static_cast<size_t>(i) * H + j] += sacc;
       }
     }
@@ -232,11 +266,14 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
     for (int k = j; k < Din; k += H) {
       float xcol[kUpdRows];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) xcol[r] = xs[r * Din + k];
+      for (int r = 0; r < kUpdRows; ++r) xcol[r] = xs[r * Dp + k];
       for (int i = 0; i < H; ++i) {
         float sacc = 0.0f;
 #pragma unroll
-        for (int r = 0; r < kUpdRows; ++r) sacc = fmaf(dz1s[r * H + i], xcol[r], sacc);
+        for (int r = 0; r < kUpdRows; r += 4) {
+          const float4 d = ld4(dz1t + i * kUpdTS + r);
+          sacc = fmaf(d.x, xcol[r], fmaf(d.y, xcol[r + 1], fmaf(d.z, xcol[r + 2], fmaf(d.w, xcol[r + 3], sacc))));
+        }
         part[net.oW1 + static_cast<size_t>(i) * Din + k] += sacc;
       }
     }
@@ -295,6 +332,11 @@ __global__ void adam_kernel(float *__restrict__ params, const float *__restrict_
 
 // Scratch of the update block, made on first use: [stats: 3 doubles][stat partials][term partials][transposed
 // weights][partial gradients: one slice per CTA].
+size_t upd_smem_bytes(int Din, int H) {
+  return sizeof(float) * (static_cast<size_t>(kUpdRows) * ((Din + 3) & ~3) + 3 * static_cast<size_t>(kUpdRows) * H +
+                          2 * static_cast<size_t>(H) * kUpdTS + kUpdRows * 8);
+}
+
 struct UpdScratch {
   double *stats, *stat_part, *term_part;
   float *wt, *partial;
@@ -337,13 +379,21 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   if (err != cudaSuccess) return err;
   const long long R = static_cast<long long>(T) * E * N, S = static_cast<long long>(T) * E;
   const long long tiles = (R + kUpdRows - 1) / kUpdRows;
-  const int slices = static_cast<int>(tiles < sms ? tiles : sms);
+  // as many CTAs (= gradient slices) as are resident at once with the larger of the two nets' shared-memory needs
+  const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
+  const int joint = N * D;
+  const size_t smem_max = upd_smem_bytes(central ? joint : D, H);
+  err = cudaFuncSetAttribute(ppo_net_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_max));
+  if (err != cudaSuccess) return err;
+  int per_sm = 1;
+  err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ppo_net_kernel, H, smem_max);
+  if (err != cudaSuccess) return err;
+  if (per_sm < 1) per_sm = 1;
+  const int slices = static_cast<int>(tiles < static_cast<long long>(sms) * per_sm ? tiles : static_cast<long long>(sms) * per_sm);
   err = ensure_update_scratch(h, P, slices);
   if (err != cudaSuccess) return err;
   const UpdScratch sc = carve(h, P, slices);
   cudaStream_t st = h->stream;
-  const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
-  const int joint = N * D;
   // transposed copies of the hidden layers' weights, in the parameters' own order
   auto tr = [&](size_t off, int out, int in) {
     transpose_kernel<<<64, 256, 0, st>>>(params_dev + off, sc.wt + off, out, in);
@@ -359,7 +409,7 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   if (err != cudaSuccess) return err;
   const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
   auto run_net = [&](const UpdNet &net, const UpdRows &rows) {
-    const size_t smem = sizeof(float) * (static_cast<size_t>(kUpdRows) * net.Din + 4 * static_cast<size_t>(kUpdRows) * net.H + kUpdRows * 8);
+    const size_t smem = upd_smem_bytes(net.Din, net.H);
     cudaError_t e = cudaFuncSetAttribute(ppo_net_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     ppo_net_kernel<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part);
