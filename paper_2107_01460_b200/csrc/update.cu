@@ -6,8 +6,9 @@
 // A CTA of H threads (thread j = hidden unit j) walks over tiles of 32 rows: forward through the two hidden
 // layers with the activations of the tile in shared memory, heads and per-row loss derivatives by one warp per
 // row, backward through the layers, and the tile's contribution to every weight gradient added into the CTA's
-// own slice of a partial-gradient array (no atomics; a last kernel adds the slices in a fixed order, so the
-// result does not depend on scheduling).  Sums that decide a mean are kept in double.
+// own slice of a partial-gradient array (reductions without a return value: an address is only ever added to by
+// one thread, in program order; a last kernel adds the slices in a fixed order, so the result does not depend
+// on scheduling).  Sums that decide a mean are kept in double.
 // This is the validation path of the update block, as rollout_simt.cu is the rollout's; a tensor-core path
 // (the weight gradients are GEMMs over millions of rows) is not built yet.
 #include "common.cuh"
@@ -259,7 +260,7 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
           const float4 d = ld4(dz2t + i * kUpdTS + r);
           sacc = fmaf(d.x, hcol[r], fmaf(d.y, hcol[r + 1], fmaf(d.z, hcol[r + 2], fmaf(d.w, hcol[r + 3], sacc))));
         }
-        part[net.oW2 + static_cast<size_t>(i) * H + j] += sacc;
+        atomicAdd(part + net.oW2 + static_cast<size_t>(i) * H + j, sacc);  // result unused: a fire-and-forget reduction, no load to wait for
       }
     }
     // d W1[i][k] += sum_r d z1[r][i] x[r][k]    (thread k, coalesced over k)
@@ -274,7 +275,7 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
           const float4 d = ld4(dz1t + i * kUpdTS + r);
           sacc = fmaf(d.x, xcol[r], fmaf(d.y, xcol[r + 1], fmaf(d.z, xcol[r + 2], fmaf(d.w, xcol[r + 3], sacc))));
         }
-        part[net.oW1 + static_cast<size_t>(i) * Din + k] += sacc;
+        atomicAdd(part + net.oW1 + static_cast<size_t>(i) * Din + k, sacc);
       }
     }
     __syncthreads();
