@@ -37,7 +37,8 @@ def _oracle_batch(w, ro, T):
 
 
 @pytest.mark.parametrize("idx,n_envs,T,precision", [(0, 16, 32, FP32), (1, 77, 20, FP32), (2, 50, 33, BF16), (3, 45, 17, BF16),
-                                                    (3, 9, 5, FP32), (4, 21, 11, FP32)])
+                                                    (3, 9, 5, FP32), (4, 21, 11, FP32),
+                                                    (1, 1024, 128, BF16)])  # the size and precision the benchmark times
 def test_loss_and_gradient_match_the_oracle(idx, n_envs, T, precision):
     import torch
 
