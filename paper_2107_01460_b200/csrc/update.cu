@@ -18,8 +18,8 @@ namespace mava {
 namespace {
 
 constexpr int kUpdRows = 32;       // rows per tile
-constexpr int kUpdTS = 36;         // row stride of the transposed d z tiles [unit][row]: 16-byte aligned, and consecutive
-                                   // units' 16-byte stores fall into different banks
+constexpr int kUpdTS = kUpdRows;   // row stride of the transposed d z tiles [unit][row] (read by 16-byte broadcasts; the few
+                                   // stores that fill them collide on banks, which costs less than the room padding takes)
 constexpr int kStatBlocks = 256;   // partial sums of the two reductions
 
 struct UpdNet {
@@ -77,8 +77,9 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
   const int H = net.H, Din = net.Din, j = threadIdx.x, lane = j & 31, warp = j >> 5, n_warps = H >> 5;
   const int Dp = (Din + 3) & ~3;  // row stride of the input tile; the pad columns hold zeros
   // every inner product below reads four operands per shared-memory access (16-byte broadcast loads)
-  float *xs = smf, *h1s = xs + kUpdRows * Dp, *h2s = h1s + kUpdRows * H, *dz2s = h2s + kUpdRows * H,
-        *dz2t = dz2s + kUpdRows * H, *dz1t = dz2t + H * kUpdTS, *dl = dz1t + H * kUpdTS;  // dl [32][8]: d logits (6), d value
+  // d z1 takes the place of h2, which is dead by then: three CTAs fit an SM at H = 128
+  float *xs = smf, *h1s = xs + kUpdRows * Dp, *h2s = h1s + kUpdRows * H, *dz2t = h2s + kUpdRows * H, *dz1t = h2s,
+        *dl = dz2t + H * kUpdTS;  // dl [32][8]: d logits (6), d value
   auto ld4 = [](const float *p) { return *reinterpret_cast<const float4 *>(p); };
   float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
   const bool has_actor = net.Wa != nullptr, has_value = net.Wv != nullptr;
@@ -217,7 +218,6 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
         gWv = fmaf(dv, hv, gWv);
       }
       const float dz = hv > 0.0f ? dh : 0.0f;
-      dz2s[r * H + j] = dz;
       dzr[r] = dz;
       gb2 += dz;
       if (j < 8) gbh += dl[r * 8 + j];  // threads 0..6: the heads' biases
@@ -234,9 +234,15 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
 #pragma unroll
       for (int q = 0; q < 4; ++q) w[q] = net.W2[static_cast<size_t>(i + q) * H + j];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) {
-        const float4 x = ld4(dz2s + r * H + i);
-        acc[r] = fmaf(x.x, w[0], fmaf(x.y, w[1], fmaf(x.z, w[2], fmaf(x.w, w[3], acc[r]))));
+      for (int q = 0; q < 4; ++q) {
+#pragma unroll
+        for (int r = 0; r < kUpdRows; r += 4) {
+          const float4 d = ld4(dz2t + (i + q) * kUpdTS + r);
+          acc[r] = fmaf(d.x, w[q], acc[r]);
+          acc[r + 1] = fmaf(d.y, w[q], acc[r + 1]);
+          acc[r + 2] = fmaf(d.z, w[q], acc[r + 2]);
+          acc[r + 3] = fmaf(d.w, w[q], acc[r + 3]);
+        }
       }
     }
 #pragma unroll
@@ -334,8 +340,8 @@ __global__ void adam_kernel(float *__restrict__ params, const float *__restrict_
 // Scratch of the update block, made on first use: [stats: 3 doubles][stat partials][term partials][transposed
 // weights][partial gradients: one slice per CTA].
 size_t upd_smem_bytes(int Din, int H) {
-  return sizeof(float) * (static_cast<size_t>(kUpdRows) * ((Din + 3) & ~3) + 3 * static_cast<size_t>(kUpdRows) * H +
-                          2 * static_cast<size_t>(H) * kUpdTS + kUpdRows * 8);
+  return sizeof(float) * (static_cast<size_t>(kUpdRows) * ((Din + 3) & ~3) + 2 * static_cast<size_t>(kUpdRows) * H +
+                          static_cast<size_t>(H) * kUpdTS + kUpdRows * 8);
 }
 
 struct UpdScratch {
