@@ -1,0 +1,76 @@
+"""The whole on-device loop the report describes (Section 2, Figure 2): roll out, estimate advantages, update,
+repeat, with evaluation blocks in between -- every step a call into the C ABI, nothing computed in Python.
+
+    python -m paper_2107_01460_b200.train [--workload 1] [--envs 1024] [--steps 64] [--iters 200] [--epochs 4]
+                                          [--lr 1e-3] [--eval-every 25]
+
+Each iteration: mava_rollout_run (T steps of every environment, continuing where the last one stopped), mava_gae,
+then `epochs` passes of mava_ppo_grad + mava_adam_step over all rows of that rollout as one minibatch.  Every
+`eval-every` iterations a second handle with the same shape runs a greedy evaluation block from fresh episodes and
+the mean return of the episodes that ended is printed (1.0 = every food item collected).
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import binding, build, workloads as wl
+
+
+def mean_return(ev: "binding.Rollout", params, T: int, seed: int) -> float:
+    """Mean return of the episodes that end inside a greedy block of T steps from fresh episodes."""
+    ev.reset(seed)
+    count, ret, _, _ = ev.evaluate(params, T, greedy=True)
+    n = int(count.sum().item())
+    return float(ret.sum().item()) / n if n else float("nan")
+
+
+def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, epochs: int = 4, lr: float = 1e-3,
+          eval_every: int = 25, precision: int | None = None, log=print):
+    """Runs the loop and returns the list of (iteration, mean greedy return) it evaluated."""
+    build.build()
+    w = wl.workload(workload)
+    cfg = binding.make_config(w, precision=precision, n_envs=n_envs, max_T=T)
+    ro = binding.Rollout(cfg)
+    cap = w["episode_cap"]
+    ev = binding.Rollout(binding.make_config(w, precision=precision, n_envs=n_envs, max_T=2 * cap), with_gae=False)
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    m, v = torch.zeros_like(params), torch.zeros_like(params)
+    hp = binding.ppo_defaults()
+    hp.lr = lr
+    history, step = [], 0
+    for it in range(iters + 1):
+        if it % eval_every == 0 or it == iters:
+            r = mean_return(ev, params, 2 * cap, seed=10_000 + it)
+            history.append((it, r))
+            log(f"iteration {it:4d}: mean greedy return {r:.4f}")
+        if it == iters:
+            break
+        ro.run(params, T)
+        ro.gae(wl.GAMMA, wl.LAMBDA)
+        for _ in range(epochs):
+            step += 1
+            terms, grad = ro.ppo_grad(params, hp)
+            ro.adam_step(params, grad, m, v, step, hp)
+    assert ro.status() == binding.MAVA_OK and ev.status() == binding.MAVA_OK
+    ro.close()
+    ev.close()
+    return history
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", type=int, default=1)
+    ap.add_argument("--envs", type=int, default=1024)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--iters", type=int, default=200)
+    ap.add_argument("--epochs", type=int, default=4)
+    ap.add_argument("--lr", type=float, default=1e-3)
+    ap.add_argument("--eval-every", type=int, default=25)
+    args = ap.parse_args()
+    train(args.workload, args.envs, args.steps, args.iters, args.epochs, args.lr, args.eval_every)
+
+
+if __name__ == "__main__":
+    main()
