@@ -8,6 +8,11 @@ Each iteration: mava_rollout_run (T steps of every environment, continuing where
 then `epochs` passes of mava_ppo_grad + mava_adam_step over all rows of that rollout as one minibatch.  Every
 `eval-every` iterations a second handle with the same shape runs a greedy evaluation block from fresh episodes and
 the mean return of the episodes that ended is printed (1.0 = every food item collected).
+
+Under torchrun (one process per GPU) every rank rolls out its own shard of the environments (`first_env` = rank x
+envs, so the shards are the environments of one large batch) and the ranks exchange one thing per update: the
+gradient, averaged with an NCCL all-reduce (the report's `pmean`, Section 2).  Parameters and optimiser state start
+equal and see the same averaged gradient, so they stay equal without being sent.
 """
 from __future__ import annotations
 
@@ -26,15 +31,26 @@ def mean_return(ev: "binding.Rollout", params, T: int, seed: int) -> float:
     return float(ret.sum().item()) / n if n else float("nan")
 
 
+def average_gradients(grad):
+    """In place: the mean of `grad` over the ranks of the default process group (a no-op without one)."""
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(grad, op=dist.ReduceOp.SUM)
+        grad /= dist.get_world_size()
+    return grad
+
+
 def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, epochs: int = 4, lr: float = 1e-3,
-          eval_every: int = 25, precision: int | None = None, log=print):
+          eval_every: int = 25, precision: int | None = None, log=print, rank: int = 0):
     """Runs the loop and returns the list of (iteration, mean greedy return) it evaluated."""
     build.build()
     w = wl.workload(workload)
-    cfg = binding.make_config(w, precision=precision, n_envs=n_envs, max_T=T)
-    ro = binding.Rollout(cfg)
+    cfg = binding.make_config(w, precision=precision, n_envs=n_envs, max_T=T, first_env=wl.shard_first_env(n_envs, rank))
+    device = f"cuda:{torch.cuda.current_device()}"
+    ro = binding.Rollout(cfg, device=device)
     cap = w["episode_cap"]
-    ev = binding.Rollout(binding.make_config(w, precision=precision, n_envs=n_envs, max_T=2 * cap), with_gae=False)
+    ev = binding.Rollout(binding.make_config(w, precision=precision, n_envs=n_envs, max_T=2 * cap), device=device, with_gae=False)
     params = torch.from_numpy(wl.make_params(w)).cuda()
     m, v = torch.zeros_like(params), torch.zeros_like(params)
     hp = binding.ppo_defaults()
@@ -52,6 +68,7 @@ def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, 
         for _ in range(epochs):
             step += 1
             terms, grad = ro.ppo_grad(params, hp)
+            average_gradients(grad)
             ro.adam_step(params, grad, m, v, step, hp)
     assert ro.status() == binding.MAVA_OK and ev.status() == binding.MAVA_OK
     ro.close()
@@ -69,7 +86,22 @@ def main():
     ap.add_argument("--lr", type=float, default=1e-3)
     ap.add_argument("--eval-every", type=int, default=25)
     args = ap.parse_args()
-    train(args.workload, args.envs, args.steps, args.iters, args.epochs, args.lr, args.eval_every)
+    import os
+
+    rank = 0
+    if "RANK" in os.environ and int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        dist.init_process_group("nccl")
+        rank = dist.get_rank()
+    train(args.workload, args.envs, args.steps, args.iters, args.epochs, args.lr, args.eval_every,
+          log=print if rank == 0 else (lambda *_: None), rank=rank)
+    if rank or "RANK" in os.environ:
+        import torch.distributed as dist
+
+        if dist.is_initialized():
+            dist.destroy_process_group()
 
 
 if __name__ == "__main__":
