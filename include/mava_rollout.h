@@ -176,6 +176,14 @@ void mava_ppo_defaults(mava_ppo_hyper_t *hp);
  * Errors: INVALID_ARG (NULL pointers, no run yet, adv/ret NULL), CUDA. */
 int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, float *grad_dev, float *terms_dev);
 
+/* The same over a minibatch of environments: the rows of the n_ids environments env_ids_dev[0..n_ids) (device
+ * pointer, local indices 0..n_envs-1, any order; a repeated index counts twice) at every step of the last run; the
+ * advantages are normalised over that minibatch.  A permutation of all environments cut into pieces gives the
+ * shuffled minibatches of a PPO epoch.  An index outside 0..n_envs-1 makes the kernel skip that environment's rows
+ * and mava_rollout_status answer MAVA_ERR_INVALID_ARG.  Errors: as mava_ppo_grad, and INVALID_ARG for n_ids < 1. */
+int mava_ppo_grad_envs(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, const int32_t *env_ids_dev,
+                       int32_t n_ids, float *grad_dev, float *terms_dev);
+
 /* One Adam step in place (Kingma & Ba 2015, bias-corrected; `step` counts from 1) after the gradient has been
  * scaled to a global 2-norm of at most max_grad_norm:  m = b1 m + (1 - b1) g;  v = b2 v + (1 - b2) g^2;
  * params -= lr * (m / (1 - b1^step)) / (sqrt(v / (1 - b2^step)) + adam_eps).  All arrays are device pointers of
@@ -188,7 +196,8 @@ int mava_adam_step(mava_rollout_t *h, float *params_dev, const float *grad_dev, 
 int mava_rollout_reset(mava_rollout_t *h, uint64_t seed);
 
 /* Waits for the stream, then returns MAVA_OK, MAVA_ERR_DEVICE_TIMEOUT if a kernel's bounded wait
- * gave up since the last call (the status word is cleared), or MAVA_ERR_CUDA. */
+ * gave up since the last call, MAVA_ERR_INVALID_ARG if a kernel met an environment index out of range
+ * (the status word is cleared either way), or MAVA_ERR_CUDA. */
 int mava_rollout_status(mava_rollout_t *h);
 
 /* Environment states as int32 records of mava_state_record_len(cfg) words per environment:

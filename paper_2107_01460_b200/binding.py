@@ -30,7 +30,7 @@ EXPORTS = [
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
     "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate", "mava_ppo_defaults", "mava_ppo_grad",
-    "mava_adam_step",
+    "mava_adam_step", "mava_ppo_grad_envs",
 ]
 
 
@@ -89,6 +89,7 @@ def lib():
         hpp = C.POINTER(mava_ppo_hyper_t)
         L.mava_ppo_defaults.argtypes = [hpp]; L.mava_ppo_defaults.restype = None
         L.mava_ppo_grad.argtypes = [vp, vp, hpp, vp, vp]; L.mava_ppo_grad.restype = C.c_int
+        L.mava_ppo_grad_envs.argtypes = [vp, vp, hpp, vp, C.c_int32, vp, vp]; L.mava_ppo_grad_envs.restype = C.c_int
         L.mava_adam_step.argtypes = [vp, vp, vp, vp, vp, C.c_int32, hpp]; L.mava_adam_step.restype = C.c_int
         _lib = L
     return _lib
@@ -194,13 +195,19 @@ class Rollout:
     def gae(self, gamma: float, lam: float):
         _check(lib().mava_gae(self.handle, gamma, lam), "mava_gae")
 
-    def ppo_grad(self, params, hp: "mava_ppo_hyper_t | None" = None):
-        """Loss terms [4] (total, actor, entropy, value) and dL/dparams of the last run's rows; device tensors."""
+    def ppo_grad(self, params, hp: "mava_ppo_hyper_t | None" = None, env_ids=None):
+        """Loss terms [4] (total, actor, entropy, value) and dL/dparams of the last run's rows (of the environments
+        `env_ids`, an int32 device tensor, when given); device tensors."""
         import torch
 
         hp = ppo_defaults() if hp is None else hp
         grad = torch.empty_like(params)
         terms = torch.empty(4, dtype=torch.float32, device=params.device)
+        if env_ids is not None:
+            assert env_ids.is_cuda and env_ids.dtype == torch.int32 and env_ids.is_contiguous()
+            _check(lib().mava_ppo_grad_envs(self.handle, params.data_ptr(), C.byref(hp), env_ids.data_ptr(), env_ids.numel(),
+                                            grad.data_ptr(), terms.data_ptr()), "mava_ppo_grad_envs")
+            return terms, grad
         _check(lib().mava_ppo_grad(self.handle, params.data_ptr(), C.byref(hp), grad.data_ptr(), terms.data_ptr()), "mava_ppo_grad")
         return terms, grad
 

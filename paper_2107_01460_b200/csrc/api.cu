@@ -193,7 +193,17 @@ int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyp
   if (!(hp->clip_eps > 0.0f)) return MAVA_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
-  return launch_ppo_grad(h, params_dev, *hp, grad_dev, terms_dev) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+  return launch_ppo_grad(h, params_dev, *hp, grad_dev, terms_dev, nullptr, 0) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+}
+
+int mava_ppo_grad_envs(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, const int32_t *env_ids_dev,
+                       int32_t n_ids, float *grad_dev, float *terms_dev) {
+  if (!h || !params_dev || !hp || !grad_dev || !env_ids_dev || n_ids < 1 || h->last_T < 1 || !h->buf.adv || !h->buf.ret)
+    return MAVA_ERR_INVALID_ARG;
+  if (!(hp->clip_eps > 0.0f)) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  return launch_ppo_grad(h, params_dev, *hp, grad_dev, terms_dev, env_ids_dev, n_ids) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
 }
 
 int mava_adam_step(mava_rollout_t *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
@@ -224,7 +234,7 @@ int mava_rollout_status(mava_rollout_t *h) {
     return MAVA_ERR_CUDA;
   if (status != 0) {
     cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream);
-    return MAVA_ERR_DEVICE_TIMEOUT;
+    return status == kStatusBadIndex ? MAVA_ERR_INVALID_ARG : MAVA_ERR_DEVICE_TIMEOUT;
   }
   return MAVA_OK;
 }

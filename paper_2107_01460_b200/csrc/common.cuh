@@ -21,6 +21,7 @@ constexpr uint32_t kDomainAction = 0x41435431u;    // key tweak of the action-un
 
 // Device status word values (0 = fine).
 constexpr int kStatusTimeout = 1;
+constexpr int kStatusBadIndex = 2;  // an environment index of a minibatch was out of range (its rows were skipped)
 
 // Compact per-environment state.  Coordinates and levels fit a byte (G <= 64, levels <= 31).
 struct __align__(4) EnvRec {
@@ -137,7 +138,8 @@ size_t critic_weight_bytes(const mava_config_t &cfg);
 cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T);
 
 // Update block (fp32).
-cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava_ppo_hyper_t &hp, float *grad_dev, float *terms_dev);
+cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava_ppo_hyper_t &hp, float *grad_dev, float *terms_dev,
+                            const int32_t *env_ids_dev, int32_t n_ids);
 cudaError_t launch_adam_step(mava_rollout *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
                              const mava_ppo_hyper_t &hp);
 

@@ -36,7 +36,22 @@ struct UpdRows {
   const float *value_old, *ret;    // [n * vstride] (value), element r at r * vstride
   int vstride;
   long long n;
+  // a minibatch of environments: row q of the batch is (step, env_ids[i], slot) with q = (step * n_ids + i) * per_env + slot;
+  // nullptr = every environment in order (row q is row q of the arrays)
+  const int32_t *env_ids;
+  int n_ids, E, per_env;
 };
+
+// Row of the trajectory arrays behind row q of the batch; -1 when the environment index is out of range.
+__device__ __forceinline__ long long real_row(const UpdRows &rows, long long q) {
+  if (!rows.env_ids) return q;
+  const long long per_step = static_cast<long long>(rows.n_ids) * rows.per_env;
+  const long long t = q / per_step, rem = q - t * per_step;
+  const int i = static_cast<int>(rem / rows.per_env), slot = static_cast<int>(rem - static_cast<long long>(i) * rows.per_env);
+  const int e = rows.env_ids[i];
+  if (e < 0 || e >= rows.E) return -1;
+  return (t * rows.E + e) * rows.per_env + slot;
+}
 
 __global__ void transpose_kernel(const float *__restrict__ W, float *__restrict__ Wt, int out, int in) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < out * in; i += gridDim.x * blockDim.x) {
@@ -46,11 +61,12 @@ __global__ void transpose_kernel(const float *__restrict__ W, float *__restrict_
 }
 
 // Block partial sums of x and x^2 (double), then one block turns them into mean and population std.
-__global__ void stat_partial_kernel(const float *__restrict__ x, long long n, double *__restrict__ part) {
+__global__ void stat_partial_kernel(const float *__restrict__ x, long long n, double *__restrict__ part, UpdRows map) {
   __shared__ double s0[256], s1[256];
   double a = 0.0, b = 0.0;
   for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += static_cast<long long>(gridDim.x) * blockDim.x) {
-    const double v = x[i];
+    const long long row = real_row(map, i);
+    const double v = row >= 0 ? x[row] : 0.0;
     a += v; b += v * v;
   }
   s0[threadIdx.x] = a; s1[threadIdx.x] = b;
@@ -72,7 +88,7 @@ __global__ void stat_final_kernel(const double *__restrict__ part, int nb, long 
 struct UpdHyper { float clip_eps, ent_coef, vf_coef; };
 
 __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const double *__restrict__ adv_stats,
-                               float *__restrict__ partial, size_t n_params, double *__restrict__ term_partial) {
+                               float *__restrict__ partial, size_t n_params, double *__restrict__ term_partial, int *status) {
   extern __shared__ __align__(16) float smf[];
   const int H = net.H, Din = net.Din, j = threadIdx.x, lane = j & 31, warp = j >> 5, n_warps = H >> 5;
   const int Dp = (Din + 3) & ~3;  // row stride of the input tile; the pad columns hold zeros
@@ -80,6 +96,7 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
   // d z1 takes the place of h2, which is dead by then: three CTAs fit an SM at H = 128
   float *xs = smf, *h1s = xs + kUpdRows * Dp, *h2s = h1s + kUpdRows * H, *dz2t = h2s + kUpdRows * H, *dz1t = h2s,
         *dl = dz2t + H * kUpdTS;  // dl [32][8]: d logits (6), d value
+  long long *rmap = reinterpret_cast<long long *>(dl + kUpdRows * 8);  // trajectory row of every row of the tile
   auto ld4 = [](const float *p) { return *reinterpret_cast<const float4 *>(p); };
   float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
   const bool has_actor = net.Wa != nullptr, has_value = net.Wv != nullptr;
@@ -94,9 +111,15 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
   for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     const long long row0 = tile * kUpdRows;
     const int n_valid = static_cast<int>(min(static_cast<long long>(kUpdRows), rows.n - row0));
-    for (int i = j; i < kUpdRows * Dp; i += H) {
-      const int r = i / Dp, k = i - r * Dp;
-      xs[i] = (r < n_valid && k < Din) ? rows.x[(row0 + r) * Din + k] : 0.0f;
+    if (j < kUpdRows) {
+      const long long row = j < n_valid ? real_row(rows, row0 + j) : -1;
+      rmap[j] = row;
+      if (j < n_valid && row < 0) atomicExch(status, kStatusBadIndex);
+    }
+    __syncthreads();
+    for (int r = warp; r < kUpdRows; r += n_warps) {  // a warp per row: consecutive lanes, consecutive floats
+      const long long row = rmap[r];
+      for (int k = lane; k < Dp; k += 32) xs[r * Dp + k] = (row >= 0 && k < Din) ? rows.x[row * Din + k] : 0.0f;
     }
     __syncthreads();
     float acc[kUpdRows];
@@ -157,8 +180,8 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
         float d[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) d[k] = 0.0f;
-        if (r < n_valid) {
-          const long long row = row0 + r;
+        if (rmap[r] >= 0) {
+          const long long row = rmap[r];
           if (has_actor) {
             float l[kActions], m = -INFINITY, sum = 0.0f;
 #pragma unroll
@@ -341,7 +364,7 @@ __global__ void adam_kernel(float *__restrict__ params, const float *__restrict_
 // weights][partial gradients: one slice per CTA].
 size_t upd_smem_bytes(int Din, int H) {
   return sizeof(float) * (static_cast<size_t>(kUpdRows) * ((Din + 3) & ~3) + 2 * static_cast<size_t>(kUpdRows) * H +
-                          static_cast<size_t>(H) * kUpdTS + kUpdRows * 8);
+                          static_cast<size_t>(H) * kUpdTS + kUpdRows * 8 + kUpdRows * 2);
 }
 
 struct UpdScratch {
@@ -376,7 +399,7 @@ cudaError_t ensure_update_scratch(mava_rollout *h, size_t n_params, int slices) 
 }
 
 cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava_ppo_hyper_t &hyper, float *grad_dev,
-                            float *terms_dev) {
+                            float *terms_dev, const int32_t *env_ids_dev, int32_t n_ids) {
   const mava_config_t &cfg = h->cfg;
   const int T = h->last_T, E = cfg.n_envs, N = cfg.n_agents, D = h->D, H = cfg.hidden;
   const ParamLayout L = param_layout(cfg, D, 1);
@@ -384,7 +407,8 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   int sms = 0;
   cudaError_t err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
   if (err != cudaSuccess) return err;
-  const long long R = static_cast<long long>(T) * E * N, S = static_cast<long long>(T) * E;
+  const int n_env = env_ids_dev ? n_ids : E;  // environments in the minibatch
+  const long long R = static_cast<long long>(T) * n_env * N, S = static_cast<long long>(T) * n_env;
   const long long tiles = (R + kUpdRows - 1) / kUpdRows;
   // as many CTAs (= gradient slices) as are resident at once with the larger of the two nets' shared-memory needs
   const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
@@ -408,7 +432,10 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   };
   tr(L.W1, H, D); tr(L.W2, H, H);
   if (central) { tr(L.C1, H, joint); tr(L.C2, H, H); }
-  stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part);
+  UpdRows rows{};
+  rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
+  rows.env_ids = env_ids_dev; rows.n_ids = n_env; rows.E = E; rows.per_env = N;
+  stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part, rows);
   stat_final_kernel<<<1, 1, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
   h->launches += 2;
   err = cudaMemsetAsync(sc.term_part, 0, sizeof(double) * 3 * 8 * slices, st);
@@ -419,7 +446,7 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
     const size_t smem = upd_smem_bytes(net.Din, net.H);
     cudaError_t e = cudaFuncSetAttribute(ppo_net_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    ppo_net_kernel<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part);
+    ppo_net_kernel<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part, h->d_status);
     h->launches += 1;
     return cudaGetLastError();
   };
@@ -429,8 +456,6 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   actor.Wa = params_dev + L.Wa; actor.ba = params_dev + L.ba;
   actor.Din = D; actor.H = H;
   actor.oW1 = L.W1; actor.ob1 = L.b1; actor.oW2 = L.W2; actor.ob2 = L.b2; actor.oWa = L.Wa; actor.oba = L.ba;
-  UpdRows rows{};
-  rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
   if (!central) {
     actor.Wv = params_dev + L.Wv; actor.bv = params_dev + L.bv; actor.oWv = L.Wv; actor.obv = L.bv;
     rows.value_old = h->buf.values; rows.ret = h->buf.ret; rows.vstride = 1;
@@ -446,6 +471,7 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
     critic.oW1 = L.C1; critic.ob1 = L.c1; critic.oW2 = L.C2; critic.ob2 = L.c2; critic.oWv = L.Cv; critic.obv = L.cv;
     UpdRows crows{};
     crows.x = h->buf.obs; crows.value_old = h->buf.values; crows.ret = h->buf.ret; crows.vstride = N; crows.n = S;
+    crows.env_ids = env_ids_dev; crows.n_ids = n_env; crows.E = E; crows.per_env = 1;
     err = run_net(critic, crows);
   }
   if (err != cudaSuccess) return err;
@@ -461,7 +487,7 @@ cudaError_t launch_adam_step(mava_rollout *h, float *params_dev, const float *gr
   cudaError_t err = ensure_update_scratch(h, P, 1);
   if (err != cudaSuccess) return err;
   const UpdScratch sc = carve(h, P, 1);
-  stat_partial_kernel<<<kStatBlocks, 256, 0, h->stream>>>(grad_dev, static_cast<long long>(P), sc.stat_part);
+  stat_partial_kernel<<<kStatBlocks, 256, 0, h->stream>>>(grad_dev, static_cast<long long>(P), sc.stat_part, UpdRows{});
   stat_final_kernel<<<1, 1, 0, h->stream>>>(sc.stat_part, kStatBlocks, static_cast<long long>(P), sc.stats);
   const float corr1 = static_cast<float>(1.0 - pow(static_cast<double>(hp.beta1), step));
   const float corr2 = static_cast<float>(1.0 - pow(static_cast<double>(hp.beta2), step));

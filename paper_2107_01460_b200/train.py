@@ -2,10 +2,11 @@
 repeat, with evaluation blocks in between -- every step a call into the C ABI, nothing computed in Python.
 
     python -m paper_2107_01460_b200.train [--workload 1] [--envs 1024] [--steps 64] [--iters 200] [--epochs 4]
-                                          [--lr 1e-3] [--eval-every 25]
+                                          [--lr 1e-3] [--eval-every 25] [--minibatches 1]
 
 Each iteration: mava_rollout_run (T steps of every environment, continuing where the last one stopped), mava_gae,
-then `epochs` passes of mava_ppo_grad + mava_adam_step over all rows of that rollout as one minibatch.  Every
+then `epochs` passes of mava_ppo_grad + mava_adam_step over the rows of that rollout, as one minibatch or, with
+--minibatches k, as k minibatches of environments drawn from a fresh permutation per pass.  Every
 `eval-every` iterations a second handle with the same shape runs a greedy evaluation block from fresh episodes and
 the mean return of the episodes that ended is printed (1.0 = every food item collected).
 
@@ -42,7 +43,7 @@ def average_gradients(grad):
 
 
 def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, epochs: int = 4, lr: float = 1e-3,
-          eval_every: int = 25, precision: int | None = None, log=print, rank: int = 0):
+          eval_every: int = 25, precision: int | None = None, log=print, rank: int = 0, minibatches: int = 1):
     """Runs the loop and returns the list of (iteration, mean greedy return) it evaluated."""
     build.build()
     w = wl.workload(workload)
@@ -56,6 +57,7 @@ def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, 
     hp = binding.ppo_defaults()
     hp.lr = lr
     history, step = [], 0
+    shuffle = torch.Generator(device="cuda").manual_seed(1234 + rank)
     for it in range(iters + 1):
         if it % eval_every == 0 or it == iters:
             r = mean_return(ev, params, 2 * cap, seed=10_000 + it)
@@ -66,10 +68,13 @@ def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, 
         ro.run(params, T)
         ro.gae(wl.GAMMA, wl.LAMBDA)
         for _ in range(epochs):
-            step += 1
-            terms, grad = ro.ppo_grad(params, hp)
-            average_gradients(grad)
-            ro.adam_step(params, grad, m, v, step, hp)
+            # an epoch: every environment once, in `minibatches` pieces of a fresh permutation (seeded, same on every run)
+            pieces = [None] if minibatches <= 1 else torch.randperm(n_envs, generator=shuffle, device="cuda").to(torch.int32).chunk(minibatches)
+            for ids in pieces:
+                step += 1
+                terms, grad = ro.ppo_grad(params, hp, env_ids=None if ids is None else ids.contiguous())
+                average_gradients(grad)
+                ro.adam_step(params, grad, m, v, step, hp)
     assert ro.status() == binding.MAVA_OK and ev.status() == binding.MAVA_OK
     ro.close()
     ev.close()
@@ -85,6 +90,7 @@ def main():
     ap.add_argument("--epochs", type=int, default=4)
     ap.add_argument("--lr", type=float, default=1e-3)
     ap.add_argument("--eval-every", type=int, default=25)
+    ap.add_argument("--minibatches", type=int, default=1, help="pieces of a shuffled epoch (environments per piece = envs / this)")
     args = ap.parse_args()
     import os
 
@@ -96,7 +102,7 @@ def main():
         dist.init_process_group("nccl")
         rank = dist.get_rank()
     train(args.workload, args.envs, args.steps, args.iters, args.epochs, args.lr, args.eval_every,
-          log=print if rank == 0 else (lambda *_: None), rank=rank)
+          log=print if rank == 0 else (lambda *_: None), rank=rank, minibatches=args.minibatches)
     if rank or "RANK" in os.environ:
         import torch.distributed as dist
 

@@ -124,3 +124,43 @@ def test_argument_errors():
     assert L.mava_ppo_grad(ro.handle, None, hp, grad.data_ptr(), None) == binding.MAVA_ERR_INVALID_ARG
     assert L.mava_adam_step(ro.handle, params.data_ptr(), grad.data_ptr(), grad.data_ptr(), grad.data_ptr(), 0, hp) == binding.MAVA_ERR_INVALID_ARG
     ro.close()
+
+
+@pytest.mark.parametrize("idx,n_envs,T", [(1, 60, 20), (3, 30, 9), (2, 41, 16)])
+def test_minibatches_of_environments(idx, n_envs, T):
+    """A shuffled subset of the environments as the minibatch: the oracle gets the same environments' columns."""
+    import torch
+
+    w, ro, params = _rolled_out(idx, n_envs, T, FP32)
+    g = torch.Generator(device="cuda").manual_seed(7 + idx)
+    new = params + 0.6 * torch.randn(params.shape, generator=g, device="cuda") * params.std()
+    perm = torch.randperm(n_envs, generator=g, device="cuda").to(torch.int32)
+    shapes = ppo.layer_shapes(wl.obs_dim(w), w["hidden"], w["n_agents"], w["net_kind"])
+    p64 = new.cpu().numpy().astype(np.float64)
+    total = np.zeros_like(p64)
+    pieces = [perm[: n_envs // 3].contiguous(), perm[n_envs // 3:].contiguous()]
+    for ids in pieces:
+        terms, grad = ro.ppo_grad(new, env_ids=ids)
+        assert ro.status() == binding.MAVA_OK
+        sel = ids.cpu().numpy().astype(np.int64)
+        take = lambda name, n: getattr(ro, name)[:n].cpu().numpy().astype(np.float64)[:, sel]
+        batch = ppo.batch_from_rollout(take("obs", T), ro.actions[:T].cpu().numpy()[:, sel], take("logp", T), take("values", T + 1),
+                                       take("adv", T), take("ret", T), w["net_kind"])
+        ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch)
+        ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch)
+        t = terms.cpu().numpy()
+        for k, name in enumerate(("total", "actor", "entropy", "value")):
+            assert abs(t[k] - ref[name]) <= 1e-5 * (1 + abs(ref[name])), (name, t[k], ref[name])
+        assert np.max(np.abs(grad.cpu().numpy() - ref_grad)) <= 2e-4 * np.max(np.abs(ref_grad))
+    # all environments in order as the "minibatch" = the plain call, bit for bit
+    ident = torch.arange(n_envs, dtype=torch.int32, device="cuda")
+    t1, g1 = ro.ppo_grad(new)
+    t2, g2 = ro.ppo_grad(new, env_ids=ident)
+    assert torch.equal(g1, g2) and torch.equal(t1, t2)
+    # an index out of range is reported, not followed
+    bad = ident.clone()
+    bad[3] = n_envs
+    ro.ppo_grad(new, env_ids=bad)
+    assert ro.status() == binding.MAVA_ERR_INVALID_ARG
+    assert ro.status() == binding.MAVA_OK
+    ro.close()
