@@ -368,7 +368,8 @@ def run_gpu(args):
         for idx in range(5):
             wi = wl.workload(idx)
             pi = pick_precision(binding, wi)
-            r_i, _, tr, tg, _ = time_workload(torch, binding, wi, pi, 5, 3, flush=flush)
+            r_i, p_i, tr, tg, _ = time_workload(torch, binding, wi, pi, 5, 3, flush=flush)
+            tu_ms = time_update(torch, r_i, p_i, wi, 2, 1, flush)  # update block on that rollout's rows (fp32 path)
             del r_i
             ri = wi["n_envs"] * wi["n_agents"] * wi["T"]
             tr_ms, tg_ms = sum(tr) / len(tr), sum(tg) / len(tg)
@@ -379,7 +380,9 @@ def run_gpu(args):
                           "rollout_roofline_bound": "hbm" if th >= tt else "tensor",
                           "rollout_roofline_frac": max(th, tt) / (tr_ms * 1e-3),
                           "gae_elements_per_s": ri / (tg_ms * 1e-3),
-                          "gae_hbm_frac": ri * gae_bytes_per_element(wi) / (tg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+                          "gae_hbm_frac": ri * gae_bytes_per_element(wi) / (tg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                          "update_ms": tu_ms, "update_rows_per_s": ri / (tu_ms * 1e-3),
+                          "update_alu_frac": 3 * ri * flops_per_row(wi) / (tu_ms * 1e-3) / 1e12 / alu_peak})
 
     # CPU baseline: the oracle on a bounded sample of the same workload
     cores = os.cpu_count() or 1
