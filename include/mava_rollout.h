@@ -172,7 +172,8 @@ void mava_ppo_defaults(mava_ppo_hyper_t *hp);
  * agents' observations concatenated).  Reads obs, actions, logp, values, adv, ret of the caller's buffers; writes
  * grad_dev [mava_params_count] (dL/dparams, parameter order) and, if not NULL, terms_dev [4] = L, actor term,
  * mean entropy, value term (device pointers).  fp32 arithmetic on either precision of the handle; the library
- * allocates its scratch (one gradient slice per SM) on the first call.  Asynchronous.
+ * allocates its scratch (one gradient slice per resident CTA, up to three per SM: params_count floats each) on the
+ * first call and keeps it until destroy.  Asynchronous.
  * Errors: INVALID_ARG (NULL pointers, no run yet, adv/ret NULL), CUDA. */
 int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, float *grad_dev, float *terms_dev);
 
