@@ -87,10 +87,14 @@ __global__ void stat_final_kernel(const double *__restrict__ part, int nb, long 
 
 struct UpdHyper { float clip_eps, ent_coef, vf_coef; };
 
-__global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const double *__restrict__ adv_stats,
+// HT = hidden width = threads per CTA; the register budget is set for the CTAs per SM that the shared memory allows.
+template <int HT>
+__global__ void __launch_bounds__(HT, HT == 256 ? 1 : (HT == 128 ? 3 : 4))
+ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const double *__restrict__ adv_stats,
                                float *__restrict__ partial, size_t n_params, double *__restrict__ term_partial, int *status) {
   extern __shared__ __align__(16) float smf[];
-  const int H = net.H, Din = net.Din, j = threadIdx.x, lane = j & 31, warp = j >> 5, n_warps = H >> 5;
+  constexpr int H = HT;
+  const int Din = net.Din, j = threadIdx.x, lane = j & 31, warp = j >> 5, n_warps = H >> 5;
   const int Dp = (Din + 3) & ~3;  // row stride of the input tile; the pad columns hold zeros
   // every inner product below reads four operands per shared-memory access (16-byte broadcast loads)
   // d z1 takes the place of h2, which is dead by then: three CTAs fit an SM at H = 128
@@ -98,6 +102,7 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
         *dl = dz2t + H * kUpdTS;  // dl [32][8]: d logits (6), d value
   long long *rmap = reinterpret_cast<long long *>(dl + kUpdRows * 8);  // trajectory row of every row of the tile
   auto ld4 = [](const float *p) { return *reinterpret_cast<const float4 *>(p); };
+  const int HH = H >> 1, up = j % HH, r0 = (j / HH) * (kUpdRows / 2);  // the two-unit mapping of the dense loops
   float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
   const bool has_actor = net.Wa != nullptr, has_value = net.Wv != nullptr;
   const float mean = has_actor ? static_cast<float>(adv_stats[0]) : 0.0f;
@@ -122,43 +127,37 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
       for (int k = lane; k < Dp; k += 32) xs[r * Dp + k] = (row >= 0 && k < Din) ? rows.x[row * Din + k] : 0.0f;
     }
     __syncthreads();
-    float acc[kUpdRows];
-    // hidden layer 1 and 2: thread j computes unit j of all rows of the tile
+    // hidden layer 1 and 2.  Here a thread computes two units (up, up + H/2) of half the tile's rows, so that one
+    // 16-byte broadcast read of the activations feeds eight multiply-adds.
+    auto dense2 = [&](const float *src, int stride, int K, int k_valid, const float *Wt, const float *bias, float *dst) {
+      float a0[kUpdRows / 2], a1[kUpdRows / 2];
 #pragma unroll
-    for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
-    for (int k = 0; k < Dp; k += 4) {
-      float w[4];
+      for (int r = 0; r < kUpdRows / 2; ++r) a0[r] = a1[r] = 0.0f;
+      for (int k = 0; k < K; k += 4) {
+        float w0[4], w1[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) w[q] = k + q < Din ? net.W1t[static_cast<size_t>(k + q) * H + j] : 0.0f;
+        for (int q = 0; q < 4; ++q) {
+          const bool ok = k + q < k_valid;
+          w0[q] = ok ? Wt[static_cast<size_t>(k + q) * H + up] : 0.0f;
+          w1[q] = ok ? Wt[static_cast<size_t>(k + q) * H + up + HH] : 0.0f;
+        }
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) {
-        const float4 x = ld4(xs + r * Dp + k);
-        acc[r] = fmaf(x.x, w[0], fmaf(x.y, w[1], fmaf(x.z, w[2], fmaf(x.w, w[3], acc[r]))));
+        for (int r = 0; r < kUpdRows / 2; ++r) {
+          const float4 x = ld4(src + (r0 + r) * stride + k);
+          a0[r] = fmaf(x.x, w0[0], fmaf(x.y, w0[1], fmaf(x.z, w0[2], fmaf(x.w, w0[3], a0[r]))));
+          a1[r] = fmaf(x.x, w1[0], fmaf(x.y, w1[1], fmaf(x.z, w1[2], fmaf(x.w, w1[3], a1[r]))));
+        }
       }
-    }
-    {
-      const float b = net.b1[j];
+      const float b0 = bias[up], b1v = bias[up + HH];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) h1s[r * H + j] = fmaxf(acc[r] + b, 0.0f);
-    }
+      for (int r = 0; r < kUpdRows / 2; ++r) {
+        dst[(r0 + r) * H + up] = fmaxf(a0[r] + b0, 0.0f);
+        dst[(r0 + r) * H + up + HH] = fmaxf(a1[r] + b1v, 0.0f);
+      }
+    };
+    dense2(xs, Dp, Dp, Din, net.W1t, net.b1, h1s);
     __syncthreads();
-#pragma unroll
-    for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
-    for (int k = 0; k < H; k += 4) {
-      float w[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) w[q] = net.W2t[static_cast<size_t>(k + q) * H + j];
-#pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) {
-        const float4 x = ld4(h1s + r * H + k);
-        acc[r] = fmaf(x.x, w[0], fmaf(x.y, w[1], fmaf(x.z, w[2], fmaf(x.w, w[3], acc[r]))));
-      }
-    }
-    {
-      const float b = net.b2[j];
-#pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) h2s[r * H + j] = fmaxf(acc[r] + b, 0.0f);
-    }
+    dense2(h1s, H, H, H, net.W2t, net.b2, h2s);
     __syncthreads();
     // heads and the per-row derivatives of the loss: one warp per row
     for (int r = warp; r < kUpdRows; r += n_warps) {
@@ -249,34 +248,49 @@ __global__ void ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const doub
     for (int r = 0; r < kUpdRows; r += 4)
       *reinterpret_cast<float4 *>(dz2t + j * kUpdTS + r) = make_float4(dzr[r], dzr[r + 1], dzr[r + 2], dzr[r + 3]);
     __syncthreads();
-    // d h1 = d z2 . W2 (rows of W2 are contiguous in j), d z1
+    // d h1 = d z2 . W2 (rows of W2 are contiguous in the unit index), d z1: again two units and half the rows per thread
+    {
+      float a0[kUpdRows / 2], a1[kUpdRows / 2];
 #pragma unroll
-    for (int r = 0; r < kUpdRows; ++r) acc[r] = 0.0f;
-    for (int i = 0; i < H; i += 4) {
-      float w[4];
+      for (int r = 0; r < kUpdRows / 2; ++r) a0[r] = a1[r] = 0.0f;
+      for (int i = 0; i < H; i += 4) {
+        float w0[4], w1[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) w[q] = net.W2[static_cast<size_t>(i + q) * H + j];
+        for (int q = 0; q < 4; ++q) {
+          w0[q] = net.W2[static_cast<size_t>(i + q) * H + up];
+          w1[q] = net.W2[static_cast<size_t>(i + q) * H + up + HH];
+        }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < 4; ++q) {
 #pragma unroll
-        for (int r = 0; r < kUpdRows; r += 4) {
-          const float4 d = ld4(dz2t + (i + q) * kUpdTS + r);
-          acc[r] = fmaf(d.x, w[q], acc[r]);
-          acc[r + 1] = fmaf(d.y, w[q], acc[r + 1]);
-          acc[r + 2] = fmaf(d.z, w[q], acc[r + 2]);
-          acc[r + 3] = fmaf(d.w, w[q], acc[r + 3]);
+          for (int r = 0; r < kUpdRows / 2; r += 4) {
+            const float4 d = ld4(dz2t + (i + q) * kUpdTS + r0 + r);
+            a0[r] = fmaf(d.x, w0[q], a0[r]); a0[r + 1] = fmaf(d.y, w0[q], a0[r + 1]);
+            a0[r + 2] = fmaf(d.z, w0[q], a0[r + 2]); a0[r + 3] = fmaf(d.w, w0[q], a0[r + 3]);
+            a1[r] = fmaf(d.x, w1[q], a1[r]); a1[r + 1] = fmaf(d.y, w1[q], a1[r + 1]);
+            a1[r + 2] = fmaf(d.z, w1[q], a1[r + 2]); a1[r + 3] = fmaf(d.w, w1[q], a1[r + 3]);
+          }
         }
       }
-    }
+      // d z1 takes h2's place: h2 was last read before the barrier that precedes this loop
 #pragma unroll
-    for (int r = 0; r < kUpdRows; ++r) {
-      dzr[r] = h1s[r * H + j] > 0.0f ? acc[r] : 0.0f;
-      gb1 += dzr[r];
+      for (int r = 0; r < kUpdRows / 2; r += 4) {
+        float4 z0, z1;
+        z0.x = h1s[(r0 + r) * H + up] > 0.0f ? a0[r] : 0.0f; z0.y = h1s[(r0 + r + 1) * H + up] > 0.0f ? a0[r + 1] : 0.0f;
+        z0.z = h1s[(r0 + r + 2) * H + up] > 0.0f ? a0[r + 2] : 0.0f; z0.w = h1s[(r0 + r + 3) * H + up] > 0.0f ? a0[r + 3] : 0.0f;
+        z1.x = h1s[(r0 + r) * H + up + HH] > 0.0f ? a1[r] : 0.0f; z1.y = h1s[(r0 + r + 1) * H + up + HH] > 0.0f ? a1[r + 1] : 0.0f;
+        z1.z = h1s[(r0 + r + 2) * H + up + HH] > 0.0f ? a1[r + 2] : 0.0f; z1.w = h1s[(r0 + r + 3) * H + up + HH] > 0.0f ? a1[r + 3] : 0.0f;
+        *reinterpret_cast<float4 *>(dz1t + up * kUpdTS + r0 + r) = z0;
+        *reinterpret_cast<float4 *>(dz1t + (up + HH) * kUpdTS + r0 + r) = z1;
+      }
     }
-#pragma unroll
-    for (int r = 0; r < kUpdRows; r += 4)
-      *reinterpret_cast<float4 *>(dz1t + j * kUpdTS + r) = make_float4(dzr[r], dzr[r + 1], dzr[r + 2], dzr[r + 3]);
     __syncthreads();
+    // bias gradient of layer 1: thread j sums d z1 of unit j over the tile's rows
+#pragma unroll
+    for (int r = 0; r < kUpdRows; r += 4) {
+      const float4 d = ld4(dz1t + j * kUpdTS + r);
+      gb1 += (d.x + d.y) + (d.z + d.w);
+    }
     // d W2[i][j] += sum_r d z2[r][i] h1[r][j]   (thread j, coalesced over j)
     {
       float hcol[kUpdRows];
@@ -414,10 +428,13 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
   const int joint = N * D;
   const size_t smem_max = upd_smem_bytes(central ? joint : D, H);
-  err = cudaFuncSetAttribute(ppo_net_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_max));
+  using KernelT = void (*)(UpdNet, UpdRows, UpdHyper, const double *, float *, size_t, double *, int *);
+  const KernelT kern = H == 64 ? ppo_net_kernel<64> : (H == 128 ? ppo_net_kernel<128> : (H == 256 ? ppo_net_kernel<256> : nullptr));
+  if (!kern) return cudaErrorNotSupported;
+  err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_max));
   if (err != cudaSuccess) return err;
   int per_sm = 1;
-  err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ppo_net_kernel, H, smem_max);
+  err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, H, smem_max);
   if (err != cudaSuccess) return err;
   if (per_sm < 1) per_sm = 1;
   const int slices = static_cast<int>(tiles < static_cast<long long>(sms) * per_sm ? tiles : static_cast<long long>(sms) * per_sm);
@@ -444,9 +461,9 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
   auto run_net = [&](const UpdNet &net, const UpdRows &rows) {
     const size_t smem = upd_smem_bytes(net.Din, net.H);
-    cudaError_t e = cudaFuncSetAttribute(ppo_net_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    ppo_net_kernel<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part, h->d_status);
+    kern<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part, h->d_status);
     h->launches += 1;
     return cudaGetLastError();
   };
