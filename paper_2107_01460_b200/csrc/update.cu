@@ -291,36 +291,37 @@ ppo_net_kernel(UpdNet net, UpdRows rows, UpdHyper hp, const double *__restrict__
       const float4 d = ld4(dz1t + j * kUpdTS + r);
       gb1 += (d.x + d.y) + (d.z + d.w);
     }
-    // d W2[i][j] += sum_r d z2[r][i] h1[r][j]   (thread j, coalesced over j)
-    {
-      float hcol[kUpdRows];
+    // Weight gradients, G[i][c] += sum_r dz[r][i] v[r][c]: a thread keeps two columns c of v (all 32 rows) in registers
+    // and walks over half of the units i, so that every address is added to by one thread only and a broadcast read of
+    // d z feeds eight multiply-adds.
+    auto weight_grad = [&](const float *dzt, const float *v, int v_stride, int n_cols, size_t g_off) {
+      const int i0 = (j / HH) * HH;
+      for (int cb = 0; cb < n_cols; cb += H) {
+        const int c0 = cb + up, c1 = cb + up + HH;
+        if (c0 >= n_cols) break;
+        const bool two = c1 < n_cols;
+        float v0[kUpdRows], v1[kUpdRows];
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) hcol[r] = h1s[r * H + j];
-      for (int i = 0; i < H; ++i) {
-        float sacc = 0.0f;
-#pragma unroll
-        for (int r = 0; r < kUpdRows; r += 4) {
-          const float4 d = ld4(dz2t + i * kUpdTS + r);
-          sacc = fmaf(d.x, hcol[r], fmaf(d.y, hcol[r + 1], fmaf(d.z, hcol[r + 2], fmaf(d.w, hcol[r + 3], sacc))));
+        for (int r = 0; r < kUpdRows; ++r) {
+          v0[r] = v[r * v_stride + c0];
+          v1[r] = two ? v[r * v_stride + c1] : 0.0f;
         }
-        atomicAdd(part + net.oW2 + static_cast<size_t>(i) * H + j, sacc);  // result unused: a fire-and-forget reduction, no load to wait for
-      }
-    }
-    // d W1[i][k] += sum_r d z1[r][i] x[r][k]    (thread k, coalesced over k)
-    for (int k = j; k < Din; k += H) {
-      float xcol[kUpdRows];
+        for (int i = i0; i < i0 + HH; ++i) {
+          float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-      for (int r = 0; r < kUpdRows; ++r) xcol[r] = xs[r * Dp + k];
-      for (int i = 0; i < H; ++i) {
-        float sacc = 0.0f;
-#pragma unroll
-        for (int r = 0; r < kUpdRows; r += 4) {
-          const float4 d = ld4(dz1t + i * kUpdTS + r);
-          sacc = fmaf(d.x, xcol[r], fmaf(d.y, xcol[r + 1], fmaf(d.z, xcol[r + 2], fmaf(d.w, xcol[r + 3], sacc))));
+          for (int r = 0; r < kUpdRows; r += 4) {
+            const float4 d = ld4(dzt + i * kUpdTS + r);
+            s0 = fmaf(d.x, v0[r], fmaf(d.y, v0[r + 1], fmaf(d.z, v0[r + 2], fmaf(d.w, v0[r + 3], s0))));
+            s1 = fmaf(d.x, v1[r], fmaf(d.y, v1[r + 1], fmaf(d.z, v1[r + 2], fmaf(d.w, v1[r + 3], s1))));
+          }
+          // results unused: fire-and-forget reductions, no load to wait for
+          atomicAdd(part + g_off + static_cast<size_t>(i) * n_cols + c0, s0);
+          if (two) atomicAdd(part + g_off + static_cast<size_t>(i) * n_cols + c1, s1);
         }
-        atomicAdd(part + net.oW1 + static_cast<size_t>(i) * Din + k, sacc);
       }
-    }
+    };
+    weight_grad(dz2t, h1s, H, H, net.oW2);    // d W2[i][j] = sum_r d z2[r][i] h1[r][j]
+    weight_grad(dz1t, xs, Dp, Din, net.oW1);  // d W1[i][k] = sum_r d z1[r][i] x[r][k]
     __syncthreads();
   }
   // what was kept in registers over all tiles
