@@ -77,9 +77,17 @@ __global__ void stat_partial_kernel(const float *__restrict__ x, long long n, do
   }
   if (threadIdx.x == 0) { part[2 * blockIdx.x] = s0[0]; part[2 * blockIdx.x + 1] = s1[0]; }
 }
+// One warp; lane l adds its contiguous share of the partials, lane 0 the 32 shares: the same order on every call.
 __global__ void stat_final_kernel(const double *__restrict__ part, int nb, long long n, double *__restrict__ out) {
+  __shared__ double sa[32], sb[32];
+  const int per = (nb + 31) / 32, lane = threadIdx.x;
   double a = 0.0, b = 0.0;
-  for (int i = 0; i < nb; ++i) { a += part[2 * i]; b += part[2 * i + 1]; }
+  for (int i = lane * per; i < min(nb, (lane + 1) * per); ++i) { a += part[2 * i]; b += part[2 * i + 1]; }
+  sa[lane] = a; sb[lane] = b;
+  __syncwarp();
+  if (lane != 0) return;
+  a = 0.0; b = 0.0;
+  for (int i = 0; i < 32; ++i) { a += sa[i]; b += sb[i]; }
   const double mean = a / static_cast<double>(n);
   const double var = fmax(b / static_cast<double>(n) - mean * mean, 0.0);
   out[0] = mean; out[1] = sqrt(var); out[2] = sqrt(b);  // [2]: the 2-norm, for the gradient clipping
@@ -348,12 +356,23 @@ __global__ void reduce_partials_kernel(const float *__restrict__ partial, size_t
                                        UpdHyper hp, float *__restrict__ terms) {
   for (size_t p = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; p < n_params; p += static_cast<size_t>(gridDim.x) * blockDim.x) {
     float s = 0.0f;
-    for (int c = 0; c < n_slices; ++c) s += partial[static_cast<size_t>(c) * n_params + p];
+#pragma unroll 8
+    for (int c = 0; c < n_slices; ++c) s += partial[static_cast<size_t>(c) * n_params + p];  // the loads do not wait for the sum
     grad[p] = s;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0 && terms) {
+  if (blockIdx.x != 0 || !terms) return;
+  // the loss terms: every thread of block 0 adds a contiguous share of the partial sums, thread 0 the shares
+  __shared__ double st[3][256];
+  {
+    const int per = (n_term + static_cast<int>(blockDim.x) - 1) / static_cast<int>(blockDim.x), t = threadIdx.x;
     double a = 0.0, e = 0.0, v = 0.0;
-    for (int i = 0; i < n_term; ++i) { a += term_partial[3 * i]; e += term_partial[3 * i + 1]; v += term_partial[3 * i + 2]; }
+    for (int i = t * per; i < min(n_term, (t + 1) * per); ++i) { a += term_partial[3 * i]; e += term_partial[3 * i + 1]; v += term_partial[3 * i + 2]; }
+    st[0][t] = a; st[1][t] = e; st[2][t] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0, e = 0.0, v = 0.0;
+    for (int i = 0; i < static_cast<int>(blockDim.x); ++i) { a += st[0][i]; e += st[1][i]; v += st[2][i]; }
     const double actor = -a / static_cast<double>(n_actor), ent = e / static_cast<double>(n_actor), val = v / static_cast<double>(n_value);
     terms[0] = static_cast<float>(actor - hp.ent_coef * ent + hp.vf_coef * val);
     terms[1] = static_cast<float>(actor);
@@ -454,7 +473,7 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
   rows.env_ids = env_ids_dev; rows.n_ids = n_env; rows.E = E; rows.per_env = N;
   stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part, rows);
-  stat_final_kernel<<<1, 1, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
+  stat_final_kernel<<<1, 32, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
   h->launches += 2;
   err = cudaMemsetAsync(sc.term_part, 0, sizeof(double) * 3 * 8 * slices, st);
   if (err == cudaSuccess) err = cudaMemsetAsync(sc.partial, 0, sizeof(float) * P * slices, st);
@@ -506,7 +525,7 @@ cudaError_t launch_adam_step(mava_rollout *h, float *params_dev, const float *gr
   if (err != cudaSuccess) return err;
   const UpdScratch sc = carve(h, P, 1);
   stat_partial_kernel<<<kStatBlocks, 256, 0, h->stream>>>(grad_dev, static_cast<long long>(P), sc.stat_part, UpdRows{});
-  stat_final_kernel<<<1, 1, 0, h->stream>>>(sc.stat_part, kStatBlocks, static_cast<long long>(P), sc.stats);
+  stat_final_kernel<<<1, 32, 0, h->stream>>>(sc.stat_part, kStatBlocks, static_cast<long long>(P), sc.stats);
   const float corr1 = static_cast<float>(1.0 - pow(static_cast<double>(hp.beta1), step));
   const float corr2 = static_cast<float>(1.0 - pow(static_cast<double>(hp.beta2), step));
   adam_kernel<<<128, 256, 0, h->stream>>>(params_dev, grad_dev, m_dev, v_dev, P, sc.stats, hp.max_grad_norm, hp.lr, hp.beta1, hp.beta2,
