@@ -33,8 +33,7 @@ from paper_2107_01460_b200 import workloads as wl  # noqa: E402
 
 METRIC = "env_agent_steps_per_s"
 UNIT = "env-agent-steps/s"
-# Filled from profiles/rollout_tc_cfg1_full.md; reset an entry to None when its kernel changes.
-NCU_TRAFFIC_BYTES = {("cfg1_8x8_2p2f_h128", "bf16"): 28624384 + 179968}
+DEFAULT_WORKLOAD = 4  # the largest workload that fits one GPU
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -69,6 +68,39 @@ def load_peaks():
             p = json.load(fh)
         return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
     return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def ncu_traffic(w, precision_name):
+    """DRAM bytes (read + write) of one launch of the rollout kernel on workload `w`, from the table of ncu captures
+    kept with the profiler summaries; None when there is no capture of this workload or when the kernel's sources
+    have changed since it was taken.  A capture of fewer environments is scaled by the environment count (traffic is
+    trajectory writes, proportional to the rows)."""
+    import hashlib
+
+    path = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+    if not os.path.exists(path):
+        return None, None
+    csrc = os.path.join(ROOT, "paper_2107_01460_b200", "csrc")
+    digest = hashlib.sha256()
+    for name in ("rollout_tc.cu", "rollout_tc_small.cuh", "env.cuh", "tc_common.cuh", "common.cuh"):
+        with open(os.path.join(csrc, name), "rb") as fh:
+            digest.update(fh.read())
+    digest = digest.hexdigest()[:16]
+    with open(path) as fh:
+        for line in fh:
+            parts = line.split()
+            if len(parts) < 6 or parts[0].startswith("#"):
+                continue
+            name, prec, envs, read_b, write_b, src = parts[:6]
+            if name == w["name"] and prec == precision_name:
+                if src != digest:
+                    return None, "the rollout kernel's sources changed after the ncu capture"
+                scale = w["n_envs"] / float(envs)
+                note = "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch"
+                if scale != 1.0:
+                    note += f", captured at {envs} environments and scaled by {scale:g}"
+                return (float(read_b) + float(write_b)) * scale, note
+    return None, None
 
 
 # ---- clock sampling -----------------------------------------------------------------------------
@@ -152,6 +184,27 @@ def sample_envs_for(w, seconds_target: float, cores: int) -> int:
     return n
 
 
+def oracle_baseline(w, seconds_each: float):
+    """The oracle as it stands on a bounded sample of workload `w` (the first min(E, 256) environments for the full T,
+    rollout + GAE; env-agent-steps/s is per row, so the figure does not depend on E): once on one thread with a
+    smaller sample, once with the environments split over all host cores; each repeated until `seconds_each` of wall
+    time have gone by."""
+    params = wl.make_params(w)
+    cores = os.cpu_count() or 1
+    n_multi = min(w["n_envs"], 256)
+    n_single = max(1, min(n_multi, sample_envs_for(w, seconds_each / 2.0, 1)))
+    out = {}
+    for label, n_env, n_thr in (("single_thread", n_single, 1), ("all_cores", n_multi, cores)):
+        rows, secs, passes, used = 0, 0.0, 0, n_thr
+        while secs < seconds_each and passes < 256:
+            r_, s_, used = oracle_sample_run(w, params, n_env, n_thr)
+            rows += r_; secs += s_; passes += 1
+        out[label] = {"value": rows / secs, "unit": UNIT, "cores": used, "kind": "oracle",
+                      "sample": f"first {n_env} of {w['n_envs']} envs x full T={w['T']} (rollout + GAE), {passes} pass(es), "
+                                f"{secs:.1f} s wall"}
+    return out
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -173,8 +226,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total_s / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w["name"], "n_envs": w["n_envs"], "T": w["T"], "n_agents": w["n_agents"],
-                   "hidden": w["hidden"]},
+        "config": {"workload": w["name"], "n_envs_per_gpu": w["n_envs"], "T": w["T"], "n_agents": w["n_agents"],
+                   "hidden": w["hidden"], "obs_dim": wl.obs_dim(w), "global_envs": w["n_envs"],
+                   "parallelism": "env-shards x1", "l2": "host run: no device cache to flush"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -239,8 +293,9 @@ def time_evaluate(torch, ro, params, w, steps, warmup, flush):
     return sum(times) / len(times)
 
 
-def time_update(torch, ro, params, w, steps, warmup, flush):
-    """Device timing of the update block on the rows of one rollout: PPO loss + gradient, then one Adam step (ms)."""
+def time_update(torch, binding, ro, params, w, steps, warmup, flush):
+    """Device timing of the update block on the rows of one rollout: PPO loss + gradient, then one Adam step (ms);
+    also names the arithmetic path the handle's precision selects."""
     ro.run(params, w["T"])
     ro.gae(wl.GAMMA, wl.LAMBDA)
     p = params.clone()
@@ -256,7 +311,8 @@ def time_update(torch, ro, params, w, steps, warmup, flush):
         e1.synchronize()
         if i >= warmup:
             times.append(e0.elapsed_time(e1))
-    return sum(times) / len(times)
+    path = "bf16 tcgen05" if ro.cfg.precision == binding.MAVA_PRECISION_BF16 and binding.update_on_tensor_cores(ro.cfg) else "fp32 SIMT"
+    return sum(times) / len(times), path
 
 
 def time_e2e(torch, binding, ro, w, steps, warmup):
@@ -278,6 +334,38 @@ def time_e2e(torch, binding, ro, w, steps, warmup):
         if i >= warmup:
             times.append(dt)
     return sum(times) / len(times), h2d, d2h
+
+
+def rollout_roofline(w, rows, roll_ms, peaks, precision):
+    """The rollout launch against the slower of its two bounds.  A kernel timed alone between L2 flushes is measured
+    against the burst tensor peak; the fraction of the sustained (power-capped, seconds-long) peak is given beside it."""
+    t_hbm = rows * bytes_per_row(w) / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = rows * flops_per_row(w) / (peaks["bf16_tflops"] * 1e12)
+    if t_hbm >= t_tensor:
+        ach = rows * bytes_per_row(w) / (roll_ms * 1e-3) / 1e9
+        r = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
+    else:
+        ach = rows * flops_per_row(w) / (roll_ms * 1e-3) / 1e12
+        r = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+             "frac": ach / peaks["bf16_tflops"], "peak_kind": "burst (kernel timed alone)",
+             "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"],
+             "sustained_peak": peaks["bf16_tflops_sustained"]}
+    r["kernel"] = "rollout (fused env step + MLP + sampler), %s" % ("bf16 tcgen05" if precision else "fp32 SIMT")
+    r["traffic"], r["traffic_note"] = ncu_traffic(w, "bf16" if precision else "fp32")
+    r["peak_source"] = "of " + peaks["source"]
+    r["kernel_ms"] = roll_ms
+    r["algorithmic_bytes"] = rows * bytes_per_row(w)
+    r["algorithmic_flops"] = rows * flops_per_row(w)
+    return r
+
+
+def update_report(w, rows, upd_ms, upd_path, peaks):
+    """Update block: forward and the two backward products of every layer = 3 x the forward FLOPs, against the bf16
+    tensor peak (the block's products are GEMMs over the rollout's rows)."""
+    ach = 3 * rows * flops_per_row(w) / (upd_ms * 1e-3) / 1e12
+    return {"value": rows / (upd_ms * 1e-3), "unit": "rows/s", "ms": upd_ms, "bound": "tensor", "achieved": ach,
+            "peak": peaks["bf16_tflops"], "unit_roofline": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+            "path": upd_path + " (mava_ppo_grad + mava_adam_step), all rows of the rollout as one minibatch"}
 
 
 def run_gpu(args):
@@ -318,7 +406,7 @@ def run_gpu(args):
     step_ms = (sum(t_roll) + sum(t_gae)) / args.steps
     e2e_s, h2d, d2h = time_e2e(torch, binding, ro, w, max(3, args.steps // 4), 2)
     eval_ms = time_evaluate(torch, ro, params, w, max(3, args.steps // 4), 3, flush)  # rank-local, reported by rank 0
-    upd_ms = time_update(torch, ro, params, w, max(3, args.steps // 4), 3, flush) if rank == 0 else 0.0
+    upd_ms, upd_path = time_update(torch, binding, ro, params, w, max(3, args.steps // 4), 3, flush) if rank == 0 else (0.0, "")
     if dist is not None:
         t = torch.tensor([step_ms, e2e_s], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -330,67 +418,48 @@ def run_gpu(args):
 
     roll_ms = sum(t_roll) / len(t_roll)
     gae_ms = sum(t_gae) / len(t_gae)
-    t_hbm = rows * bytes_per_row(w) / (peaks["hbm_gbs"] * 1e9)
-    t_tensor = rows * flops_per_row(w) / (peaks["bf16_tflops_sustained"] * 1e12)
-    if t_hbm >= t_tensor:
-        ach = rows * bytes_per_row(w) / (roll_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"], "traffic": None}
-    else:
-        ach = rows * flops_per_row(w) / (roll_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None}
-    roofline["kernel"] = "rollout (fused env step + MLP + sampler), %s" % ("bf16 tcgen05" if precision else "fp32 SIMT")
-    # dram__bytes_read.sum + dram__bytes_write.sum of one launch of that kernel, from the ncu capture
-    # summarised under profiles/ (None when no capture of the current kernel exists for the workload)
-    roofline["traffic"] = NCU_TRAFFIC_BYTES.get((w["name"], "bf16" if precision else "fp32"))
-    roofline["traffic_note"] = ("ncu, one launch; below the algorithmic bytes because the 126 MB L2 still holds part of "
-                                "the trajectory when the kernel ends") if roofline["traffic"] else None
-    roofline["peak_source"] = "of " + peaks["source"]
-    roofline["kernel_ms"] = roll_ms
+    roofline = rollout_roofline(w, rows, roll_ms, peaks, precision)
     gae_ach = rows * gae_bytes_per_element(w) / (gae_ms * 1e-3) / 1e9
     gae = {"elements_per_s": rows / (gae_ms * 1e-3), "kernel_ms": gae_ms, "bound": "hbm", "achieved": gae_ach,
            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gae_ach / peaks["hbm_gbs"]}
+    update = update_report(w, rows, upd_ms, upd_path, peaks)
+    del ro, params
+    torch.cuda.empty_cache()
 
-    # update block (PPO loss + gradient + Adam over the rollout's rows): forward and the two backward products of every
-    # layer = 3 x the forward FLOPs; its only path so far is fp32 on the plain ALUs, whose peak is
-    # SMs x 128 lanes x 2 FLOP x the SM clock
-    alu_peak = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
-    upd_ach = 3 * rows * flops_per_row(w) / (upd_ms * 1e-3) / 1e12
-    update = {"value": rows / (upd_ms * 1e-3), "unit": "rows/s", "ms": upd_ms, "bound": "alu", "achieved": upd_ach,
-              "peak": alu_peak, "unit_roofline": "TFLOP/s", "frac": upd_ach / alu_peak,
-              "path": "fp32 validation path (mava_ppo_grad + mava_adam_step), all rows as one minibatch; no tensor-core path yet"}
-
-    # the other workloads, briefly (reported alongside; the headline stays the workload above)
+    # every workload of the table, briefly: device times, roofline fractions, and the oracle beside each
     sweep = []
     if not args.no_sweep and world == 1:
-        del ro
         for idx in range(5):
             wi = wl.workload(idx)
             pi = pick_precision(binding, wi)
             r_i, p_i, tr, tg, _ = time_workload(torch, binding, wi, pi, 5, 3, flush=flush)
-            tu_ms = time_update(torch, r_i, p_i, wi, 2, 1, flush)  # update block on that rollout's rows (fp32 path)
-            del r_i
+            tu_ms, tu_path = time_update(torch, binding, r_i, p_i, wi, 2, 1, flush)
+            del r_i, p_i
+            torch.cuda.empty_cache()
             ri = wi["n_envs"] * wi["n_agents"] * wi["T"]
             tr_ms, tg_ms = sum(tr) / len(tr), sum(tg) / len(tg)
-            th = ri * bytes_per_row(wi) / (peaks["hbm_gbs"] * 1e9)
-            tt = ri * flops_per_row(wi) / (peaks["bf16_tflops_sustained"] * 1e12)
-            sweep.append({"workload": wi["name"], "precision": "bf16" if pi else "fp32", "rollout_ms": tr_ms,
-                          "gae_ms": tg_ms, "env_agent_steps_per_s": ri / ((tr_ms + tg_ms) * 1e-3),
-                          "rollout_roofline_bound": "hbm" if th >= tt else "tensor",
-                          "rollout_roofline_frac": max(th, tt) / (tr_ms * 1e-3),
-                          "gae_elements_per_s": ri / (tg_ms * 1e-3),
-                          "gae_hbm_frac": ri * gae_bytes_per_element(wi) / (tg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                          "update_ms": tu_ms, "update_rows_per_s": ri / (tu_ms * 1e-3),
-                          "update_alu_frac": 3 * ri * flops_per_row(wi) / (tu_ms * 1e-3) / 1e12 / alu_peak})
+            rf = rollout_roofline(wi, ri, tr_ms, peaks, pi)
+            entry = {"workload": wi["name"], "precision": "bf16" if pi else "fp32", "rollout_ms": tr_ms,
+                     "gae_ms": tg_ms, "env_agent_steps_per_s": ri / ((tr_ms + tg_ms) * 1e-3),
+                     "rollout_roofline_bound": rf["bound"], "rollout_roofline_frac": rf["frac"],
+                     "rollout_roofline_frac_of_sustained_peak": rf.get("frac_of_sustained_peak"),
+                     "rollout_us_per_env_step": 1e3 * tr_ms / wi["T"],
+                     "gae_elements_per_s": ri / (tg_ms * 1e-3),
+                     "gae_hbm_frac": ri * gae_bytes_per_element(wi) / (tg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "update_ms": tu_ms, "update_path": tu_path, "update_rows_per_s": ri / (tu_ms * 1e-3),
+                     "update_tensor_frac": 3 * ri * flops_per_row(wi) / (tu_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+            if not args.no_oracle:
+                entry["cpu_baseline"] = oracle_baseline(wi, args.oracle_seconds)
+            sweep.append(entry)
 
-    # CPU baseline: the oracle on a bounded sample of the same workload
-    cores = os.cpu_count() or 1
-    n_sample = sample_envs_for(w, 12.0, cores)
-    cpu_rows, cpu_s, used, passes = 0, 0.0, cores, 0
-    while cpu_s < 1.5 and passes < 64:  # small workloads: several passes, so that the sample is tens of core-seconds
-        r_, s_, used = oracle_sample_run(w, wl.make_params(w), n_sample, cores)
-        cpu_rows += r_; cpu_s += s_; passes += 1
+    # CPU baseline of the headline workload: the oracle on a bounded sample of it
+    if sweep and "cpu_baseline" in sweep[args.workload]:
+        cpu = dict(sweep[args.workload]["cpu_baseline"]["all_cores"])
+        cpu["single_thread"] = sweep[args.workload]["cpu_baseline"]["single_thread"]
+    else:
+        both = oracle_baseline(w, args.oracle_seconds)
+        cpu = dict(both["all_cores"])
+        cpu["single_thread"] = both["single_thread"]
 
     line = {
         "metric": METRIC, "value": world * rows / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -407,8 +476,7 @@ def run_gpu(args):
         "evaluate": {"value": rows / (eval_ms * 1e-3), "unit": UNIT, "ms_per_block": eval_ms,
                      "block": f"greedy, T={T} steps, no trajectory stored (mava_rollout_evaluate), one GPU"},
         "update": update,
-        "cpu_baseline": {"value": cpu_rows / cpu_s, "unit": UNIT, "cores": used, "kind": "oracle",
-                         "sample": f"first {n_sample} of {E} envs x full T={T} (rollout + GAE), {passes} pass(es), {cpu_s:.1f} s wall"},
+        "cpu_baseline": cpu,
         "workloads": sweep,
     }
     print(json.dumps(line))
@@ -423,8 +491,10 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, help="index 0..4 of the workload table")
+    ap.add_argument("--workload", type=int, default=DEFAULT_WORKLOAD, help="index 0..4 of the workload table")
     ap.add_argument("--no-sweep", action="store_true", help="skip the brief timing of the other workloads")
+    ap.add_argument("--no-oracle", action="store_true", help="skip the oracle timing beside every workload of the sweep")
+    ap.add_argument("--oracle-seconds", type=float, default=8.0, help="wall time of each oracle timing (per workload: one thread, all cores)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     return run_reference(args) if args.impl == "reference" else run_gpu(args)

@@ -1,10 +1,10 @@
 /*
  * mava_rollout.h -- C ABI of the fused multi-agent rollout + GAE library (CUDA, sm_100a).
  *
- * The library runs, entirely on one GPU, the data-parallel "roll out experience from
- * vectorised environment copies" stage of the Anakin training loop described in the Mava
- * technical report (Section 2, "Strong baseline algorithms and training architectures",
- * and Figure 2), followed by advantage estimation for the multi-agent PPO systems the
+ * The library runs, entirely on one GPU, the experience-collection stage of the Anakin
+ * training loop of the Mava technical report (Section 2, "Strong baseline algorithms and
+ * training architectures", and Figure 2: every update function steps its own batch of
+ * environment copies), followed by advantage estimation for the multi-agent PPO systems the
  * report names (IPPO with per-agent critics, MAPPO with a centralised critic).
  *
  * E level-based-foraging gridworlds (the report's LBF tasks, Section 4) with N agents
@@ -114,8 +114,7 @@ size_t mava_params_count(const mava_config_t *cfg);
 int mava_rollout_create(const mava_config_t *cfg, const mava_buffers_t *buffers, void *cuda_stream,
                         mava_rollout_t **out);
 
-/* The fused rollout (Figure 2: "rolls out independent experience from N copies of the
- * environment").  Continues from the handle's environment states for T steps (1 <= T <= max_T),
+/* The fused rollout (the per-update experience collection of Figure 2).  Continues from the handle's environment states for T steps (1 <= T <= max_T),
  * writing rows 0..T-1 of obs, actions, logp, values, rewards, dones (and logits when flagged) and
  * the bootstrap row values[T].  params_dev: device pointer to mava_params_count floats, read
  * during the call's kernels (must stay valid until they finish).  With the central critic the one
@@ -148,8 +147,10 @@ int mava_rollout_evaluate(mava_rollout_t *h, const float *params_dev, int32_t T,
 /* Generalised advantage estimation over the rows of the last run (multi-agent PPO, Section 2):
  *   delta_t = r_t + gamma V_{t+1} (1-d_t) - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1},
  *   A_T = 0;  Ret_t = A_t + V_t.
- * Reads values, rewards, dones; writes adv and ret.  Asynchronous.
- * Errors: INVALID_ARG (no run yet, adv/ret NULL), CUDA. */
+ * Reads values, rewards, dones; writes adv and ret.  Handles runs of up to MAVA_GAE_MAX_T steps.  Asynchronous.
+ * Errors: INVALID_ARG (no run yet, adv/ret NULL, gamma or lambda outside [0, 1]), CAPACITY (the last run
+ * was longer than MAVA_GAE_MAX_T steps), CUDA. */
+#define MAVA_GAE_MAX_T 1024
 int mava_gae(mava_rollout_t *h, float gamma, float lambda);
 
 /* Update block (Section 2: each update function minimises the multi-agent PPO loss on the rolled-out experience;
@@ -226,19 +227,40 @@ int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32
  * and calls no allocating routine: the library's scratch (status word, environment states,
  * re-laid-out weights) lives in one static device array of MAVA_STATIC_SCRATCH_BYTES that every
  * GPU loading the library holds until the process exits.
- *   - Shapes whose scratch does not fit (60 bytes per environment plus up to 201 KB of weights,
- *     i.e. roughly 13 000 environments) are refused with MAVA_ERR_CAPACITY; T > cfg->max_T too.
+ *   - The scratch of a shape is 256 bytes + 60 bytes per environment + the re-laid-out weights, each part
+ *     rounded up to 256 bytes.  The weights depend on the shape and the precision: bf16 images take 18 KB
+ *     (H = 64), 70 KB (H = 128) or 205 KB (H = 256, about 13 000 environments fit beside them); the fp32 path
+ *     keeps 4 bytes per parameter (24 KB ... 350 KB for the shared-torso shapes, 930 KB with the centralised
+ *     critic, which leaves room for about 1 600 environments).  A shape whose scratch is larger than the
+ *     array is refused with MAVA_ERR_CAPACITY, and so is T > cfg->max_T.  The bf16 path with the centralised
+ *     critic needs far more scratch than the array (critic weight images and an observation block) and is
+ *     refused with MAVA_ERR_UNSUPPORTED: use the fp32 path or a handle.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress);
  *     make that first call before any stream capture.
  *   - All calls share the array and it keeps the previous call's contents; the call clears what
  *     must start at zero.  Two calls that overlap on the GPU (different streams or threads) race:
  *     serialise them.  It does not touch handles made by mava_rollout_create.
- *   - cfg, buffers, params_dev and T mean what they mean for create and run; GAE is not included
- *     (mava_gae needs no scratch).  The call waits for the stream and returns MAVA_OK,
- *     MAVA_ERR_DEVICE_TIMEOUT, or the errors of create/run. */
+ *   - cfg, buffers, params_dev and T mean what they mean for create and run.  GAE is not included and
+ *     cannot be reached from here: mava_gae works on a handle made by mava_rollout_create (which
+ *     allocates).  The call waits for the stream and returns MAVA_OK, MAVA_ERR_DEVICE_TIMEOUT, or the
+ *     errors of create/run. */
 #define MAVA_STATIC_SCRATCH_BYTES (1u << 20)
 int mava_rollout_run_static(const mava_config_t *cfg, const mava_buffers_t *buffers, const float *params_dev,
                             int32_t T, void *cuda_stream);
+
+/* Self-test hook of the failure-detection path (no counterpart in the report).  Every wait of a kernel on an
+ * mbarrier is bounded; when one runs out the kernel records it in the status word, lets the copies it still has
+ * in flight land, frees its tensor memory and returns, and mava_rollout_status answers MAVA_ERR_DEVICE_TIMEOUT.
+ * This call arms the NEXT launch of `which` (MAVA_EXPIRE_GAE: the copy-engine GAE kernel; MAVA_EXPIRE_ROLLOUT:
+ * the 128-row tensor-core rollout kernel) so that one thread block makes one extra wait, with a limit of a few
+ * thousand polls, on a barrier phase that nothing will complete, at a point where none of its copies or MMAs is
+ * outstanding.  That block gives up exactly as after a real time-out; its outputs (and, for the rollout, the
+ * environment states of its tile) are then incomplete, so the caller resets the handle afterwards.  One launch
+ * only; a launch that takes another kernel (a shape the armed kernel does not serve) leaves the request armed.
+ * Errors: INVALID_ARG. */
+#define MAVA_EXPIRE_GAE 1
+#define MAVA_EXPIRE_ROLLOUT 2
+int mava_debug_expire_next_wait(mava_rollout_t *h, int32_t which);
 
 /* Number of kernels this handle has launched so far (for launch accounting). */
 int64_t mava_rollout_launch_count(const mava_rollout_t *h);

@@ -23,6 +23,9 @@ MAVA_PRECISION_BF16 = 1
 MAVA_FLAG_WRITE_LOGITS = 1
 MAVA_FLAG_HIDDEN_IN_TMEM = 2
 MAVA_FLAG_WIDE_TILES = 4
+MAVA_EXPIRE_GAE = 1
+MAVA_EXPIRE_ROLLOUT = 2
+MAVA_GAE_MAX_T = 1024
 N_ACTIONS = 6
 
 EXPORTS = [
@@ -30,7 +33,7 @@ EXPORTS = [
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
     "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate", "mava_ppo_defaults", "mava_ppo_grad",
-    "mava_adam_step", "mava_ppo_grad_envs",
+    "mava_adam_step", "mava_ppo_grad_envs", "mava_debug_expire_next_wait",
 ]
 
 
@@ -91,6 +94,7 @@ def lib():
         L.mava_ppo_grad.argtypes = [vp, vp, hpp, vp, vp]; L.mava_ppo_grad.restype = C.c_int
         L.mava_ppo_grad_envs.argtypes = [vp, vp, hpp, vp, C.c_int32, vp, vp]; L.mava_ppo_grad_envs.restype = C.c_int
         L.mava_adam_step.argtypes = [vp, vp, vp, vp, vp, C.c_int32, hpp]; L.mava_adam_step.restype = C.c_int
+        L.mava_debug_expire_next_wait.argtypes = [vp, C.c_int32]; L.mava_debug_expire_next_wait.restype = C.c_int
         _lib = L
     return _lib
 
@@ -109,6 +113,11 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
         view_radius=w["view_radius"], episode_cap=w["episode_cap"], n_envs=w["n_envs"] if n_envs is None else n_envs,
         max_T=w["T"] if max_T is None else max_T, hidden=w["hidden"], net_kind=w["net_kind"], precision=precision,
         flags=flags, first_env=first_env, reserved=0, seed=w["seed"] if seed is None else seed)
+
+
+def update_on_tensor_cores(cfg: mava_config_t) -> bool:
+    """Whether mava_ppo_grad takes the bf16 tensor-core kernels for a handle of this configuration."""
+    return False
 
 
 def ppo_defaults() -> mava_ppo_hyper_t:
@@ -222,6 +231,9 @@ class Rollout:
 
     def status(self) -> int:
         return int(lib().mava_rollout_status(self.handle))
+
+    def debug_expire_next_wait(self, which: int):
+        _check(lib().mava_debug_expire_next_wait(self.handle, which), "mava_debug_expire_next_wait")
 
     def launch_count(self) -> int:
         return int(lib().mava_rollout_launch_count(self.handle))

@@ -71,6 +71,10 @@ int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_
   args.write_logits = (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) ? 1 : 0;
   args.status = h->d_status;
   args.obs_last = h->d_obs_last;
+  if (!ev && (h->expire_next & MAVA_EXPIRE_ROLLOUT) && h->cfg.precision == MAVA_PRECISION_BF16 && tc_rollout_is_wide(h)) {
+    args.debug_expire = 1;
+    h->expire_next &= ~MAVA_EXPIRE_ROLLOUT;
+  }
   if (ev) {
     args.eval = 1;
     args.greedy = ev->greedy;
@@ -176,9 +180,16 @@ int mava_rollout_evaluate(mava_rollout_t *h, const float *params_dev, int32_t T,
 int mava_gae(mava_rollout_t *h, float gamma, float lambda) {
   if (!h || h->last_T < 1 || !h->buf.adv || !h->buf.ret) return MAVA_ERR_INVALID_ARG;
   if (!(gamma >= 0.0f && gamma <= 1.0f && lambda >= 0.0f && lambda <= 1.0f)) return MAVA_ERR_INVALID_ARG;
+  if (h->last_T > MAVA_GAE_MAX_T) return MAVA_ERR_CAPACITY;
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
   return launch_gae(h, gamma, lambda) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
+}
+
+int mava_debug_expire_next_wait(mava_rollout_t *h, int32_t which) {
+  if (!h || (which != MAVA_EXPIRE_GAE && which != MAVA_EXPIRE_ROLLOUT)) return MAVA_ERR_INVALID_ARG;
+  h->expire_next |= which;
+  return MAVA_OK;
 }
 
 void mava_ppo_defaults(mava_ppo_hyper_t *hp) {
@@ -293,14 +304,14 @@ int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host) {
 int mava_rollout_collect_host(mava_rollout_t *h, const float *params_host, int32_t T, float gamma, float lambda,
                               const mava_host_buffers_t *out) {
   if (!h || !params_host || !out) return MAVA_ERR_INVALID_ARG;
+  if (T < 1) return MAVA_ERR_INVALID_ARG;
+  if (T > h->cfg.max_T || (h->buf.adv && h->buf.ret && T > MAVA_GAE_MAX_T)) return MAVA_ERR_CAPACITY;  // before anything is enqueued
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
   const size_t np = param_layout(h->cfg, h->D, 1).total;
   if (cudaMemcpyAsync(h->d_params_stage, params_host, np * sizeof(float), cudaMemcpyHostToDevice, h->stream) !=
       cudaSuccess)
     return MAVA_ERR_CUDA;
-  if (T < 1) return MAVA_ERR_INVALID_ARG;
-  if (T > h->cfg.max_T) return MAVA_ERR_CAPACITY;
   if (!h->copy_ready) {
     bool made = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; made && i <= kCollectChunks; ++i)

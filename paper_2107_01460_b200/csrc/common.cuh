@@ -57,6 +57,9 @@ struct RolloutArgs {
   float *ev_ret;        // [E]
   int32_t *ev_len;      // [E]
   int32_t *ev_actions;  // [T][E][N] or nullptr
+  // Self-test of the give-up path: block 0's first thread group makes one extra, short, bounded wait that nothing
+  // completes (after step 1's heads, when none of its MMAs or copies is outstanding) and treats it as a time-out.
+  int32_t debug_expire;
 };
 
 // Episode bookkeeping of one environment inside an evaluation block (all in step order, fp32 sums).
@@ -110,6 +113,7 @@ struct mava_rollout {
   uint32_t t_global;
   int32_t last_T;
   int64_t launches;
+  int32_t expire_next;  // MAVA_EXPIRE_* bits armed by mava_debug_expire_next_wait
   // collect_host: a second stream carries the device-to-host copies of the steps already rolled
   // out while the rest of the rollout runs (created on first use)
   cudaStream_t copy_stream;
@@ -134,6 +138,7 @@ size_t tc_weight_bytes(const mava_config_t &cfg, int D);
 cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev);
 cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args);
 bool tc_supported(const mava_config_t &cfg);
+bool tc_rollout_is_wide(const mava_rollout *h);  // the next bf16 rollout launch takes the 128-row kernel (not the few-rows form)
 size_t critic_weight_bytes(const mava_config_t &cfg);
 cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T);
 

@@ -191,7 +191,7 @@ template <int MAXT>
 __global__ void __launch_bounds__(MAXT, 1)
 gae_tma_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_r,
                const __grid_constant__ CUtensorMap map_d, float *__restrict__ adv, float *__restrict__ ret, int T, int E, int N, int C,
-               int W, int n_tiles, float gamma, float lambda, int *status) {
+               int W, int n_tiles, float gamma, float lambda, int *status, int debug_expire) {
   constexpr int L = kGaeL, S = kGaeStages;
   extern __shared__ __align__(128) unsigned char smem[];
   const int QW = C / 4;  // column quads per tile row
@@ -244,6 +244,10 @@ gae_tma_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant_
       if (!timed_out) { request(issued); ++issued; }
     }
     timed_out |= !mbar_wait(full0 + 8u * s, (i / S) & 1);
+    // self-test of the give-up path: block 0, at its last tile (every copy it asked for has landed by now), waits
+    // briefly for the phase of this stage that no further copy will complete
+    if (debug_expire && blockIdx.x == 0 && tid == 0 && i == my_tiles - 1)
+      timed_out |= !mbar_wait(full0 + 8u * s, ((i / S) & 1) ^ 1, 1u << 12);
     if (__syncthreads_or(timed_out)) { timed_out = true; break; }
     const uint32_t vbase = smem0 + static_cast<uint32_t>(s) * stage_stride, rbase = vbase + static_cast<uint32_t>(T + 1) * C * 4;
     // bit 4 k + j: column j of this thread's quad is not done at step t0 + k.  One division per tile; the quad's
@@ -381,11 +385,13 @@ cudaError_t launch_gae(mava_rollout *h, float gamma, float lambda) {
         encode_f32_map(&map_r, b.rewards, M, T, C, T, CU_TENSOR_MAP_SWIZZLE_NONE) &&
         encode_map_2d(&map_d, b.dones, true, E, T, W, T, CU_TENSOR_MAP_SWIZZLE_NONE)) {
       const int n_tiles = static_cast<int>((M + C - 1) / C);
+      const int expire = (h->expire_next & MAVA_EXPIRE_GAE) ? 1 : 0;
+      h->expire_next &= ~MAVA_EXPIRE_GAE;
       auto run = [&](auto kern) {
         cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (err != cudaSuccess) return err;
         kern<<<n_tiles < sms ? n_tiles : sms, threads, smem, h->stream>>>(map_v, map_r, map_d, b.adv, b.ret, T, E, N, C, W, n_tiles,
-                                                                          gamma, lambda, h->d_status);
+                                                                          gamma, lambda, h->d_status, expire);
         h->launches += 1;
         return cudaGetLastError();
       };

@@ -556,6 +556,9 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       if (PP) pair_arrive(kBarHid + (1 - g));  // the heads MMA is done reading the hidden-activation columns
+      // self-test of the give-up path: nothing of this group is outstanding here, and nothing will complete the
+      // barrier's next phase before this group's own next MMA batch
+      if (a.debug_expire && blockIdx.x == 0 && g == 0 && it == 0 && t == 1) timed_out |= !mbar_wait(bar, phase, 1u << 12);
       tc_fence_after();
       int action = 0;
       {
@@ -640,6 +643,18 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
 
 #include "rollout_tc_small.cuh"
 
+// Rows per tile of the few-rows form that serves this batch (0: the 128-row kernel).
+template <int N, int H, bool TM>
+int few_rows_tile(const mava_rollout *h, int sms) {
+  if constexpr (!TM && H == kTileRows) {
+    if ((h->cfg.flags & MAVA_FLAG_WIDE_TILES) == 0) {
+      if (h->cfg.n_envs <= sms * SmallShape<N, H, 16>::EPT_MAX) return 16;
+      if (h->cfg.n_envs <= sms * SmallShape<N, H, 32>::EPT_MAX) return 32;
+    }
+  }
+  return 0;
+}
+
 template <int N, int F, int H, bool TM>
 cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   using S = TcShape<N, H, TM>;
@@ -652,10 +667,9 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   if (err != cudaSuccess) return err;
   // Few rows per SM: the form with the rows as the N operand of the MMA.
   if constexpr (!TM && H == kTileRows) {
-    if ((h->cfg.flags & MAVA_FLAG_WIDE_TILES) == 0) {
-      if (h->cfg.n_envs <= sms * SmallShape<N, H, 16>::EPT_MAX) return launch_tc_small<N, F, H, 16>(h, args, sms);
-      if (h->cfg.n_envs <= sms * SmallShape<N, H, 32>::EPT_MAX) return launch_tc_small<N, F, H, 32>(h, args, sms);
-    }
+    const int rb = few_rows_tile<N, H, TM>(h, sms);
+    if (rb == 16) return launch_tc_small<N, F, H, 16>(h, args, sms);
+    if (rb == 32) return launch_tc_small<N, F, H, 32>(h, args, sms);
   }
   // Environments per tile: full tiles when there is enough work for every group of every SM,
   // otherwise smaller tiles so that all groups have one (the per-step chain is latency-bound).
@@ -697,6 +711,15 @@ bool tc_supported(const mava_config_t &cfg) {
 // Hidden activations in tensor memory: always for H = 256; for the smaller shapes only when the
 // handle asks for it (MAVA_FLAG_HIDDEN_IN_TMEM), which lets small cases exercise that path.
 static bool use_tm(const mava_rollout *h) { return h->variant >= 3 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0; }
+
+bool tc_rollout_is_wide(const mava_rollout *h) {
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return false;
+  if (use_tm(h)) return true;
+  if (h->variant == 1) return few_rows_tile<2, 128, false>(h, sms) == 0;
+  if (h->variant == 2) return few_rows_tile<3, 128, false>(h, sms) == 0;
+  return true;
+}
 
 size_t tc_weight_bytes(const mava_config_t &cfg, int) {
   switch (find_variant(cfg)) {  // the two layouts of a shape have the same image size

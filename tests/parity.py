@@ -1,13 +1,41 @@
 """GPU-vs-oracle comparison used by the gpu tests (the oracle replays the GPU's recorded actions)."""
 from __future__ import annotations
 
+import os
+import threading
+
 import numpy as np
 
 import oracle
 from paper_2107_01460_b200 import binding, workloads as wl
 
 TOL = {binding.MAVA_PRECISION_FP32: 1e-4, binding.MAVA_PRECISION_BF16: 2e-2}
+TOL_BF16_OPERANDS = 2e-3  # bf16 path against the oracle run with bf16-rounded operands
 GAE_TOL = 1e-5
+
+
+def oracle_rollout_threaded(ocfg, seed, params, T, env_ids, forced_actions, states=None, n_threads=None, **kw):
+    """oracle.rollout over `env_ids`, the environments split over the host cores (they are independent;
+    the C call releases the interpreter lock).  Same result as one call: arrays joined along the env axis."""
+    env_ids = np.asarray(env_ids, dtype=np.int32)
+    n_threads = min(n_threads or os.cpu_count() or 1, max(1, env_ids.size))
+    cuts = np.array_split(np.arange(env_ids.size), n_threads)
+    parts = [None] * len(cuts)
+
+    def work(i):
+        c = cuts[i]
+        parts[i] = oracle.rollout(ocfg, seed, params, T, env_ids[c], forced_actions=forced_actions[:, c],
+                                  states=None if states is None else [states[j] for j in c], **kw)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(len(cuts))]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    join = lambda name: (None if getattr(parts[0], name) is None  # noqa: E731
+                         else np.concatenate([getattr(p, name) for p in parts], axis=1))
+    return oracle.Rollout(*(join(n) for n in ("obs", "actions", "own_actions", "logp", "values", "rewards", "dones",
+                                               "logits", "margin")), sum((p.states for p in parts), []))
 
 
 def close(x, ref, tol):
@@ -46,8 +74,8 @@ def check_against_oracle(w, ro, params, T, precision, mlp_env_ids, obs_env_ids=N
     # 1. environment: bit-exact under the GPU's own actions, all environments
     all_ids = np.arange(E, dtype=np.int32)
     small = obs_env_ids is None
-    env = oracle.rollout(ocfg, seed, None, T, all_ids, forced_actions=g["actions"], compute_mlp=False,
-                         want_obs=small, t_global0=t_global0, states=states0)
+    env = oracle_rollout_threaded(ocfg, seed, None, T, all_ids, g["actions"], states=states0, compute_mlp=False,
+                                  want_obs=small, t_global0=t_global0)
     assert np.array_equal(env.rewards.view(np.uint32), g["rewards"].view(np.uint32)), "rewards differ"
     assert np.array_equal(env.dones, g["dones"]), "dones differ"
     if small:
@@ -71,8 +99,8 @@ def check_against_oracle(w, ro, params, T, precision, mlp_env_ids, obs_env_ids=N
     # 2. network + sampler on a subset of environments
     ids = np.asarray(mlp_env_ids, dtype=np.int32)
     sub_states = None if states0 is None else [states0[i] for i in ids]
-    ref = oracle.rollout(ocfg, seed, params, T, ids, forced_actions=g["actions"][:, ids], want_obs=False,
-                         t_global0=t_global0, states=sub_states)
+    ref = oracle_rollout_threaded(ocfg, seed, params, T, ids, g["actions"][:, ids], states=sub_states, want_obs=False,
+                                  t_global0=t_global0)
     out = {}
     out["logits"] = close(g["logits"][:, ids], ref.logits, tol)
     out["values"] = close(g["values"][:, ids], ref.values, tol)
@@ -86,6 +114,20 @@ def check_against_oracle(w, ro, params, T, precision, mlp_env_ids, obs_env_ids=N
     out["excused_actions"] = int(differ.sum())
     out["rows"] = int(differ.size)
     assert out["excused_actions"] <= max(2, int(10 * tol * differ.size)), out
+    if precision == binding.MAVA_PRECISION_BF16:
+        # the tight comparison: the oracle with its operands (observations, weights, hidden activations) rounded to
+        # bf16 as the tensor-core path rounds them; the action rule then uses this tolerance as well
+        emu = oracle_rollout_threaded(ocfg, seed, params, T, ids, g["actions"][:, ids], states=sub_states, want_obs=False,
+                                      t_global0=t_global0, emulate_bf16=True)
+        out["logits_bf16_operands"] = close(g["logits"][:, ids], emu.logits, TOL_BF16_OPERANDS)
+        out["values_bf16_operands"] = close(g["values"][:, ids], emu.values, TOL_BF16_OPERANDS)
+        out["logp_bf16_operands"] = close(g["logp"][:, ids], emu.logp, TOL_BF16_OPERANDS)
+        assert max(out["logits_bf16_operands"], out["values_bf16_operands"], out["logp_bf16_operands"]) <= 1.0, out
+        eps = 4.0 * TOL_BF16_OPERANDS * (1.0 + np.max(np.abs(emu.logits), axis=-1))
+        differ = g["actions"][:, ids] != emu.own_actions
+        assert not np.any(differ & (emu.margin > eps)), "an action differs away from a CDF boundary (bf16-operand oracle)"
+        out["excused_actions_bf16_operands"] = int(differ.sum())
+        assert out["excused_actions_bf16_operands"] <= max(2, int(10 * TOL_BF16_OPERANDS * differ.size)), out
 
     # 3. the sampler itself, exactly: re-sample in double from the GPU's own logits
     lg = g["logits"][:, ids].astype(np.float64)

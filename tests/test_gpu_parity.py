@@ -86,15 +86,6 @@ def test_reduced_configs_bf16(idx, n_envs, T, mode):
     ids = wl.sample_env_ids(n_envs, 6, 6, 6, seed=idx)
     out = check_against_oracle(w, ro, params, T, BF16, ids)
     print(idx, out)
-    # tighter: against the oracle run with bf16-rounded operands
-    ocfg = oracle.make_config(w)
-    acts = ro.actions[:T].cpu().numpy()
-    ref = oracle.rollout(ocfg, w["seed"], params, T, ids, forced_actions=acts[:, ids], want_obs=False,
-                         emulate_bf16=True)
-    lg = ro.logits[:T].cpu().numpy()[:, ids]
-    assert np.max(np.abs(lg - ref.logits) / (1 + np.abs(ref.logits))) < 2e-3
-    v = ro.values[:T + 1].cpu().numpy()[:, ids]
-    assert np.max(np.abs(v - ref.values) / (1 + np.abs(ref.values))) < 2e-3
 
 
 @pytest.mark.parametrize("idx,n_envs", [(1, 1024), (1, 2000), (2, 700), (2, 1400)])
@@ -115,17 +106,20 @@ def test_few_rows_form_equals_wide_tiles(idx, n_envs):
 
 # ---- full-size configs in the launch configuration the benchmark times ------------------------
 
-@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
 def test_full_size_configs(idx):
+    """Every workload at its full size, in bf16 with default flags (the launch shape the benchmark times).  Environment
+    arrays: all environments.  Network, sampler and log-probabilities: the first 64, the last 64 and 128 seeded-random
+    environments at every step, against the float64 oracle (2e-2) and against the oracle with bf16-rounded operands
+    (2e-3, which also sets the margin of the action rule)."""
     w = wl.workload(idx)
     precision = _precision(w) if _tc_available(w) else FP32
     params = wl.make_params(w)
     T, E = w["T"], w["n_envs"]
     ro, _ = run_gpu(w, precision, T, params=params)
-    mlp_ids = wl.sample_env_ids(E, 3, 3, 6, seed=idx)
-    obs_ids = wl.sample_env_ids(E, 64, 64, 128, seed=idx)
-    out = check_against_oracle(w, ro, params, T, precision, mlp_ids, obs_env_ids=obs_ids)
-    print(idx, precision, out)
+    ids = wl.sample_env_ids(E, 64, 64, 128, seed=idx)
+    out = check_against_oracle(w, ro, params, T, precision, ids, obs_env_ids=None if E <= 256 else ids)
+    print(idx, precision, len(ids), out)
 
 
 # ---- hand-worked transitions through set_state + forced actions -------------------------------

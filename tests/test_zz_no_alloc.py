@@ -38,18 +38,21 @@ def test_static_scratch_rollout_matches_handle_rollout(idx, precision, n_envs, T
                                   out["values"].data_ptr(), out["rewards"].data_ptr(), out["dones"].data_ptr(),
                                   None, None, out["logits"].data_ptr())
     stream = torch.cuda.current_stream().cuda_stream
-    tol = 1e-4 if precision == binding.MAVA_PRECISION_FP32 else 2e-2
     for call in range(2):
         for t in out.values():
             t.fill_(7)
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         rc = binding.mava_rollout_run_static(cfg, bufs, params.data_ptr(), T, stream)
+        free_after = torch.cuda.mem_get_info()[0]
         assert rc == binding.MAVA_OK, binding.strerror(rc)
-        for n in ("obs", "actions", "rewards", "dones"):
+        # the same kernels on the same inputs: the same bits in every array
+        for n in names:
             assert torch.equal(out[n], want[n]), (call, n)
-        for n in ("logp", "values", "logits"):
-            a, b = out[n].double(), want[n].double()
-            assert torch.all((a - b).abs() <= tol * (1 + b.abs())), (call, n)
+        # the first call on a device may make the driver load the module that holds the array; from then on the
+        # device's free memory must not move across a call
+        if call == 1:
+            assert free_after >= free_before, (free_before, free_after)
 
 
 def test_static_scratch_rejects_what_does_not_fit():
