@@ -24,6 +24,16 @@ observations concatenated, its target and old value those of agent 0's slot, all
 The optimiser is Adam (Kingma & Ba 2015) with bias correction, after scaling the gradient so that
 its global 2-norm is at most `max_grad_norm`.
 
+bf16-operand mode (`emulate_bf16=True`).  The tensor-core kernels of the update block multiply bf16 operands and
+accumulate in fp32; this mode states which quantities are rounded to bf16 (round to nearest even) and where, so
+that those kernels can be compared tightly: the observations x, the weights W1, W2 and the head weights as
+operands of every product (biases stay unrounded and are added to the accumulated sum); the hidden activations
+h1 = bf16(relu(z1)) and h2 = bf16(relu(z2)); the per-row derivatives of the loss with respect to the six logits
+and the value, rounded before they enter the products d h2 = dhead . Wh and d Wh = dhead^T . h2 (the head-bias
+gradients sum the unrounded derivatives); d z2 = bf16(d h2 * [h2 > 0]) and d z1 = bf16(d h1 * [h1 > 0]) before
+d W = d z^T . (input), d b = sum d z and d h1 = d z2 . W2.  Everything else (softmax, ratios, clips, means) is
+not rounded.  This is a reading of how a bf16 tensor-core path rounds, not something the report states.
+
 Pins (tests/test_oracle_ppo.py): float64 autograd of the same loss written with torch primitives as
 referee, central finite differences of `ppo_loss` (no autograd involved), the closed forms at
 rho = 1, the zero gradient of clipped rows, `torch.optim.Adam` and `clip_grad_norm_`.
@@ -72,27 +82,42 @@ def unpack(params: np.ndarray, shapes):
     return out
 
 
-def _forward_torso(x, W1, b1, W2, b2):
+def bf16_round(x):
+    """float64 array -> the nearest bfloat16 values (ties to even), as float64.  Written on the bit pattern of
+    binary32: add 0x7FFF plus the lowest kept bit, drop the low 16 bits."""
+    f = np.asarray(x, dtype=np.float64).astype(np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def _r(x, emulate_bf16):
+    return bf16_round(x) if emulate_bf16 else x
+
+
+def _forward_torso(x, W1, b1, W2, b2, emulate_bf16=False):
+    """z1, h1, z2, h2 of the two hidden layers; in bf16-operand mode x, W1, W2 arrive rounded and h1, h2 are rounded here."""
     z1 = x @ W1.T + b1
-    h1 = np.maximum(z1, 0.0)
+    h1 = _r(np.maximum(z1, 0.0), emulate_bf16)
     z2 = h1 @ W2.T + b2
-    h2 = np.maximum(z2, 0.0)
+    h2 = _r(np.maximum(z2, 0.0), emulate_bf16)
     return z1, h1, z2, h2
 
 
-def forward(params, shapes, net_kind, obs, joint_obs=None):
+def forward(params, shapes, net_kind, obs, joint_obs=None, emulate_bf16=False):
     """logits [R][6] and values (shared torso: [R]; centralised critic: [S] over `joint_obs`)."""
+    e = emulate_bf16
     p = unpack(np.asarray(params, dtype=np.float64), shapes)
     (W1, b1), (W2, b2), (Wa, ba) = p[0], p[1], p[2]
-    _, _, _, h2 = _forward_torso(obs, W1, b1, W2, b2)
-    logits = h2 @ Wa.T + ba
+    _, _, _, h2 = _forward_torso(_r(obs, e), _r(W1, e), b1, _r(W2, e), b2, e)
+    logits = h2 @ _r(Wa, e).T + ba
     if net_kind == 0:
         (Wv, bv) = p[3]
-        values = (h2 @ Wv.T + bv)[:, 0]
+        values = (h2 @ _r(Wv, e).T + bv)[:, 0]
     else:
         (C1, c1), (C2, c2), (Cv, cv) = p[3], p[4], p[5]
-        _, _, _, g2 = _forward_torso(joint_obs, C1, c1, C2, c2)
-        values = (g2 @ Cv.T + cv)[:, 0]
+        _, _, _, g2 = _forward_torso(_r(joint_obs, e), _r(C1, e), c1, _r(C2, e), c2, e)
+        values = (g2 @ _r(Cv, e).T + cv)[:, 0]
     return logits, values
 
 
@@ -107,11 +132,11 @@ def normalise(adv):
     return (adv - adv.mean()) / (adv.std() + 1e-8)
 
 
-def ppo_loss(params, shapes, net_kind, batch, hp: Hyper = Hyper()):
+def ppo_loss(params, shapes, net_kind, batch, hp: Hyper = Hyper(), emulate_bf16=False):
     """The loss terms of one minibatch.  `batch`: obs [R][D], actions [R], logp_old [R], adv [R] and,
     for the value rows, value_old, ret (shared torso: [R]; centralised: [S] with joint_obs [S][N*D])."""
     obs = np.asarray(batch["obs"], dtype=np.float64)
-    logits, values = forward(params, shapes, net_kind, obs, batch.get("joint_obs"))
+    logits, values = forward(params, shapes, net_kind, obs, batch.get("joint_obs"), emulate_bf16)
     a = np.asarray(batch["actions"], dtype=np.int64)
     logp_all = _log_softmax(logits)
     logp = logp_all[np.arange(a.size), a]
@@ -129,26 +154,30 @@ def ppo_loss(params, shapes, net_kind, batch, hp: Hyper = Hyper()):
             "clip_frac": float(np.mean(np.abs(rho - 1.0) > hp.clip_eps))}
 
 
-def _backward_torso(x, z1, h1, z2, dh2, W2):
-    """Gradients of the two hidden layers given dL/dh2; returns (dW1, db1, dW2, db2)."""
-    dz2 = dh2 * (z2 > 0.0)
+def _backward_torso(x, z1, h1, z2, h2, dh2, W2, emulate_bf16=False):
+    """Gradients of the two hidden layers given dL/dh2; returns (dW1, db1, dW2, db2).  The ReLU gates are
+    [z > 0]; in bf16-operand mode they are [h > 0] of the rounded activations (the same set unless a positive z
+    rounds to zero, below 1e-40) and d z2, d z1 are rounded before every use."""
+    dz2 = _r(dh2 * ((h2 if emulate_bf16 else z2) > 0.0), emulate_bf16)
     dW2 = dz2.T @ h1
     db2 = dz2.sum(axis=0)
     dh1 = dz2 @ W2
-    dz1 = dh1 * (z1 > 0.0)
+    dz1 = _r(dh1 * ((h1 if emulate_bf16 else z1) > 0.0), emulate_bf16)
     dW1 = dz1.T @ x
     db1 = dz1.sum(axis=0)
     return dW1, db1, dW2, db2
 
 
-def ppo_grad(params, shapes, net_kind, batch, hp: Hyper = Hyper()):
+def ppo_grad(params, shapes, net_kind, batch, hp: Hyper = Hyper(), emulate_bf16=False):
     """dL/dparams as a flat float64 array in the parameter order, by the chain rule written out."""
+    e = emulate_bf16
     params = np.asarray(params, dtype=np.float64)
     p = unpack(params, shapes)
     (W1, b1), (W2, b2), (Wa, ba) = p[0], p[1], p[2]
-    x = np.asarray(batch["obs"], dtype=np.float64)
+    W1, W2, Wa = _r(W1, e), _r(W2, e), _r(Wa, e)
+    x = _r(np.asarray(batch["obs"], dtype=np.float64), e)
     R = x.shape[0]
-    z1, h1, z2, h2 = _forward_torso(x, W1, b1, W2, b2)
+    z1, h1, z2, h2 = _forward_torso(x, W1, b1, W2, b2, e)
     logits = h2 @ Wa.T + ba
     a = np.asarray(batch["actions"], dtype=np.int64)
     logp_all = _log_softmax(logits)
@@ -176,28 +205,33 @@ def ppo_grad(params, shapes, net_kind, batch, hp: Hyper = Hyper()):
     v_old = np.asarray(batch["value_old"], dtype=np.float64)
     ret = np.asarray(batch["ret"], dtype=np.float64)
     grads = []
+    dba = d_logits.sum(axis=0)          # the unrounded derivatives
+    d_logits = _r(d_logits, e)          # as operands of the two products below
     dWa = d_logits.T @ h2
-    dba = d_logits.sum(axis=0)
     dh2 = d_logits @ Wa
     if net_kind == 0:
         (Wv, bv) = p[3]
+        Wv = _r(Wv, e)
         values = (h2 @ Wv.T + bv)[:, 0]
         dv = value_grad(values, v_old, ret)
-        dWv = dv[None, :] @ h2
         dbv = np.array([dv.sum()])
+        dv = _r(dv, e)
+        dWv = dv[None, :] @ h2
         dh2 = dh2 + dv[:, None] * Wv
-        dW1, db1, dW2, db2 = _backward_torso(x, z1, h1, z2, dh2, W2)
+        dW1, db1, dW2, db2 = _backward_torso(x, z1, h1, z2, h2, dh2, W2, e)
         grads = [dW1, db1, dW2, db2, dWa, dba, dWv, dbv]
     else:
-        dW1, db1, dW2, db2 = _backward_torso(x, z1, h1, z2, dh2, W2)
+        dW1, db1, dW2, db2 = _backward_torso(x, z1, h1, z2, h2, dh2, W2, e)
         (C1, c1), (C2, c2), (Cv, cv) = p[3], p[4], p[5]
-        xj = np.asarray(batch["joint_obs"], dtype=np.float64)
-        y1, g1, y2, g2 = _forward_torso(xj, C1, c1, C2, c2)
+        C1, C2, Cv = _r(C1, e), _r(C2, e), _r(Cv, e)
+        xj = _r(np.asarray(batch["joint_obs"], dtype=np.float64), e)
+        y1, g1, y2, g2 = _forward_torso(xj, C1, c1, C2, c2, e)
         values = (g2 @ Cv.T + cv)[:, 0]
         dv = value_grad(values, v_old, ret)
-        dCv = dv[None, :] @ g2
         dcv = np.array([dv.sum()])
-        dC1, dc1, dC2, dc2 = _backward_torso(xj, y1, g1, y2, dv[:, None] * Cv, C2)
+        dv = _r(dv, e)
+        dCv = dv[None, :] @ g2
+        dC1, dc1, dC2, dc2 = _backward_torso(xj, y1, g1, y2, g2, dv[:, None] * Cv, C2, e)
         grads = [dW1, db1, dW2, db2, dWa, dba, dC1, dc1, dC2, dc2, dCv, dcv]
     return np.concatenate([g.ravel() for g in grads])
 

@@ -166,3 +166,113 @@ def test_a_rolled_out_trajectory_feeds_the_update_and_a_small_step_lowers_the_lo
     assert np.isfinite(grad).all() and np.linalg.norm(grad) > 0
     loss1 = ppo.ppo_loss(params - 1e-3 * grad / np.linalg.norm(grad), shapes, w["net_kind"], batch)
     assert loss1["total"] < loss0["total"]
+
+
+# ---- bf16-operand mode -------------------------------------------------------------------------------------------
+
+def test_bf16_round_is_the_cast_torch_makes():
+    rng = np.random.default_rng(11)
+    x = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.integers(-30, 30, 4000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.0e-39, 65280.0, -2.5e-8],  # two exact ties among them
+                        np.float32(1.0) + np.arange(0, 64) * 2.0 ** -9])
+    want = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    got = ppo.bf16_round(x)
+    assert np.array_equal(got, want)
+    assert np.array_equal(ppo.bf16_round(got), got)  # idempotent
+
+
+class _RoundForward(torch.autograd.Function):
+    """y = bf16(x); the gradient passes through unchanged."""
+    @staticmethod
+    def forward(ctx, x):
+        return x.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+
+    @staticmethod
+    def backward(ctx, g):
+        return g
+
+
+class _RoundBackward(torch.autograd.Function):
+    """y = x; the gradient that flows back through here is rounded to bf16."""
+    @staticmethod
+    def forward(ctx, x):
+        return x.clone()
+
+    @staticmethod
+    def backward(ctx, g):
+        return g.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+
+
+@pytest.mark.parametrize("net_kind", [0, 1])
+def test_bf16_operand_mode_against_autograd_with_torch_bfloat16_casts(net_kind):
+    """The rounding points of the bf16-operand mode, restated as a torch graph: operands cast to torch.bfloat16 on the
+    way in (gradient passes), pre-activations and head outputs (before their bias) wrapped so that the gradient
+    flowing back through them is cast to torch.bfloat16.  Autograd then yields what the oracle must compute."""
+    hp = ppo.Hyper()
+    rng, shapes, params, batch = _setup(net_kind, seed=21, R=64)
+    # gradients of a realistic size (the 1/R of the mean and small derivatives): bf16 keeps the exponent
+    F = torch.nn.functional
+    rf, rb = _RoundForward.apply, _RoundBackward.apply
+    p_t = torch.from_numpy(params.copy()).requires_grad_(True)
+    off, layers = 0, []
+    for _, (o, i) in shapes:
+        W = p_t[off:off + o * i].reshape(o, i); off += o * i
+        b = p_t[off:off + o]; off += o
+        layers.append((W, b))
+    t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+
+    def torso(x, l1, l2):
+        h1 = rf(F.relu(rb(F.linear(rf(x), rf(l1[0]), l1[1]))))
+        return rf(F.relu(rb(F.linear(h1, rf(l2[0]), l2[1]))))
+
+    h = torso(t(batch["obs"]), layers[0], layers[1])
+    logits = rb(F.linear(h, rf(layers[2][0]))) + layers[2][1]
+    if net_kind == 0:
+        values = (rb(F.linear(h, rf(layers[3][0]))) + layers[3][1])[:, 0]
+    else:
+        g = torso(t(batch["joint_obs"]), layers[3], layers[4])
+        values = (rb(F.linear(g, rf(layers[5][0]))) + layers[5][1])[:, 0]
+    dist = torch.distributions.Categorical(logits=logits)
+    logp = dist.log_prob(torch.from_numpy(np.asarray(batch["actions"])))
+    ratio = torch.exp(logp - t(batch["logp_old"]))
+    adv = t(batch["adv"])
+    adv = (adv - adv.mean()) / (adv.std(unbiased=False) + 1e-8)
+    actor = -torch.minimum(ratio * adv, torch.clamp(ratio, 1 - hp.clip_eps, 1 + hp.clip_eps) * adv).mean()
+    v_old, ret = t(batch["value_old"]), t(batch["ret"])
+    v_clip = v_old + torch.clamp(values - v_old, -hp.clip_eps, hp.clip_eps)
+    value = 0.5 * torch.maximum((values - ret) ** 2, (v_clip - ret) ** 2).mean()
+    total = actor - hp.ent_coef * dist.entropy().mean() + hp.vf_coef * value
+    total.backward()
+    got = ppo.ppo_loss(params, shapes, net_kind, batch, hp, emulate_bf16=True)
+    assert abs(got["total"] - total.item()) < 1e-12 and abs(got["value"] - value.item()) < 1e-12
+    grad = ppo.ppo_grad(params, shapes, net_kind, batch, hp, emulate_bf16=True)
+    ref = p_t.grad.numpy()
+    assert np.max(np.abs(grad - ref)) < 1e-12 * max(1.0, np.max(np.abs(ref)))
+    # and the mode is a perturbation of the exact gradient of the size bf16 rounding gives, not something else
+    exact = ppo.ppo_grad(params, shapes, net_kind, batch, hp)
+    err = np.max(np.abs(grad - exact)) / np.max(np.abs(exact))
+    assert 1e-5 < err < 0.15, err  # 64 rows: a single ratio that changes sides of a clip is visible
+
+
+def test_bf16_operand_mode_changes_nothing_when_every_quantity_is_representable():
+    """Weights, observations and hidden activations that are small integers are bf16 numbers already; with the loss
+    reduced to the value term and targets that make every derivative a power of two, no rounding point changes a value
+    and the mode must return the exact gradient."""
+    D, H, R = 5, 4, 8
+    shapes = ppo.layer_shapes(D, H, 2, 0)
+    rng = np.random.default_rng(2)
+    parts = []
+    for _, (o, i) in shapes:
+        parts += [rng.integers(-2, 3, (o, i)).astype(np.float64).ravel(), rng.integers(-1, 2, o).astype(np.float64)]
+    params = np.concatenate(parts)
+    batch = {"obs": rng.integers(0, 3, (R, D)).astype(np.float64), "actions": rng.integers(0, 6, R),
+             "logp_old": np.full(R, np.log(1 / 6)), "adv": rng.standard_normal(R)}
+    _, values = ppo.forward(params, shapes, 0, batch["obs"])
+    batch["value_old"] = values.copy()
+    batch["ret"] = values - 0.5                       # V - R = 1/2 on every row, inside the clip range
+    hp = ppo.Hyper(ent_coef=0.0, vf_coef=1.0, clip_eps=0.2)
+    only_value = dict(batch, adv=np.zeros(R) + 0.0)
+    only_value["adv"] = np.array([1.0, -1.0] * (R // 2)) * 0.0  # zero advantages: the surrogate has no gradient
+    a = ppo.ppo_grad(params, shapes, 0, only_value, hp)
+    b = ppo.ppo_grad(params, shapes, 0, only_value, hp, emulate_bf16=True)
+    assert np.abs(a).max() > 0 and np.array_equal(a, b)
