@@ -56,6 +56,9 @@ extern "C" {
 #define MAVA_FLAG_WIDE_TILES 4 /* bf16 path: always use 128-row tiles, also for batches small
                                   enough for the few-rows form of the kernel; results are identical */
 
+#define MAVA_FLAG_UPDATE_FP32 8 /* bf16 handle: the update block (mava_ppo_grad*) still computes in fp32 on the
+                                  plain ALUs instead of taking the tensor-core kernels */
+
 typedef struct mava_rollout mava_rollout_t; /* opaque, owned by the library */
 
 /* Plain data, copied at create.  The observation width is D = 3*(2*view_radius+1)^2 + 2 + n_agents. */

@@ -23,6 +23,7 @@ MAVA_PRECISION_BF16 = 1
 MAVA_FLAG_WRITE_LOGITS = 1
 MAVA_FLAG_HIDDEN_IN_TMEM = 2
 MAVA_FLAG_WIDE_TILES = 4
+MAVA_FLAG_UPDATE_FP32 = 8
 MAVA_EXPIRE_GAE = 1
 MAVA_EXPIRE_ROLLOUT = 2
 MAVA_GAE_MAX_T = 1024
@@ -116,8 +117,10 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
 
 
 def update_on_tensor_cores(cfg: mava_config_t) -> bool:
-    """Whether mava_ppo_grad takes the bf16 tensor-core kernels for a handle of this configuration."""
-    return False
+    """Whether mava_ppo_grad takes the bf16 tensor-core kernels for a handle of this configuration (the shapes
+    they serve: shared torso, H <= 128, D <= 80)."""
+    return (cfg.precision == MAVA_PRECISION_BF16 and not cfg.flags & MAVA_FLAG_UPDATE_FP32 and
+            cfg.net_kind == MAVA_NET_SHARED_TORSO and cfg.hidden <= 128 and 77 + cfg.n_agents <= 80)
 
 
 def ppo_defaults() -> mava_ppo_hyper_t:

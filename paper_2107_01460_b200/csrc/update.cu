@@ -13,6 +13,7 @@
 // (the weight gradients are GEMMs over millions of rows) is not built yet.
 #include "common.cuh"
 #include "layout.h"
+#include "update_common.cuh"
 
 namespace mava {
 namespace {
@@ -21,37 +22,6 @@ constexpr int kUpdRows = 32;       // rows per tile
 constexpr int kUpdTS = kUpdRows;   // row stride of the transposed d z tiles [unit][row] (read by 16-byte broadcasts; the few
                                    // stores that fill them collide on banks, which costs less than the room padding takes)
 constexpr int kStatBlocks = 256;   // partial sums of the two reductions
-
-struct UpdNet {
-  const float *W1, *b1, *W2, *b2;  // caller layout [out][in]
-  const float *W1t, *W2t;          // [in][out] copies
-  const float *Wa, *ba, *Wv, *bv;  // heads (nullptr when the net has none of that kind)
-  int Din, H;
-  size_t oW1, ob1, oW2, ob2, oWa, oba, oWv, obv;  // offsets of the gradients in the flat array
-};
-struct UpdRows {
-  const float *x;                  // [n][Din]
-  const int32_t *actions;          // [n]          (actor)
-  const float *logp_old, *adv;     // [n]          (actor)
-  const float *value_old, *ret;    // [n * vstride] (value), element r at r * vstride
-  int vstride;
-  long long n;
-  // a minibatch of environments: row q of the batch is (step, env_ids[i], slot) with q = (step * n_ids + i) * per_env + slot;
-  // nullptr = every environment in order (row q is row q of the arrays)
-  const int32_t *env_ids;
-  int n_ids, E, per_env;
-};
-
-// Row of the trajectory arrays behind row q of the batch; -1 when the environment index is out of range.
-__device__ __forceinline__ long long real_row(const UpdRows &rows, long long q) {
-  if (!rows.env_ids) return q;
-  const long long per_step = static_cast<long long>(rows.n_ids) * rows.per_env;
-  const long long t = q / per_step, rem = q - t * per_step;
-  const int i = static_cast<int>(rem / rows.per_env), slot = static_cast<int>(rem - static_cast<long long>(i) * rows.per_env);
-  const int e = rows.env_ids[i];
-  if (e < 0 || e >= rows.E) return -1;
-  return (t * rows.E + e) * rows.per_env + slot;
-}
 
 __global__ void transpose_kernel(const float *__restrict__ W, float *__restrict__ Wt, int out, int in) {
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < out * in; i += gridDim.x * blockDim.x) {
@@ -93,7 +63,6 @@ __global__ void stat_final_kernel(const double *__restrict__ part, int nb, long 
   out[0] = mean; out[1] = sqrt(var); out[2] = sqrt(b);  // [2]: the 2-norm, for the gradient clipping
 }
 
-struct UpdHyper { float clip_eps, ent_coef, vf_coef; };
 
 // HT = hidden width = threads per CTA; the register budget is set for the CTAs per SM that the shared memory allows.
 template <int HT>
@@ -404,6 +373,7 @@ size_t upd_smem_bytes(int Din, int H) {
 struct UpdScratch {
   double *stats, *stat_part, *term_part;
   float *wt, *partial;
+  unsigned char *image;  // weight image of the tensor-core path
   int slices;
 };
 UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
@@ -413,6 +383,7 @@ UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
   s.stat_part = reinterpret_cast<double *>(p); p += sizeof(double) * 2 * kStatBlocks;
   s.term_part = reinterpret_cast<double *>(p); p += sizeof(double) * 3 * 8 * slices;
   s.wt = reinterpret_cast<float *>(p); p += sizeof(float) * ((n_params + 3) / 4 * 4);
+  s.image = p; p += (ppo_tc_image_bytes() + 255) / 256 * 256;
   s.partial = reinterpret_cast<float *>(p);
   s.slices = slices;
   return s;
@@ -420,9 +391,14 @@ UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
 
 }  // namespace
 
+// A bf16 handle takes the tensor-core kernels for the shapes they serve, unless it asked for the fp32 path.
+bool update_takes_tensor_cores(const mava_config_t &cfg, int D) {
+  return cfg.precision == MAVA_PRECISION_BF16 && (cfg.flags & MAVA_FLAG_UPDATE_FP32) == 0 && ppo_tc_supported(cfg, D);
+}
+
 cudaError_t ensure_update_scratch(mava_rollout *h, size_t n_params, int slices) {
   const size_t bytes = 64 + sizeof(double) * 2 * kStatBlocks + sizeof(double) * 3 * 8 * slices + sizeof(float) * ((n_params + 3) / 4 * 4) +
-                       sizeof(float) * n_params * slices;
+                       (ppo_tc_image_bytes() + 255) / 256 * 256 + sizeof(float) * n_params * slices;
   if (h->d_upd && h->upd_bytes >= bytes) return cudaSuccess;
   cudaFree(h->d_upd);
   h->d_upd = nullptr;
@@ -443,6 +419,28 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   if (err != cudaSuccess) return err;
   const int n_env = env_ids_dev ? n_ids : E;  // environments in the minibatch
   const long long R = static_cast<long long>(T) * n_env * N, S = static_cast<long long>(T) * n_env;
+  if (update_takes_tensor_cores(cfg, D)) {
+    // one CTA (= one gradient slice) per SM over tiles of 128 rows
+    const long long tiles128 = (R + 127) / 128;
+    const int slices = static_cast<int>(tiles128 < sms ? tiles128 : sms);
+    err = ensure_update_scratch(h, P, slices);
+    if (err != cudaSuccess) return err;
+    const UpdScratch sc = carve(h, P, slices);
+    cudaStream_t st = h->stream;
+    UpdRows rows{};
+    rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
+    rows.env_ids = env_ids_dev; rows.n_ids = n_env; rows.E = E; rows.per_env = N;
+    rows.value_old = h->buf.values; rows.ret = h->buf.ret; rows.vstride = 1;
+    stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part, rows);
+    stat_final_kernel<<<1, 32, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
+    h->launches += 2;
+    const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
+    err = launch_ppo_net_tc(h, params_dev, L, rows, hp, sc.stats, sc.image, sc.partial, P, sc.term_part, slices);
+    if (err != cudaSuccess) return err;
+    reduce_partials_kernel<<<128, 256, 0, st>>>(sc.partial, P, slices, grad_dev, sc.term_part, 8 * slices, R, R, hp, terms_dev);
+    h->launches += 1;
+    return cudaGetLastError();
+  }
   const long long tiles = (R + kUpdRows - 1) / kUpdRows;
   // as many CTAs (= gradient slices) as are resident at once with the larger of the two nets' shared-memory needs
   const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;

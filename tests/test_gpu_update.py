@@ -18,11 +18,13 @@ pytestmark = pytest.mark.gpu
 FP32, BF16 = binding.MAVA_PRECISION_FP32, binding.MAVA_PRECISION_BF16
 
 
-def _rolled_out(idx, n_envs, T, precision, bias_scale=0.1):
+def _rolled_out(idx, n_envs, T, precision, bias_scale=0.1, flags=binding.MAVA_FLAG_UPDATE_FP32):
+    """A handle after run + gae.  By default a bf16 handle keeps the fp32 update block (the path most cases here
+    check); flags=0 lets it take the tensor-core kernels."""
     import torch
 
     w = wl.workload(idx)
-    cfg = binding.make_config(w, precision=precision, max_T=T, n_envs=n_envs)
+    cfg = binding.make_config(w, precision=precision, max_T=T, n_envs=n_envs, flags=flags)
     ro = binding.Rollout(cfg)
     params = torch.from_numpy(wl.make_params(w, bias_scale=bias_scale)).cuda()
     ro.run(params, T)
@@ -164,3 +166,98 @@ def test_minibatches_of_environments(idx, n_envs, T):
     assert ro.status() == binding.MAVA_ERR_INVALID_ARG
     assert ro.status() == binding.MAVA_OK
     ro.close()
+
+
+# ---- tensor-core path (bf16 handles, shared torso, H <= 128) ----------------------------------------------------------
+# Tolerances.  Against the oracle in bf16-operand mode (same rounding points): every product of two bf16 numbers is
+# exact in the fp32 accumulator, so what is left is the order of the fp32 additions (about sqrt(R) * 2^-24 of the
+# largest partial sum), hidden activations that land on the other side of a bf16 rounding boundary (a fraction of
+# about 2^-24 / 2^-8 of the elements, one bf16 ulp each) and rows whose ratio or value sits within fp32 rounding of a
+# clip boundary (each worth 1/R of the gradient): 2e-3 * max|grad| and 2e-4 * (1 + |ref|) on the loss terms bound
+# these with a wide margin.  Against the exact float64 oracle the operands' rounding itself shows (2^-9 relative per
+# operand, logits good to 2e-2): 5e-2 * max|grad| and 2e-2 * (1 + |ref|).
+
+@pytest.mark.parametrize("idx,n_envs,T", [(0, 16, 32), (1, 77, 20), (2, 50, 33), (2, 300, 40), (0, 1, 3),
+                                          (1, 1024, 128)])  # the last: the size the benchmark times
+def test_tensor_core_update_matches_the_bf16_operand_oracle(idx, n_envs, T):
+    import torch
+
+    w, ro, params = _rolled_out(idx, n_envs, T, BF16, flags=0)
+    assert binding.update_on_tensor_cores(ro.cfg)
+    g = torch.Generator(device="cuda").manual_seed(idx)
+    new = params + 0.6 * torch.randn(params.shape, generator=g, device="cuda") * params.std()
+    hp = binding.ppo_defaults()
+    terms, grad = ro.ppo_grad(new, hp)
+    assert ro.status() == binding.MAVA_OK
+    shapes = ppo.layer_shapes(wl.obs_dim(w), w["hidden"], w["n_agents"], w["net_kind"])
+    batch = _oracle_batch(w, ro, T)
+    p64 = new.cpu().numpy().astype(np.float64)
+    t = terms.cpu().numpy()
+    gg = grad.cpu().numpy().astype(np.float64)
+    for emulate, g_tol, l_tol in ((True, 2e-3, 2e-4), (False, 5e-2, 2e-2)):
+        ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
+        ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
+        for k, name in enumerate(("total", "actor", "entropy", "value")):
+            assert abs(t[k] - ref[name]) <= l_tol * (1 + abs(ref[name])), (emulate, name, t[k], ref[name])
+        worst = np.max(np.abs(gg - ref_grad)) / np.max(np.abs(ref_grad))
+        assert worst <= g_tol, (emulate, worst)
+        # layer by layer as well: a layer with small gradients must not hide behind the largest one
+        off = 0
+        for name, (o, i) in shapes:
+            for lo, hi in ((off, off + o * i), (off + o * i, off + o * i + o)):
+                seg = np.max(np.abs(ref_grad[lo:hi]))
+                assert np.max(np.abs(gg[lo:hi] - ref_grad[lo:hi])) <= 5 * g_tol * seg + 1e-12, (emulate, name, lo)
+            off += o * i + o
+    terms2, grad2 = ro.ppo_grad(new, hp)
+    assert torch.equal(grad, grad2) and torch.equal(terms, terms2)  # fixed summation order
+    ro.close()
+
+
+@pytest.mark.parametrize("idx,n_envs,T", [(1, 333, 20), (2, 141, 16)])
+def test_tensor_core_update_on_minibatches_of_environments(idx, n_envs, T):
+    import torch
+
+    w, ro, params = _rolled_out(idx, n_envs, T, BF16, flags=0)
+    g = torch.Generator(device="cuda").manual_seed(17 + idx)
+    new = params + 0.6 * torch.randn(params.shape, generator=g, device="cuda") * params.std()
+    perm = torch.randperm(n_envs, generator=g, device="cuda").to(torch.int32)
+    shapes = ppo.layer_shapes(wl.obs_dim(w), w["hidden"], w["n_agents"], w["net_kind"])
+    p64 = new.cpu().numpy().astype(np.float64)
+    for ids in (perm[: n_envs // 3].contiguous(), perm[n_envs // 3:].contiguous()):
+        terms, grad = ro.ppo_grad(new, env_ids=ids)
+        assert ro.status() == binding.MAVA_OK
+        sel = ids.cpu().numpy().astype(np.int64)
+        take = lambda name, n: getattr(ro, name)[:n].cpu().numpy().astype(np.float64)[:, sel]
+        batch = ppo.batch_from_rollout(take("obs", T), ro.actions[:T].cpu().numpy()[:, sel], take("logp", T), take("values", T + 1),
+                                       take("adv", T), take("ret", T), w["net_kind"])
+        ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch, emulate_bf16=True)
+        ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch, emulate_bf16=True)
+        t = terms.cpu().numpy()
+        for k, name in enumerate(("total", "actor", "entropy", "value")):
+            assert abs(t[k] - ref[name]) <= 2e-4 * (1 + abs(ref[name])), (name, t[k], ref[name])
+        assert np.max(np.abs(grad.cpu().numpy() - ref_grad)) <= 2e-3 * np.max(np.abs(ref_grad))
+    ident = torch.arange(n_envs, dtype=torch.int32, device="cuda")
+    t1, g1 = ro.ppo_grad(new)
+    t2, g2 = ro.ppo_grad(new, env_ids=ident)
+    assert torch.equal(g1, g2) and torch.equal(t1, t2)  # rows through the copy engine or gathered by loads: the same bytes
+    bad = ident.clone()
+    bad[3] = n_envs
+    ro.ppo_grad(new, env_ids=bad)
+    assert ro.status() == binding.MAVA_ERR_INVALID_ARG
+    ro.close()
+
+
+def test_at_unchanged_parameters_the_ratios_of_a_bf16_handle_stay_near_one():
+    """logp and values stored by the bf16 rollout come from bf16 tensor-core arithmetic.  Re-evaluated by the update
+    block at the same parameters, the ratio must be 1 up to that arithmetic's noise: the tensor-core update (same
+    operand rounding as the rollout) keeps the surrogate within 1e-3 of zero and the clipped fraction at nothing;
+    the fp32 update on the same handle sees the rollout's bf16 rounding as policy change (reported, bounded)."""
+    out = {}
+    for name, flags in (("tensor", 0), ("fp32", binding.MAVA_FLAG_UPDATE_FP32)):
+        w, ro, params = _rolled_out(1, 256, 64, BF16, flags=flags)
+        terms, _ = ro.ppo_grad(params)
+        out[name] = abs(terms[1].item())
+        ro.close()
+    print(out)
+    assert out["tensor"] < 1e-3
+    assert out["fp32"] < 3e-2
