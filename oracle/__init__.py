@@ -112,6 +112,16 @@ def lib():
             C.POINTER(EnvState), C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
         ]
         L.orc_evaluate.restype = C.c_int
+        L.orc_rec_params_count.argtypes = [C.POINTER(Config)]
+        L.orc_rec_params_count.restype = C.c_int64
+        L.orc_rec_forward_env.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_rec_forward_env.restype = None
+        L.orc_rollout_rec.argtypes = [
+            C.POINTER(Config), C.c_uint64, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int32, C.c_uint32,
+            C.POINTER(EnvState), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+        ]
+        L.orc_rollout_rec.restype = C.c_int
         L.orc_gae.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_double,
                               C.c_double, C.c_void_p, C.c_void_p]
         L.orc_gae.restype = None
@@ -238,6 +248,58 @@ def rollout(cfg: Config, seed: int, params, T: int, env_ids, *, forced_actions=N
     if rc != 0:
         raise ValueError("orc_rollout rejected its arguments")
     return Rollout(obs, actions, own, logp, values, rewards, dones, logits, margin, list(st))
+
+
+def rec_params_count(cfg: Config) -> int:
+    return int(lib().orc_rec_params_count(C.byref(cfg)))
+
+
+def rec_forward_env(cfg: Config, params: np.ndarray, obs: np.ndarray, hidden: np.ndarray, emulate_bf16: bool = False):
+    """Recurrent policy, one environment, one step: obs [N][D] float32, hidden [N][H] float64 ->
+    (logits [N][6], values [N], new hidden [N][H]), all float64."""
+    p = np.ascontiguousarray(params, dtype=np.float32)
+    o = np.ascontiguousarray(obs, dtype=np.float32)
+    h = np.array(hidden, dtype=np.float64, order="C", copy=True)
+    assert p.size == rec_params_count(cfg) and o.size == cfg.n_agents * obs_dim(cfg) and h.shape == (cfg.n_agents, cfg.hidden)
+    logits = np.empty((cfg.n_agents, N_ACTIONS), dtype=np.float64)
+    values = np.empty(cfg.n_agents, dtype=np.float64)
+    lib().orc_rec_forward_env(C.byref(cfg), _ptr(p), _ptr(o), _ptr(h), int(emulate_bf16), _ptr(logits), _ptr(values))
+    return logits, values, h
+
+
+def rollout_rec(cfg: Config, seed: int, params, T: int, env_ids, *, forced_actions=None, states=None, hidden=None,
+                t_global0: int = 0, emulate_bf16: bool = False, want_obs: bool = True):
+    """The rollout with the recurrent policy; returns (Rollout, hidden [n][N][H] float64 after the run).  `hidden`
+    defaults to zeros (every environment at the start of an episode)."""
+    env_ids = np.ascontiguousarray(env_ids, dtype=np.int32)
+    n = int(env_ids.size)
+    N, D, H = cfg.n_agents, obs_dim(cfg), cfg.hidden
+    if states is None:
+        states = [env_reset(cfg, seed, int(e), 0) for e in env_ids]
+    st = (EnvState * n)(*states)
+    hid = np.zeros((n, N, H), dtype=np.float64) if hidden is None else np.array(hidden, dtype=np.float64, order="C", copy=True)
+    assert hid.shape == (n, N, H)
+    fa = None
+    if forced_actions is not None:
+        fa = np.ascontiguousarray(forced_actions, dtype=np.int32)
+        assert fa.shape == (T, n, N)
+    p = np.ascontiguousarray(params, dtype=np.float32)
+    assert p.size == rec_params_count(cfg)
+    obs = np.empty((T, n, N, D), dtype=np.float32) if want_obs else None
+    actions = np.empty((T, n, N), dtype=np.int32)
+    own = np.empty((T, n, N), dtype=np.int32)
+    logp = np.empty((T, n, N), dtype=np.float64)
+    values = np.empty((T + 1, n, N), dtype=np.float64)
+    rewards = np.empty((T, n, N), dtype=np.float32)
+    dones = np.empty((T, n), dtype=np.uint8)
+    logits = np.empty((T, n, N, N_ACTIONS), dtype=np.float64)
+    margin = np.empty((T, n, N), dtype=np.float64)
+    rc = lib().orc_rollout_rec(C.byref(cfg), C.c_uint64(seed), _ptr(p), int(emulate_bf16), n, _ptr(env_ids), T, t_global0,
+                               st, _ptr(hid), _ptr(fa), _ptr(obs), _ptr(actions), _ptr(own), _ptr(logp), _ptr(values),
+                               _ptr(rewards), _ptr(dones), _ptr(logits), _ptr(margin))
+    if rc != 0:
+        raise ValueError("orc_rollout_rec rejected its arguments")
+    return Rollout(obs, actions, own, logp, values, rewards, dones, logits, margin, list(st)), hid
 
 
 @dataclass

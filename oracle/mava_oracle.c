@@ -5,7 +5,8 @@
  * restatement of what the rollout computes: the foraging gridworld
  * (reset, observation, transition, reward, done), the shared actor-critic MLP,
  * the Philox4x32-10 inverse-CDF categorical sampler, generalised advantage
- * estimation, and the evaluation block (greedy or sampled episodes, returns).  It shares no code with the CUDA library and is used only by the
+ * estimation, the evaluation block (greedy or sampled episodes, returns) and
+ * the recurrent (gated-recurrent-unit) policy.  It shares no code with the CUDA library and is used only by the
  * tests, by the smoke check and by the benchmark's CPU-baseline leg.
  *
  * The technical report this follows describes the loop only in words
@@ -432,6 +433,130 @@ int orc_rollout(const orc_config_t *cfg, uint64_t seed, const float *params, int
     }
   }
   free(o);
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Recurrent policy (Section 2: every system comes in a feed-forward and a      */
+/* recurrent version; Section 4: the LBF and SMAX results are recurrent).  The  */
+/* report names no cell and no sizes.  Reading taken here: the observation is   */
+/* embedded by one dense ReLU layer, a gated recurrent unit (Cho et al. 2014)   */
+/* of the same width carries one hidden vector per agent, and the two heads     */
+/* read the new hidden vector:                                                  */
+/*   e  = relu(W1 x + b1)                                                       */
+/*   r  = sigma(Wir e + bir + Whr h + bhr)                                      */
+/*   z  = sigma(Wiz e + biz + Whz h + bhz)                                      */
+/*   n  = tanh(Win e + bin + r * (Whn h + bhn))                                 */
+/*   h' = (1 - z) * n + z * h                                                   */
+/*   logits = Wa h' + ba,  value = Wv h' + bv.                                  */
+/* Parameter order: W1[H][D] b1[H]  Wih[3H][H] bih[3H]  Whh[3H][H] bhh[3H]      */
+/* Wa[6][H] ba[6]  Wv[1][H] bv[1]; the three H-row blocks of Wih/Whh/bih/bhh are */
+/* the gates r, z, n in that order.  h is zero at the start of every episode:   */
+/* after a step that ends the episode every agent of that environment goes on   */
+/* with h = 0.  With emulate_bf16 the operands of every product (x, e, h and    */
+/* the weights) are rounded to bf16, the gate arithmetic is not, and the        */
+/* carried state itself is the bf16-rounded h' (it is what the next step        */
+/* multiplies and blends).                                                      */
+/* ------------------------------------------------------------------------- */
+int64_t orc_rec_params_count(const orc_config_t *cfg) {
+  const int64_t D = orc_obs_dim(cfg), H = cfg->hidden;
+  return H * D + H + 2 * (3 * H * H + 3 * H) + ORC_N_ACTIONS * H + ORC_N_ACTIONS + H + 1;
+}
+
+static double sigmoid(double v) { return 1.0 / (1.0 + exp(-v)); }
+
+/* One environment, one step: obs [N][D] binary32, h [N][H] in and out (double). */
+void orc_rec_forward_env(const orc_config_t *cfg, const float *params, const float *obs, double *h,
+                         int emulate_bf16, double *logits, double *values) {
+  const int D = orc_obs_dim(cfg), H = cfg->hidden, N = cfg->n_agents;
+  const float *W1 = params, *b1 = W1 + (size_t)H * D;
+  const float *Wih = b1 + H, *bih = Wih + (size_t)3 * H * H;
+  const float *Whh = bih + 3 * H, *bhh = Whh + (size_t)3 * H * H;
+  const float *Wa = bhh + 3 * H, *ba = Wa + (size_t)ORC_N_ACTIONS * H, *Wv = ba + ORC_N_ACTIONS, *bv = Wv + H;
+  double *x = (double *)malloc(sizeof(double) * (size_t)D);
+  double *e = (double *)malloc(sizeof(double) * (size_t)H);
+  double *gi = (double *)malloc(sizeof(double) * (size_t)3 * H);
+  double *gh = (double *)malloc(sizeof(double) * (size_t)3 * H);
+  for (int n = 0; n < N; ++n) {
+    double *hn = h + (size_t)n * H;
+    round_vec(hn, H, emulate_bf16); /* a carried state already is a bf16 number; any other input becomes one */
+    for (int k = 0; k < D; ++k) x[k] = q(obs[(size_t)n * D + k], emulate_bf16);
+    dense(W1, b1, x, D, H, 1, emulate_bf16, e);
+    round_vec(e, H, emulate_bf16);
+    dense(Wih, bih, e, H, 3 * H, 0, emulate_bf16, gi);   /* input part of the three gates, biases included  */
+    dense(Whh, bhh, hn, H, 3 * H, 0, emulate_bf16, gh);  /* hidden part of the three gates, biases included */
+    for (int j = 0; j < H; ++j) {
+      const double r = sigmoid(gi[j] + gh[j]);
+      const double z = sigmoid(gi[H + j] + gh[H + j]);
+      const double c = tanh(gi[2 * H + j] + r * gh[2 * H + j]);
+      hn[j] = (1.0 - z) * c + z * hn[j];
+    }
+    round_vec(hn, H, emulate_bf16);
+    dense(Wa, ba, hn, H, ORC_N_ACTIONS, 0, emulate_bf16, logits + (size_t)n * ORC_N_ACTIONS);
+    dense(Wv, bv, hn, H, 1, 0, emulate_bf16, values + n);
+  }
+  free(x); free(e); free(gi); free(gh);
+}
+
+/* The rollout loop of orc_rollout with the recurrent policy.  `hidden` is        */
+/* [n_local][N][H] (double): the state every listed environment's agents enter    */
+/* the first step with; on return, the state they would enter step T with.  The   */
+/* bootstrap row values[T] is the value head on the hidden vector after one more  */
+/* cell update on the observation that follows the last step; that update is not  */
+/* kept (the next call repeats it on the same observation and state).             */
+int orc_rollout_rec(const orc_config_t *cfg, uint64_t seed, const float *params, int emulate_bf16,
+                    int32_t n_local, const int32_t *env_ids, int32_t T, uint32_t t_global0,
+                    orc_env_state_t *states, double *hidden, const int32_t *forced_actions, float *obs,
+                    int32_t *actions, int32_t *own_actions, double *logp, double *values, float *rewards,
+                    uint8_t *dones, double *logits, double *margin) {
+  const int N = cfg->n_agents, D = orc_obs_dim(cfg), H = cfg->hidden;
+  if (N > ORC_MAX_AGENTS || cfg->n_food > ORC_MAX_FOOD || !params || !hidden) return -1;
+  float *o = (float *)malloc(sizeof(float) * (size_t)N * D);
+  double *hb = (double *)malloc(sizeof(double) * (size_t)N * H);
+  double lg[ORC_MAX_AGENTS * ORC_N_ACTIONS], val[ORC_MAX_AGENTS], lp[ORC_N_ACTIONS];
+  int32_t act[ORC_MAX_AGENTS];
+  for (int i = 0; i < n_local; ++i) {
+    const int32_t env = env_ids[i];
+    orc_env_state_t *s = &states[i];
+    double *h = hidden + (size_t)i * N * H;
+    for (int t = 0; t <= T; ++t) {
+      const size_t row0 = ((size_t)t * n_local + (size_t)i) * N;
+      for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
+      if (t < T && obs) memcpy(obs + row0 * D, o, sizeof(float) * (size_t)N * D);
+      if (t == T) {  /* bootstrap: on a copy of the state */
+        memcpy(hb, h, sizeof(double) * (size_t)N * H);
+        orc_rec_forward_env(cfg, params, o, hb, emulate_bf16, lg, val);
+        if (values) for (int n = 0; n < N; ++n) values[row0 + n] = val[n];
+        break;
+      }
+      orc_rec_forward_env(cfg, params, o, h, emulate_bf16, lg, val);
+      if (values) for (int n = 0; n < N; ++n) values[row0 + n] = val[n];
+      for (int n = 0; n < N; ++n) {
+        int32_t own = 0;
+        double mg;
+        const float u = orc_action_uniform(seed, t_global0 + (uint32_t)t, (uint32_t)env, (uint32_t)n);
+        orc_sample(lg + n * ORC_N_ACTIONS, u, &own, lp, &mg);
+        if (own_actions) own_actions[row0 + n] = own;
+        if (margin) margin[row0 + n] = mg;
+        if (logits)
+          for (int k = 0; k < ORC_N_ACTIONS; ++k) logits[(row0 + n) * ORC_N_ACTIONS + k] = lg[n * ORC_N_ACTIONS + k];
+        act[n] = forced_actions ? forced_actions[row0 + n] : own;
+        if (act[n] < 0 || act[n] >= ORC_N_ACTIONS) { free(o); free(hb); return -1; }
+        if (actions) actions[row0 + n] = act[n];
+        if (logp) logp[row0 + n] = lp[act[n]];
+      }
+      float reward;
+      uint8_t done;
+      orc_env_step(cfg, s, act, &reward, &done);
+      if (rewards) for (int n = 0; n < N; ++n) rewards[row0 + n] = reward;
+      if (dones) dones[(size_t)t * n_local + i] = done;
+      if (done) {
+        orc_env_reset(cfg, seed, env, s->episode + 1, s);
+        for (int k = 0; k < N * H; ++k) h[k] = 0.0;  /* a new episode starts without memory */
+      }
+    }
+  }
+  free(o); free(hb);
   return 0;
 }
 

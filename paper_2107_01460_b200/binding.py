@@ -117,10 +117,13 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
 
 
 def update_on_tensor_cores(cfg: mava_config_t) -> bool:
-    """Whether mava_ppo_grad takes the bf16 tensor-core kernels for a handle of this configuration (the shapes
-    they serve: shared torso, H <= 128, D <= 80)."""
-    return (cfg.precision == MAVA_PRECISION_BF16 and not cfg.flags & MAVA_FLAG_UPDATE_FP32 and
-            cfg.net_kind == MAVA_NET_SHARED_TORSO and cfg.hidden <= 128 and 77 + cfg.n_agents <= 80)
+    """Whether mava_ppo_grad takes the bf16 tensor-core kernels for a handle of this configuration: the shared-torso
+    shapes with H <= 128 and D <= 80 (one fused kernel), and H = 256 with 64 < D <= 96 (row kernel + weight kernel; with
+    a centralised critic only the actor net, the critic net stays on the fp32 kernel)."""
+    if cfg.precision != MAVA_PRECISION_BF16 or cfg.flags & MAVA_FLAG_UPDATE_FP32:
+        return False
+    D = 77 + cfg.n_agents
+    return (cfg.net_kind == MAVA_NET_SHARED_TORSO and cfg.hidden <= 128 and D <= 80) or (cfg.hidden == 256 and 64 < D <= 96)
 
 
 def ppo_defaults() -> mava_ppo_hyper_t:

@@ -461,6 +461,7 @@ void mava_rollout_destroy(mava_rollout_t *h) {
   cudaFree(h->d_critic);
   cudaFree(h->d_obs_last);
   cudaFree(h->d_upd);
+  cudaFree(h->d_upd_stage);
   if (h->copy_ready) {
     cudaStreamSynchronize(h->copy_stream);
     for (int i = 0; i <= kCollectChunks; ++i) cudaEventDestroy(h->chunk_done[i]);

@@ -110,6 +110,8 @@ struct mava_rollout {
   float *d_obs_last;   //   and the observations after the last step [E][N][D]
   void *d_upd;         // scratch of the update block (made on its first call)
   size_t upd_bytes;
+  void *d_upd_stage;   // staging buffer of the H = 256 tensor-core update (made on its first call)
+  size_t upd_stage_bytes;
   uint32_t t_global;
   int32_t last_T;
   int64_t launches;

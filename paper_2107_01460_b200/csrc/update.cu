@@ -373,9 +373,13 @@ size_t upd_smem_bytes(int Din, int H) {
 struct UpdScratch {
   double *stats, *stat_part, *term_part;
   float *wt, *partial;
-  unsigned char *image;  // weight image of the tensor-core path
+  unsigned char *image;  // weight image of the tensor-core paths
   int slices;
 };
+size_t image_room() {
+  const size_t a = ppo_tc_image_bytes(), b = ppo_tc256_image_bytes();
+  return ((a > b ? a : b) + 255) / 256 * 256;
+}
 UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
   unsigned char *p = static_cast<unsigned char *>(h->d_upd);
   UpdScratch s{};
@@ -383,11 +387,13 @@ UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
   s.stat_part = reinterpret_cast<double *>(p); p += sizeof(double) * 2 * kStatBlocks;
   s.term_part = reinterpret_cast<double *>(p); p += sizeof(double) * 3 * 8 * slices;
   s.wt = reinterpret_cast<float *>(p); p += sizeof(float) * ((n_params + 3) / 4 * 4);
-  s.image = p; p += (ppo_tc_image_bytes() + 255) / 256 * 256;
+  s.image = p; p += image_room();
   s.partial = reinterpret_cast<float *>(p);
   s.slices = slices;
   return s;
 }
+
+constexpr int kChunkTiles = 4096;  // rows of a chunk of the H = 256 tensor-core path: 524 288 (1.2 GB of staging)
 
 }  // namespace
 
@@ -395,16 +401,29 @@ UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
 bool update_takes_tensor_cores(const mava_config_t &cfg, int D) {
   return cfg.precision == MAVA_PRECISION_BF16 && (cfg.flags & MAVA_FLAG_UPDATE_FP32) == 0 && ppo_tc_supported(cfg, D);
 }
+bool update_takes_tensor_cores_256(const mava_config_t &cfg, int D) {
+  return cfg.precision == MAVA_PRECISION_BF16 && (cfg.flags & MAVA_FLAG_UPDATE_FP32) == 0 && ppo_tc256_supported(cfg, D);
+}
 
 cudaError_t ensure_update_scratch(mava_rollout *h, size_t n_params, int slices) {
   const size_t bytes = 64 + sizeof(double) * 2 * kStatBlocks + sizeof(double) * 3 * 8 * slices + sizeof(float) * ((n_params + 3) / 4 * 4) +
-                       (ppo_tc_image_bytes() + 255) / 256 * 256 + sizeof(float) * n_params * slices;
+                       image_room() + sizeof(float) * n_params * slices;
   if (h->d_upd && h->upd_bytes >= bytes) return cudaSuccess;
   cudaFree(h->d_upd);
   h->d_upd = nullptr;
   h->upd_bytes = 0;
   cudaError_t err = cudaMalloc(&h->d_upd, bytes);
   if (err == cudaSuccess) h->upd_bytes = bytes;
+  return err;
+}
+
+cudaError_t ensure_update_staging(mava_rollout *h, size_t bytes) {
+  if (h->d_upd_stage && h->upd_stage_bytes >= bytes) return cudaSuccess;
+  cudaFree(h->d_upd_stage);
+  h->d_upd_stage = nullptr;
+  h->upd_stage_bytes = 0;
+  cudaError_t err = cudaMalloc(&h->d_upd_stage, bytes);
+  if (err == cudaSuccess) h->upd_stage_bytes = bytes;
   return err;
 }
 
@@ -419,31 +438,36 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   if (err != cudaSuccess) return err;
   const int n_env = env_ids_dev ? n_ids : E;  // environments in the minibatch
   const long long R = static_cast<long long>(T) * n_env * N, S = static_cast<long long>(T) * n_env;
+  const long long tiles128 = (R + 127) / 128;
+  const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
+  const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
+  cudaStream_t st = h->stream;
+  UpdRows rows{};
+  rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
+  rows.env_ids = env_ids_dev; rows.n_ids = n_env; rows.E = E; rows.per_env = N;
+  if (!central) { rows.value_old = h->buf.values; rows.ret = h->buf.ret; rows.vstride = 1; }
+
   if (update_takes_tensor_cores(cfg, D)) {
-    // one CTA (= one gradient slice) per SM over tiles of 128 rows
-    const long long tiles128 = (R + 127) / 128;
+    // H <= 128: one CTA (= one gradient slice) per SM over tiles of 128 rows
     const int slices = static_cast<int>(tiles128 < sms ? tiles128 : sms);
     err = ensure_update_scratch(h, P, slices);
     if (err != cudaSuccess) return err;
     const UpdScratch sc = carve(h, P, slices);
-    cudaStream_t st = h->stream;
-    UpdRows rows{};
-    rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
-    rows.env_ids = env_ids_dev; rows.n_ids = n_env; rows.E = E; rows.per_env = N;
-    rows.value_old = h->buf.values; rows.ret = h->buf.ret; rows.vstride = 1;
     stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part, rows);
     stat_final_kernel<<<1, 32, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
     h->launches += 2;
-    const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
     err = launch_ppo_net_tc(h, params_dev, L, rows, hp, sc.stats, sc.image, sc.partial, P, sc.term_part, slices);
     if (err != cudaSuccess) return err;
     reduce_partials_kernel<<<128, 256, 0, st>>>(sc.partial, P, slices, grad_dev, sc.term_part, 8 * slices, R, R, hp, terms_dev);
     h->launches += 1;
     return cudaGetLastError();
   }
+
+  // H = 256 on the tensor cores: the actor / shared-torso net; a centralised critic stays on the fp32 kernel below
+  const bool tc256 = update_takes_tensor_cores_256(cfg, D);
+  const int slices_tc = tc256 ? static_cast<int>(tiles128 < sms ? (tiles128 < 2 ? 2 : tiles128) : sms) : 0;
   const long long tiles = (R + kUpdRows - 1) / kUpdRows;
-  // as many CTAs (= gradient slices) as are resident at once with the larger of the two nets' shared-memory needs
-  const bool central = cfg.net_kind == MAVA_NET_CENTRAL_CRITIC;
+  // fp32 kernel: as many CTAs (= gradient slices) as are resident at once with the larger of the two nets' shared-memory needs
   const int joint = N * D;
   const size_t smem_max = upd_smem_bytes(central ? joint : D, H);
   using KernelT = void (*)(UpdNet, UpdRows, UpdHyper, const double *, float *, size_t, double *, int *);
@@ -455,33 +479,34 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, H, smem_max);
   if (err != cudaSuccess) return err;
   if (per_sm < 1) per_sm = 1;
-  const int slices = static_cast<int>(tiles < static_cast<long long>(sms) * per_sm ? tiles : static_cast<long long>(sms) * per_sm);
+  const int slices_fp32 = static_cast<int>(tiles < static_cast<long long>(sms) * per_sm ? tiles : static_cast<long long>(sms) * per_sm);
+  const int slices = slices_fp32 > slices_tc ? slices_fp32 : slices_tc;
   err = ensure_update_scratch(h, P, slices);
   if (err != cudaSuccess) return err;
+  const int chunk_tiles = static_cast<int>(tiles128 < kChunkTiles ? tiles128 : kChunkTiles);
+  if (tc256) {
+    err = ensure_update_staging(h, ppo_tc256_staging_bytes(chunk_tiles));
+    if (err != cudaSuccess) return err;
+  }
   const UpdScratch sc = carve(h, P, slices);
-  cudaStream_t st = h->stream;
-  // transposed copies of the hidden layers' weights, in the parameters' own order
+  // transposed copies of the hidden layers' weights, in the parameters' own order (fp32 kernel only)
   auto tr = [&](size_t off, int out, int in) {
     transpose_kernel<<<64, 256, 0, st>>>(params_dev + off, sc.wt + off, out, in);
     h->launches += 1;
   };
-  tr(L.W1, H, D); tr(L.W2, H, H);
+  if (!tc256) { tr(L.W1, H, D); tr(L.W2, H, H); }
   if (central) { tr(L.C1, H, joint); tr(L.C2, H, H); }
-  UpdRows rows{};
-  rows.x = h->buf.obs; rows.actions = h->buf.actions; rows.logp_old = h->buf.logp; rows.adv = h->buf.adv; rows.n = R;
-  rows.env_ids = env_ids_dev; rows.n_ids = n_env; rows.E = E; rows.per_env = N;
   stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part, rows);
   stat_final_kernel<<<1, 32, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
   h->launches += 2;
   err = cudaMemsetAsync(sc.term_part, 0, sizeof(double) * 3 * 8 * slices, st);
   if (err == cudaSuccess) err = cudaMemsetAsync(sc.partial, 0, sizeof(float) * P * slices, st);
   if (err != cudaSuccess) return err;
-  const UpdHyper hp{hyper.clip_eps, hyper.ent_coef, hyper.vf_coef};
   auto run_net = [&](const UpdNet &net, const UpdRows &rows) {
     const size_t smem = upd_smem_bytes(net.Din, net.H);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    kern<<<slices, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part, h->d_status);
+    kern<<<slices_fp32, net.H, smem, st>>>(net, rows, hp, sc.stats, sc.partial, P, sc.term_part, h->d_status);
     h->launches += 1;
     return cudaGetLastError();
   };
@@ -493,10 +518,13 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   actor.oW1 = L.W1; actor.ob1 = L.b1; actor.oW2 = L.W2; actor.ob2 = L.b2; actor.oWa = L.Wa; actor.oba = L.ba;
   if (!central) {
     actor.Wv = params_dev + L.Wv; actor.bv = params_dev + L.bv; actor.oWv = L.Wv; actor.obv = L.bv;
-    rows.value_old = h->buf.values; rows.ret = h->buf.ret; rows.vstride = 1;
-    err = run_net(actor, rows);
+    err = tc256 ? launch_ppo_net_tc256(h, params_dev, L, rows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P, sc.term_part,
+                                       slices_tc, true)
+                : run_net(actor, rows);
   } else {
-    err = run_net(actor, rows);
+    err = tc256 ? launch_ppo_net_tc256(h, params_dev, L, rows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P, sc.term_part,
+                                       slices_tc, false)
+                : run_net(actor, rows);
     if (err != cudaSuccess) return err;
     UpdNet critic{};
     critic.W1 = params_dev + L.C1; critic.b1 = params_dev + L.c1; critic.W2 = params_dev + L.C2; critic.b2 = params_dev + L.c2;

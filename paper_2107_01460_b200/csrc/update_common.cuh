@@ -47,4 +47,15 @@ size_t ppo_tc_image_bytes();
 cudaError_t launch_ppo_net_tc(mava_rollout *h, const float *params_dev, const ParamLayout &L, const UpdRows &rows, const UpdHyper &hp,
                               const double *adv_stats, void *image, float *partial, size_t n_params, double *term_partial, int slices);
 
+
+// Tensor-core path for H = 256 (update_tc256.cu): the actor / shared-torso net with 64 < D <= 96, a chunk of
+// `chunk_tiles` 128-row tiles at a time through `staging` (ppo_tc256_staging_bytes(chunk_tiles) bytes).  Adds into the
+// slices of `partial` and into `term_partial` (both zeroed by the caller); needs slices >= 2.
+bool ppo_tc256_supported(const mava_config_t &cfg, int D);
+size_t ppo_tc256_image_bytes();
+size_t ppo_tc256_staging_bytes(int chunk_tiles);
+cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const ParamLayout &L, const UpdRows &rows, const UpdHyper &hp,
+                                 const double *adv_stats, void *image, void *staging, int chunk_tiles, float *partial, size_t n_params,
+                                 double *term_partial, int slices, bool has_value);
+
 }  // namespace mava

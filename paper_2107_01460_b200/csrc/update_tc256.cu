@@ -1,0 +1,544 @@
+// Update block on the tensor cores for hidden width 256 (sm_100a, tcgen05): the actor / shared-torso net of the two
+// largest shapes.  The weight gradient of the second layer alone (256 x 256 fp32) fills all 512 columns of an SM's tensor
+// memory, and the weights (184 KB in bf16) leave no room for bf16 activation tiles in shared memory, so the work is cut in
+// two kernels that meet in a staging buffer (a chunk of rows at a time, so that the buffer stays small):
+//   row kernel     per 128-row tile: forward and backward through the layers with the activations kept in tensor memory
+//                  as the A operand of the next product (as the rollout does), the loss and its per-row derivatives in
+//                  fp32; every bf16 matrix that a weight gradient needs (x, h1, h2, d z2, d z1, the derivatives of the
+//                  heads) is written to the staging buffer as tiles in the canonical core-matrix layout [row][feature];
+//   weight kernel  streams those tiles back with bulk copies and reads them with the row index as K (MN-major operands,
+//                  see update_tc.cu): d W2 += d z2^T . h1 by one group of CTAs (four 128 x 128 accumulators = all of
+//                  tensor memory), d W1 += d z1^T . x and d Wh^T += h2^T . dhead by another; the bias gradients are column
+//                  sums of the same tiles by the plain ALUs.  Every CTA adds its accumulators into its own slice of the
+//                  partial-gradient array, which update.cu's reducer sums in slice order: same bytes on every call.
+// Rounding points are those of the bf16-operand mode of the float64 oracle.  Every mbarrier wait is bounded.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "layout.h"
+#include "tc_common.cuh"
+#include "update_common.cuh"
+
+namespace mava {
+namespace {
+
+constexpr int kR = 128;       // rows per tile
+constexpr int kH = 256;       // hidden width
+constexpr int kK1 = 96;       // input width, padded (D = 81, 85)
+constexpr int kHeads = 16;
+constexpr int kThreads = 256;
+
+constexpr uint32_t kImgW1 = 0, kImgW2 = kImgW1 + kH * kK1 * 2, kImgWh = kImgW2 + kH * kH * 2;
+constexpr uint32_t kImgB1 = kImgWh + kHeads * kH * 2, kImgB2 = kImgB1 + kH * 4, kImgBh = kImgB2 + kH * 4;
+constexpr uint32_t kImgBytes = kImgBh + 32;
+static_assert(kImgBytes % 16 == 0, "bulk copies");
+
+// staging buffer, per tile: x [128][96]; h1, h2, d z2, d z1 as two unit halves [128][128] each; dhead [128][16]
+constexpr size_t kStX = 0, kStXBytes = kR * kK1 * 2;
+constexpr size_t kHalfBytes = kR * 128 * 2, kActBytes = 2 * kHalfBytes;
+constexpr size_t kStH1 = kStX + kStXBytes, kStH2 = kStH1 + kActBytes, kStDz2 = kStH2 + kActBytes, kStDz1 = kStDz2 + kActBytes;
+constexpr size_t kStDh = kStDz1 + kActBytes, kStDhBytes = kR * kHeads * 2;
+constexpr size_t kStTile = kStDh + kStDhBytes;  // 290 816 bytes
+
+constexpr uint32_t kColAcc = 0, kColHid = 256, kColHead = 384, kTmemRow = 512;
+
+struct RowSmem {
+  alignas(128) unsigned char img[(kImgBytes + 127) / 128 * 128];
+  alignas(128) unsigned char x[kR * kK1 * 2];
+  alignas(128) unsigned char dhead[kR * kHeads * 2];
+  long long rmap[kR];
+  float red[4][8];
+  alignas(8) uint64_t bar_load, bar_mma;
+  uint32_t tmem_base;
+};
+
+__global__ void prep_upd256_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, ParamLayout L, int D, int has_value) {
+  auto bf = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(image + off); };
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  for (int i = tid; i < kH * kK1; i += nth) {
+    const int n = i / kK1, k = i - n * kK1;
+    bf(kImgW1)[canon_offset(n, k, kK1) / 2] = __float2bfloat16_rn(k < D ? params[L.W1 + static_cast<size_t>(n) * D + k] : 0.0f);
+  }
+  for (int i = tid; i < kH * kH; i += nth) {
+    const int n = i / kH, k = i - n * kH;
+    bf(kImgW2)[canon_offset(n, k, kH) / 2] = __float2bfloat16_rn(params[L.W2 + static_cast<size_t>(n) * kH + k]);
+  }
+  for (int i = tid; i < kHeads * kH; i += nth) {
+    const int n = i / kH, k = i - n * kH;
+    float v = 0.0f;
+    if (n < kActions) v = params[L.Wa + static_cast<size_t>(n) * kH + k];
+    else if (n == kActions && has_value) v = params[L.Wv + k];
+    bf(kImgWh)[canon_offset(n, k, kH) / 2] = __float2bfloat16_rn(v);
+  }
+  float *b1 = reinterpret_cast<float *>(image + kImgB1), *b2 = reinterpret_cast<float *>(image + kImgB2),
+        *bh = reinterpret_cast<float *>(image + kImgBh);
+  for (int i = tid; i < kH; i += nth) { b1[i] = params[L.b1 + i]; b2[i] = params[L.b2 + i]; }
+  if (tid < 8) bh[tid] = tid < kActions ? params[L.ba + tid] : ((tid == kActions && has_value) ? params[L.bv] : 0.0f);
+}
+
+__device__ __forceinline__ uint64_t desc_k(uint32_t tile, int C, int k) { return smem_desc(tile + k * 256, 128, C * 16); }
+__device__ __forceinline__ uint64_t desc_mn(uint32_t tile, int C, int k) { return smem_desc(tile + k * 2 * C * 16, C * 16, 128); }
+constexpr uint32_t kAmn = 1u << 15, kBmn = 1u << 16;
+
+__device__ __forceinline__ void stg_v4(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+struct HeadOffsets { size_t ba, bv; };
+
+// ---- row kernel ------------------------------------------------------------------------------------------------------
+// Tiles [tile0, tile0 + n_tiles) of the minibatch; tile t's staging record is number t - tile0.
+__global__ void __launch_bounds__(kThreads, 1)
+ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyper hp, const double *__restrict__ adv_stats,
+                   unsigned char *__restrict__ staging, long long tile0, int n_tiles, float *__restrict__ partial, size_t n_params,
+                   double *__restrict__ term_partial, int *status, HeadOffsets off, int D, int has_value) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  RowSmem &sm = *reinterpret_cast<RowSmem *>(smem_raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row = tid & (kR - 1), half = tid >> 7;
+  const uint32_t bar_load = smem_u32(&sm.bar_load), bar_mma = smem_u32(&sm.bar_mma);
+  if (tid == 0) {
+    mbar_init(bar_load, 1); mbar_init(bar_mma, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemRow) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int i = tid; i < static_cast<int>(sizeof(sm.x) / 16); i += kThreads) sts_zero16(smem_u32(sm.x) + 16u * i);
+  for (int i = tid; i < static_cast<int>(sizeof(sm.dhead) / 16); i += kThreads) sts_zero16(smem_u32(sm.dhead) + 16u * i);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (tid == 0) {
+    mbar_expect_tx(bar_load, kImgBytes);
+    constexpr uint32_t kChunk = 16384;
+    for (uint32_t o = 0; o < kImgBytes; o += kChunk) bulk_load(smem_u32(sm.img + o), image + o, min(kChunk, kImgBytes - o), bar_load);
+  }
+  bool timed_out = !mbar_wait(bar_load, 0);
+  timed_out = __syncthreads_or(timed_out) != 0;
+
+  const uint32_t tmem = sm.tmem_base;
+  const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+  const uint32_t w1 = smem_u32(sm.img + kImgW1), w2 = smem_u32(sm.img + kImgW2), wh = smem_u32(sm.img + kImgWh);
+  const uint32_t xt = smem_u32(sm.x), dht = smem_u32(sm.dhead);
+  const float *b1 = reinterpret_cast<const float *>(sm.img + kImgB1), *b2 = reinterpret_cast<const float *>(sm.img + kImgB2),
+              *bh = reinterpret_cast<const float *>(sm.img + kImgBh);
+  const float mean = static_cast<float>(adv_stats[0]);
+  const float inv_std = 1.0f / (static_cast<float>(adv_stats[1]) + 1e-8f);
+  const float inv_n = 1.0f / static_cast<float>(rows.n);
+  const int my_tiles = static_cast<int>(blockIdx.x) < n_tiles ? (n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
+
+  uint32_t ph = 0;
+  double t_actor = 0.0, t_ent = 0.0, t_value = 0.0;
+  float gbh = 0.0f;
+  // this thread's 16-byte pieces of a staged activation: unit half `half`, its own row
+  const size_t act_row_off = static_cast<size_t>(half) * kHalfBytes + static_cast<size_t>((row >> 3) * 2048 + (row & 7) * 16);
+
+  // 128 accumulator columns of this thread (+ bias, ReLU) -> bf16 -> tensor memory (A operand of the next product) and
+  // the staged tile; gate bits out
+  auto fwd_epilogue = [&](const float *bias, unsigned char *stage_act, uint32_t gate[4]) {
+#pragma unroll
+    for (int c0 = 0; c0 < 128; c0 += 32) {
+      uint32_t ra[32], pk[16];
+      tmem_ld32_nowait(tmem + kColAcc + lane_off + 128u * half + c0, ra);
+      tmem_ld_wait();
+      uint32_t g = 0;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float v0 = __uint_as_float(ra[2 * e]) + bias[128 * half + c0 + 2 * e];
+        const float v1 = __uint_as_float(ra[2 * e + 1]) + bias[128 * half + c0 + 2 * e + 1];
+        g |= (static_cast<uint32_t>(v0 > 0.0f) << (2 * e)) | (static_cast<uint32_t>(v1 > 0.0f) << (2 * e + 1));
+        pk[e] = relu_pack_bf16(__float_as_uint(v0), __float_as_uint(v1));
+      }
+      gate[c0 / 32] = g;
+      tmem_st16(tmem + kColHid + lane_off + static_cast<uint32_t>((128 * half + c0) / 2), pk);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        stg_v4(stage_act + act_row_off + static_cast<size_t>((c0 / 8 + q) * 128), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+    }
+    tmem_st_wait();
+  };
+  auto bwd_epilogue = [&](const uint32_t gate[4], unsigned char *stage_act, bool to_tmem) {
+#pragma unroll
+    for (int c0 = 0; c0 < 128; c0 += 32) {
+      uint32_t ra[32], pk[16];
+      tmem_ld32_nowait(tmem + kColAcc + lane_off + 128u * half + c0, ra);
+      tmem_ld_wait();
+      const uint32_t g = gate[c0 / 32];
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        pk[e] = pack_bf16(((g >> (2 * e)) & 1u) ? __uint_as_float(ra[2 * e]) : 0.0f, ((g >> (2 * e + 1)) & 1u) ? __uint_as_float(ra[2 * e + 1]) : 0.0f);
+      if (to_tmem) tmem_st16(tmem + kColHid + lane_off + static_cast<uint32_t>((128 * half + c0) / 2), pk);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        stg_v4(stage_act + act_row_off + static_cast<size_t>((c0 / 8 + q) * 128), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+    }
+    if (to_tmem) tmem_st_wait();
+  };
+
+  for (int i = 0; i < my_tiles && !timed_out; ++i) {
+    const int lt = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);  // tile inside the chunk
+    const long long row0 = (tile0 + lt) * kR;
+    unsigned char *st = staging + static_cast<size_t>(lt) * kStTile;
+    const int n_valid = static_cast<int>(min(static_cast<long long>(kR), rows.n - row0));
+    const long long my_row = row < n_valid ? real_row(rows, row0 + row) : -1;
+    int action = 0;
+    float logp_old = 0.0f, adv = 0.0f, v_old = 0.0f, ret = 0.0f;
+    if (half == 0) {
+      sm.rmap[row] = my_row;
+      if (row < n_valid && my_row < 0) atomicExch(status, kStatusBadIndex);
+      if (my_row >= 0) {
+        action = rows.actions[my_row]; logp_old = rows.logp_old[my_row]; adv = rows.adv[my_row];
+        if (has_value) { v_old = rows.value_old[my_row * rows.vstride]; ret = rows.ret[my_row * rows.vstride]; }
+      }
+    }
+    if (tid == 0) bulk_store_wait_read();  // the copies of the previous tile's x and dhead tiles have read them
+    tc_fence_before();
+    __syncthreads();
+    // ---- the tile's rows as bf16 into x: a warp per row, consecutive lanes consecutive features
+    {
+      constexpr int G = 8;
+      for (int g0 = warp; g0 < kR; g0 += 8 * G) {
+        float v[G][3];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const long long src = sm.rmap[g0 + 8 * g];
+#pragma unroll
+          for (int q = 0; q < 3; ++q) {
+            const int k = lane + 32 * q;
+            v[g][q] = (k < D && src >= 0) ? rows.x[src * D + k] : 0.0f;
+          }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+#pragma unroll
+          for (int q = 0; q < 3; ++q) {
+            const int k = lane + 32 * q;
+            if (k < D) sts_u16(xt + canon_offset(g0 + 8 * g, k, kK1), bf16_bits(v[g][q]));
+          }
+      }
+    }
+    fence_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      bulk_store(st + kStX, xt, static_cast<uint32_t>(kStXBytes));
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < kK1 / 16; ++k) mma_bf16(tmem + kColAcc, desc_k(xt, kK1, k), desc_k(w1, kK1, k), instr_desc(kR, kH), k > 0);
+      mma_commit(bar_mma);
+    }
+    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    tc_fence_after();
+    uint32_t gate1[4], gate2[4];
+    fwd_epilogue(b1, st + kStH1, gate1);
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < kH / 16; ++k) mma_bf16_ts(tmem + kColAcc, tmem + kColHid + k * 8, desc_k(w2, kH, k), instr_desc(kR, kH), k > 0);
+      mma_commit(bar_mma);
+    }
+    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    tc_fence_after();
+    fwd_epilogue(b2, st + kStH2, gate2);
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < kH / 16; ++k) mma_bf16_ts(tmem + kColHead, tmem + kColHid + k * 8, desc_k(wh, kH, k), instr_desc(kR, kHeads), k > 0);
+      mma_commit(bar_mma);
+    }
+    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    tc_fence_after();
+    if (half == 0) {
+      float hv[16], d[8];
+      tmem_ld16(tmem + kColHead + lane_off, hv);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) d[k] = 0.0f;
+      if (my_row >= 0) {
+        float l[kActions], m = -INFINITY, sum = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kActions; ++k) { l[k] = hv[k] + bh[k]; m = fmaxf(m, l[k]); }
+#pragma unroll
+        for (int k = 0; k < kActions; ++k) sum += expf(l[k] - m);
+        const float lse = m + logf(sum);
+        float ent = 0.0f, p[kActions], lp[kActions], lpa = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kActions; ++k) {
+          lp[k] = l[k] - lse; p[k] = expf(lp[k]); ent -= p[k] * lp[k];
+          if (k == action) lpa = lp[k];
+        }
+        const float rho = expf(lpa - logp_old);
+        const float ahat = (adv - mean) * inv_std;
+        const float clipped = fminf(fmaxf(rho, 1.0f - hp.clip_eps), 1.0f + hp.clip_eps);
+        const float s1 = rho * ahat, s2 = clipped * ahat;
+        const bool inside = rho >= 1.0f - hp.clip_eps && rho <= 1.0f + hp.clip_eps;
+        const float d_logp = (inside || s1 < s2) ? -s1 * inv_n : 0.0f;
+#pragma unroll
+        for (int k = 0; k < kActions; ++k)
+          d[k] = d_logp * ((k == action ? 1.0f : 0.0f) - p[k]) + hp.ent_coef * inv_n * p[k] * (lp[k] + ent);
+        t_actor += fminf(s1, s2);
+        t_ent += ent;
+        if (has_value) {
+          const float v = hv[kActions] + bh[kActions];
+          const float u = v - ret, uc = v_old + fminf(fmaxf(v - v_old, -hp.clip_eps), hp.clip_eps) - ret;
+          const bool in_range = fabsf(v - v_old) <= hp.clip_eps;
+          d[kActions] = (in_range || u * u > uc * uc) ? hp.vf_coef * u * inv_n : 0.0f;
+          t_value += 0.5 * fmaxf(u * u, uc * uc);
+        }
+      }
+      sts_v4(dht + static_cast<uint32_t>((row >> 3) * (kHeads * 16) + (row & 7) * 16), pack_bf16(d[0], d[1]), pack_bf16(d[2], d[3]),
+             pack_bf16(d[4], d[5]), pack_bf16(d[6], 0.0f));
+#pragma unroll
+      for (int k = 0; k <= kActions; ++k) {
+        float s = d[k];
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (lane == 0) sm.red[warp][k] = s;
+      }
+    }
+    fence_async_smem(); tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      bulk_store(st + kStDh, dht, static_cast<uint32_t>(kStDhBytes));
+      tc_fence_after();
+      mma_bf16(tmem + kColAcc, desc_k(dht, kHeads, 0), desc_mn(wh, kH, 0), instr_desc(kR, kH) | kBmn, 0);  // d h2 = dhead . Wh
+      mma_commit(bar_mma);
+    }
+    if (tid <= kActions) gbh += (sm.red[0][tid] + sm.red[1][tid]) + (sm.red[2][tid] + sm.red[3][tid]);
+    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    tc_fence_after();
+    bwd_epilogue(gate2, st + kStDz2, true);
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < kH / 16; ++k)  // d h1 = d z2 . W2
+        mma_bf16_ts(tmem + kColAcc, tmem + kColHid + k * 8, desc_mn(w2, kH, k), instr_desc(kR, kH) | kBmn, k > 0);
+      mma_commit(bar_mma);
+    }
+    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    tc_fence_after();
+    bwd_epilogue(gate1, st + kStDz1, false);
+    timed_out = __syncthreads_or(timed_out) != 0;
+  }
+  if (!timed_out) {
+    float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
+    if (tid < kActions) part[off.ba + tid] += gbh;
+    if (tid == kActions && has_value) part[off.bv] += gbh;
+  }
+  {
+    double s[3] = {t_actor, t_ent, t_value};
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+      for (int o = 16; o > 0; o >>= 1) s[k] += __shfl_xor_sync(0xFFFFFFFFu, s[k], o);
+    if (lane == 0) {
+      double *tp = term_partial + (static_cast<size_t>(blockIdx.x) * 8 + warp) * 3;
+      tp[0] += s[0]; tp[1] += s[1]; tp[2] += s[2];
+    }
+  }
+  if (tid == 0) {
+    if (timed_out) atomicExch(status, kStatusTimeout);
+    bulk_store_wait_all();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemRow) : "memory");
+  }
+}
+
+// ---- weight kernel ---------------------------------------------------------------------------------------------------
+// CTAs [0, n_w2) sum d W2 and d b2; the others d W1, d b1 and d Wh.  A CTA's work items are half tiles (64 rows) of
+// the tiles it owns; an item's operands come in by bulk copies into a ring of stages.
+constexpr int kHalfRows = 64;
+constexpr uint32_t kQ = 16384;                                // 64 rows of a [128][128] unit-half tile
+constexpr uint32_t kW2Stage = 4 * kQ, kW2Stages = 3;          // d z2 (two unit halves), h1 (two unit halves)
+constexpr uint32_t kXHalf = kHalfRows * kK1 * 2, kDhHalf = kHalfRows * kHeads * 2;
+constexpr uint32_t kW1Stage = 4 * kQ + kXHalf + kDhHalf, kW1Stages = 2;  // d z1, h2 (two unit halves each), x, dhead
+constexpr uint32_t kRingBytes = kW2Stage * kW2Stages > kW1Stage * kW1Stages ? kW2Stage * kW2Stages : kW1Stage * kW1Stages;
+
+struct WgtSmem {
+  alignas(128) unsigned char ring[kRingBytes];
+  alignas(8) uint64_t full[3], empty[3], done;
+  uint32_t tmem_base;
+};
+
+struct WgtOffsets { size_t W1, b1, W2, b2, Wa, Wv; };
+
+__global__ void __launch_bounds__(kThreads, 1)
+ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, int n_w2, float *__restrict__ partial, size_t n_params,
+                      int *status, WgtOffsets off, int D, int has_value) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  WgtSmem &sm = *reinterpret_cast<WgtSmem *>(smem_raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool role_w2 = static_cast<int>(blockIdx.x) < n_w2;
+  const int rank = role_w2 ? static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x) - n_w2;
+  const int peers = role_w2 ? n_w2 : static_cast<int>(gridDim.x) - n_w2;
+  const int S = role_w2 ? kW2Stages : kW1Stages;
+  const uint32_t stage_bytes = role_w2 ? kW2Stage : kW1Stage;
+  const uint32_t ring = smem_u32(sm.ring), full0 = smem_u32(&sm.full[0]), empty0 = smem_u32(&sm.empty[0]), done_bar = smem_u32(&sm.done);
+  constexpr uint32_t kCols = 512;
+  if (tid == 0) {
+    for (int s = 0; s < 3; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, 1 + kThreads / 32);  // the MMAs' commit and every warp's column sums
+    }
+    mbar_init(done_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+  const int my_tiles = rank < n_tiles ? (n_tiles - rank + peers - 1) / peers : 0;
+  const int n_items = 2 * my_tiles;
+  auto request = [&](int u) {  // thread 0: item u into stage u % S
+    const int lt = rank + (u >> 1) * peers, rh = u & 1;
+    const unsigned char *st = staging + static_cast<size_t>(lt) * kStTile;
+    const uint32_t dst = ring + static_cast<uint32_t>(u % S) * stage_bytes, bar = full0 + 8u * (u % S);
+    mbar_expect_tx(bar, stage_bytes);
+    const size_t a = role_w2 ? kStDz2 : kStDz1, b = role_w2 ? kStH1 : kStH2;
+    bulk_load(dst, st + a + static_cast<size_t>(rh) * kQ, kQ, bar);
+    bulk_load(dst + kQ, st + a + kHalfBytes + static_cast<size_t>(rh) * kQ, kQ, bar);
+    bulk_load(dst + 2 * kQ, st + b + static_cast<size_t>(rh) * kQ, kQ, bar);
+    bulk_load(dst + 3 * kQ, st + b + kHalfBytes + static_cast<size_t>(rh) * kQ, kQ, bar);
+    if (!role_w2) {
+      bulk_load(dst + 4 * kQ, st + kStX + static_cast<size_t>(rh) * kXHalf, kXHalf, bar);
+      bulk_load(dst + 4 * kQ + kXHalf, st + kStDh + static_cast<size_t>(rh) * kDhHalf, kDhHalf, bar);
+    }
+  };
+  bool timed_out = false;
+  int issued = 0;
+  if (tid == 0)
+    for (; issued < S && issued < n_items; ++issued) request(issued);
+  float db = 0.0f;  // thread j: bias gradient of out unit j (d b2 or d b1)
+  const uint32_t my_col = static_cast<uint32_t>(tid >> 7) * kQ + static_cast<uint32_t>(((tid & 127) >> 3) * 128 + (tid & 7) * 2);
+#pragma unroll 1
+  for (int u = 0; u < n_items; ++u) {
+    const int s = u % S;
+    const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
+    timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
+    if (__syncthreads_or(timed_out)) { timed_out = true; break; }
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t keep = u > 0 ? 1u : 0u;
+      if (role_w2) {  // d W2 [out half a][in half b] += d z2[:, a]^T . h1[:, b] over the item's 64 rows
+#pragma unroll
+        for (int k = 0; k < kHalfRows / 16; ++k)
+#pragma unroll
+          for (int ab = 0; ab < 4; ++ab)
+            mma_bf16(tmem + static_cast<uint32_t>(ab * 128), desc_mn(base + (ab >> 1) * kQ, 128, k), desc_mn(base + 2 * kQ + (ab & 1) * kQ, 128, k),
+                     instr_desc(128, 128) | kAmn | kBmn, keep | (k > 0));
+      } else {        // d W1 [out half a][in] += d z1[:, a]^T . x;  d Wh^T [unit half a][head] += h2[:, a]^T . dhead
+#pragma unroll
+        for (int k = 0; k < kHalfRows / 16; ++k)
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * kQ, 128, k), desc_mn(base + 4 * kQ, kK1, k),
+                     instr_desc(128, kK1) | kAmn | kBmn, keep | (k > 0));
+            mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * kQ, 128, k), desc_mn(base + 4 * kQ + kXHalf, kHeads, k),
+                     instr_desc(128, kHeads) | kAmn | kBmn, keep | (k > 0));
+          }
+      }
+      mma_commit(empty0 + 8u * s);  // the stage is free once these MMAs have read it
+    }
+    // bias gradient: this thread's unit, summed over the item's rows in row order
+#pragma unroll 8
+    for (int r = 0; r < kHalfRows; ++r)
+      db += __uint_as_float(lds_u16(base + my_col + static_cast<uint32_t>((r >> 3) * 2048 + (r & 7) * 16)) << 16);
+    __syncwarp();
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8u * s) : "memory");
+    if (tid == 0 && u >= 1 && issued < n_items) {
+      // the previous item's stage (its MMAs are done and every warp has summed it) takes the item S - 1 ahead
+      timed_out |= !mbar_wait(empty0 + 8u * ((u - 1) % S), ((u - 1) / S) & 1);
+      if (!timed_out) { request(issued); ++issued; }
+    }
+  }
+  if (tid == 0 && !timed_out) {  // one more commit covers every MMA issued so far
+    mma_commit(done_bar);
+    timed_out |= !mbar_wait(done_bar, 0);
+  }
+  timed_out = __syncthreads_or(timed_out) != 0;
+  if (!timed_out && my_tiles > 0) {
+    tc_fence_after();
+    float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int a = warp >> 2, unit = a * 128 + (warp & 3) * 32 + lane;  // out-unit half a; tensor-memory lane = unit inside the half
+    float v[16];
+    if (role_w2) {
+      for (int b = 0; b < 2; ++b)
+        for (int c0 = 0; c0 < 128; c0 += 16) {
+          tmem_ld16(tmem + lane_off + static_cast<uint32_t>((a * 2 + b) * 128 + c0), v);
+          float *dst = part + off.W2 + static_cast<size_t>(unit) * kH + b * 128 + c0;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) dst[c] += v[c];
+        }
+      part[off.b2 + tid] += db;
+    } else {
+      for (int c0 = 0; c0 < kK1; c0 += 16) {
+        tmem_ld16(tmem + lane_off + static_cast<uint32_t>(a * kK1 + c0), v);
+        for (int c = 0; c < 16; ++c)
+          if (c0 + c < D) part[off.W1 + static_cast<size_t>(unit) * D + c0 + c] += v[c];
+      }
+      tmem_ld16(tmem + lane_off + static_cast<uint32_t>(192 + a * 32), v);
+      for (int k = 0; k < kActions; ++k) part[off.Wa + static_cast<size_t>(k) * kH + unit] += v[k];
+      if (has_value) part[off.Wv + unit] += v[kActions];
+      part[off.b1 + tid] += db;
+    }
+  }
+  if (timed_out && tid == 0) {
+    atomicExch(status, kStatusTimeout);
+    for (int u = issued > S ? issued - S : 0; u < issued; ++u) mbar_wait(full0 + 8u * (u % S), (u / S) & 1);  // copies in flight land first
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kCols) : "memory");
+  }
+}
+
+}  // namespace
+
+bool ppo_tc256_supported(const mava_config_t &cfg, int D) { return cfg.hidden == kH && D <= kK1 && D > 64; }
+size_t ppo_tc256_image_bytes() { return kImgBytes; }
+size_t ppo_tc256_staging_bytes(int chunk_tiles) { return static_cast<size_t>(chunk_tiles) * kStTile; }
+
+cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const ParamLayout &L, const UpdRows &rows, const UpdHyper &hp,
+                                 const double *adv_stats, void *image, void *staging, int chunk_tiles, float *partial, size_t n_params,
+                                 double *term_partial, int slices, bool has_value) {
+  prep_upd256_kernel<<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(image), L, h->D, has_value ? 1 : 0);
+  h->launches += 1;
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  err = cudaFuncSetAttribute(ppo_rows256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(RowSmem)));
+  if (err == cudaSuccess)
+    err = cudaFuncSetAttribute(ppo_weights256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(WgtSmem)));
+  if (err != cudaSuccess) return err;
+  const long long tiles = (rows.n + kR - 1) / kR;
+  const HeadOffsets ho{L.ba, L.bv};
+  const WgtOffsets wo{L.W1, L.b1, L.W2, L.b2, L.Wa, L.Wv};
+  // CTAs of the weight kernel by the bytes each group streams per tile (128 KB against 156 KB)
+  const int n_w2 = slices >= 2 ? (slices * 128 + 142) / 284 : 1;
+  for (long long t0 = 0; t0 < tiles; t0 += chunk_tiles) {
+    const int nt = static_cast<int>(tiles - t0 < chunk_tiles ? tiles - t0 : chunk_tiles);
+    ppo_rows256_kernel<<<slices, kThreads, sizeof(RowSmem), h->stream>>>(static_cast<const unsigned char *>(image), rows, hp, adv_stats,
+                                                                         static_cast<unsigned char *>(staging), t0, nt, partial, n_params,
+                                                                         term_partial, h->d_status, ho, h->D, has_value ? 1 : 0);
+    ppo_weights256_kernel<<<slices, kThreads, sizeof(WgtSmem), h->stream>>>(static_cast<const unsigned char *>(staging), nt, n_w2, partial,
+                                                                            n_params, h->d_status, wo, h->D, has_value ? 1 : 0);
+    h->launches += 2;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace mava

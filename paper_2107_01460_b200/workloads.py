@@ -34,6 +34,17 @@ WORKLOADS = {
     "cfg4_20x20_8p8f_h256": dict(
         grid=20, n_agents=8, n_food=8, max_agent_level=3, view_radius=2, episode_cap=100,
         hidden=256, net_kind=0, n_envs=32768, T=64, seed=4, precision="bf16"),
+    # Recurrent-policy variants (Section 2: every system has a recurrent version; Section 4: the LBF results are
+    # recurrent).  net_kind 2: dense ReLU embedding, one gated recurrent unit of the same width, actor and value heads.
+    "rec0_tiny_8x8_2p2f_gru64": dict(
+        grid=8, n_agents=2, n_food=2, max_agent_level=2, view_radius=2, episode_cap=50,
+        hidden=64, net_kind=2, n_envs=16, T=32, seed=10, precision="bf16"),
+    "rec1_8x8_2p2f_gru64": dict(
+        grid=8, n_agents=2, n_food=2, max_agent_level=2, view_radius=2, episode_cap=50,
+        hidden=64, net_kind=2, n_envs=1024, T=128, seed=11, precision="bf16"),
+    "rec2_10x10_3p3f_gru64": dict(
+        grid=10, n_agents=3, n_food=3, max_agent_level=3, view_radius=2, episode_cap=100,
+        hidden=64, net_kind=2, n_envs=8192, T=128, seed=12, precision="bf16"),
 }
 WORKLOAD_NAMES = list(WORKLOADS)
 GAMMA = 0.99
@@ -41,7 +52,8 @@ LAMBDA = 0.95
 
 
 def workload(name_or_index) -> dict:
-    """A copy of one workload description, by name or by index 0..4."""
+    """A copy of one workload description, by name or by index (0..4: the five feed-forward shapes; 5..7: the
+    recurrent variants)."""
     if isinstance(name_or_index, int):
         name_or_index = WORKLOAD_NAMES[name_or_index]
     w = dict(WORKLOADS[name_or_index])
@@ -58,6 +70,8 @@ def param_shapes(w: dict):
     """(name, (out, in)) of every dense layer, in the order the flat parameter
     array stores them (weight [out][in] then bias [out] for each)."""
     D, H, N = obs_dim(w), w["hidden"], w["n_agents"]
+    if w["net_kind"] == 2:  # recurrent: embedding, the cell's input and hidden matrices (gates r, z, n stacked), heads
+        return [("W1", (H, D)), ("Wih", (3 * H, H)), ("Whh", (3 * H, H)), ("Wa", (N_ACTIONS, H)), ("Wv", (1, H))]
     layers = [("W1", (H, D)), ("W2", (H, H)), ("Wa", (N_ACTIONS, H))]
     if w["net_kind"] == 0:
         layers += [("Wv", (1, H))]

@@ -177,8 +177,24 @@ def test_minibatches_of_environments(idx, n_envs, T):
 # these with a wide margin.  Against the exact float64 oracle the operands' rounding itself shows (2^-9 relative per
 # operand, logits good to 2e-2): 5e-2 * max|grad| and 2e-2 * (1 + |ref|).
 
+def _tensor_path_reference(w, shapes, p64, batch, hp, emulate):
+    """Oracle loss terms and gradient for the tensor-core path.  With a centralised critic only the actor net runs on
+    the tensor cores; the critic's net stays on the fp32 kernel, so in bf16-operand mode its loss term and its layers'
+    gradients are the exact oracle's (the two nets share no parameter)."""
+    ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
+    ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
+    if emulate and w["net_kind"] == 1:
+        exact = ppo.ppo_loss(p64, shapes, 1, batch)
+        ref = dict(ref, value=exact["value"], total=ref["actor"] - hp.ent_coef * ref["entropy"] + hp.vf_coef * exact["value"])
+        n_actor = sum(o * i + o for _, (o, i) in shapes[:3])
+        ref_grad = np.concatenate([ref_grad[:n_actor], ppo.ppo_grad(p64, shapes, 1, batch)[n_actor:]])
+    return ref, ref_grad
+
+
 @pytest.mark.parametrize("idx,n_envs,T", [(0, 16, 32), (1, 77, 20), (2, 50, 33), (2, 300, 40), (0, 1, 3),
-                                          (1, 1024, 128)])  # the last: the size the benchmark times
+                                          (1, 1024, 128),  # the size the benchmark times
+                                          # H = 256: row kernel + weight kernel (with the centralised critic: the actor net)
+                                          (4, 21, 11), (4, 150, 40), (3, 45, 17), (3, 300, 20), (4, 1, 2)])
 def test_tensor_core_update_matches_the_bf16_operand_oracle(idx, n_envs, T):
     import torch
 
@@ -195,8 +211,7 @@ def test_tensor_core_update_matches_the_bf16_operand_oracle(idx, n_envs, T):
     t = terms.cpu().numpy()
     gg = grad.cpu().numpy().astype(np.float64)
     for emulate, g_tol, l_tol in ((True, 2e-3, 2e-4), (False, 5e-2, 2e-2)):
-        ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
-        ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
+        ref, ref_grad = _tensor_path_reference(w, shapes, p64, batch, hp, emulate)
         for k, name in enumerate(("total", "actor", "entropy", "value")):
             assert abs(t[k] - ref[name]) <= l_tol * (1 + abs(ref[name])), (emulate, name, t[k], ref[name])
         worst = np.max(np.abs(gg - ref_grad)) / np.max(np.abs(ref_grad))
@@ -213,7 +228,7 @@ def test_tensor_core_update_matches_the_bf16_operand_oracle(idx, n_envs, T):
     ro.close()
 
 
-@pytest.mark.parametrize("idx,n_envs,T", [(1, 333, 20), (2, 141, 16)])
+@pytest.mark.parametrize("idx,n_envs,T", [(1, 333, 20), (2, 141, 16), (4, 90, 12), (3, 70, 9)])
 def test_tensor_core_update_on_minibatches_of_environments(idx, n_envs, T):
     import torch
 
@@ -230,8 +245,7 @@ def test_tensor_core_update_on_minibatches_of_environments(idx, n_envs, T):
         take = lambda name, n: getattr(ro, name)[:n].cpu().numpy().astype(np.float64)[:, sel]
         batch = ppo.batch_from_rollout(take("obs", T), ro.actions[:T].cpu().numpy()[:, sel], take("logp", T), take("values", T + 1),
                                        take("adv", T), take("ret", T), w["net_kind"])
-        ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch, emulate_bf16=True)
-        ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch, emulate_bf16=True)
+        ref, ref_grad = _tensor_path_reference(w, shapes, p64, batch, binding.ppo_defaults(), True)
         t = terms.cpu().numpy()
         for k, name in enumerate(("total", "actor", "entropy", "value")):
             assert abs(t[k] - ref[name]) <= 2e-4 * (1 + abs(ref[name])), (name, t[k], ref[name])
