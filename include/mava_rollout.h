@@ -47,6 +47,9 @@ extern "C" {
 #define MAVA_NET_SHARED_TORSO 0 /* one torso, a 6-logit actor head and a value head (IPPO-style)   */
 #define MAVA_NET_CENTRAL_CRITIC 1 /* actor net per agent + critic on the joint observation (MAPPO) */
 
+#define MAVA_NET_RECURRENT 2 /* recurrent policy: dense ReLU embedding, one gated recurrent unit of width H that
+                                carries a hidden vector per agent, actor and value heads on the new hidden vector */
+
 #define MAVA_PRECISION_FP32 0 /* fp32 SIMT arithmetic (validation path)                            */
 #define MAVA_PRECISION_BF16 1 /* bf16 operands, fp32 accumulation on the tcgen05 tensor cores      */
 
@@ -107,7 +110,15 @@ typedef mava_buffers_t mava_host_buffers_t;
  *   MAVA_NET_CENTRAL_CRITIC: W1[H][D] b1  W2[H][H] b2  Wa[6][H] ba  (actor, per agent)
  *                            C1[H][N*D] c1  C2[H][H] c2  Cv[1][H] cv (critic; its input is the
  *                            observations of agents 0..N-1 concatenated)
- * ReLU follows both hidden layers; heads are linear.  Returns 0 for an invalid config. */
+ *   MAVA_NET_RECURRENT:      W1[H][D] b1  Wih[3H][H] bih[3H]  Whh[3H][H] bhh[3H]  Wa[6][H] ba  Wv[1][H] bv
+ * ReLU follows both hidden layers; heads are linear.  Recurrent policy (Section 2 names recurrent versions of every
+ * system and Section 4 reports them on LBF; no cell or size is given, so this is the library's reading): e = relu(W1 x +
+ * b1); gated recurrent unit of Cho et al. (2014) with the gate blocks r, z, n stacked in that order,
+ *   r = sigma(Wir e + bir + Whr h + bhr);  z = sigma(Wiz e + biz + Whz h + bhz);
+ *   n = tanh(Win e + bin + r * (Whn h + bhn));  h' = (1 - z) * n + z * h;
+ * heads on h'.  The hidden vector of every agent is zero at create/reset and restarts from zero whenever its
+ * environment's episode ends; the handle carries it from one run to the next.  The bootstrap row values[T] comes from
+ * one more cell update on the observation after the last step, which is not kept.  Returns 0 for an invalid config. */
 size_t mava_params_count(const mava_config_t *cfg);
 
 /* Validates cfg, allocates the handle and its device state on the current device, places every
@@ -212,6 +223,10 @@ int mava_rollout_status(mava_rollout_t *h);
 int32_t mava_state_record_len(const mava_config_t *cfg);
 int mava_rollout_get_state(mava_rollout_t *h, int32_t *records_host);
 int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host);
+
+/* Recurrent policy: copies the hidden vectors the next run will start from, [E][N][H] fp32, to host memory (waits
+ * for the stream).  Errors: INVALID_ARG (also when the handle's net is not recurrent), CUDA. */
+int mava_rollout_get_hidden(mava_rollout_t *h, float *hidden_host);
 
 /* End-to-end convenience with HOST buffers: copies params_host to the device, runs T steps and
  * GAE, copies every non-NULL array of `out` back to the host (rows 0..T-1; T+1 rows of values)

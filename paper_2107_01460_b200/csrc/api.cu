@@ -16,7 +16,7 @@ bool config_ok(const mava_config_t &c) {
   return c.grid >= 3 && c.grid <= 64 && c.n_agents >= 1 && c.n_agents <= kMaxAgents && c.n_food >= 1 &&
          c.n_food <= kMaxFood && c.max_agent_level >= 1 && c.max_agent_level <= 3 &&
          c.n_agents + c.n_food <= c.grid * c.grid && c.episode_cap >= 1 && c.n_envs >= 1 && c.max_T >= 1 &&
-         c.hidden >= 1 && c.first_env >= 0 && c.reserved == 0 && (c.net_kind == MAVA_NET_SHARED_TORSO || c.net_kind == MAVA_NET_CENTRAL_CRITIC) &&
+         c.hidden >= 1 && c.first_env >= 0 && c.reserved == 0 && (c.net_kind == MAVA_NET_SHARED_TORSO || c.net_kind == MAVA_NET_CENTRAL_CRITIC || c.net_kind == MAVA_NET_RECURRENT) &&
          (c.precision == MAVA_PRECISION_FP32 || c.precision == MAVA_PRECISION_BF16);
 }
 
@@ -71,7 +71,8 @@ int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_
   args.write_logits = (h->cfg.flags & MAVA_FLAG_WRITE_LOGITS) ? 1 : 0;
   args.status = h->d_status;
   args.obs_last = h->d_obs_last;
-  if (!ev && (h->expire_next & MAVA_EXPIRE_ROLLOUT) && h->cfg.precision == MAVA_PRECISION_BF16 && tc_rollout_is_wide(h)) {
+  if (!ev && (h->expire_next & MAVA_EXPIRE_ROLLOUT) && h->cfg.precision == MAVA_PRECISION_BF16 && h->cfg.net_kind != MAVA_NET_RECURRENT &&
+      tc_rollout_is_wide(h)) {
     args.debug_expire = 1;
     h->expire_next &= ~MAVA_EXPIRE_ROLLOUT;
   }
@@ -82,7 +83,10 @@ int run_common(mava_rollout *h, const float *params_dev, int32_t T, const int32_
     args.obs_last = nullptr;
   }
   cudaError_t err;
-  if (h->cfg.precision == MAVA_PRECISION_BF16) {
+  if (h->cfg.net_kind == MAVA_NET_RECURRENT) {
+    if (ev) return MAVA_ERR_UNSUPPORTED;  // no evaluation block for the recurrent policy
+    err = h->cfg.precision == MAVA_PRECISION_BF16 ? launch_rollout_rec_tc(h, params_dev, args) : launch_rollout_rec_simt(h, params_dev, args);
+  } else if (h->cfg.precision == MAVA_PRECISION_BF16) {
     err = launch_prep_tc(h, params_dev);
     if (err == cudaSuccess) err = launch_rollout_tc(h, args);
     if (err == cudaSuccess && !ev && h->cfg.net_kind == MAVA_NET_CENTRAL_CRITIC) err = launch_critic_tc(h, params_dev, T);
@@ -146,6 +150,10 @@ int mava_rollout_create(const mava_config_t *cfg, const mava_buffers_t *buffers,
             cudaMalloc(&h->d_params_stage, sizeof(float) * np) == cudaSuccess;
   if (ok && cfg->precision == MAVA_PRECISION_BF16)
     ok = cudaMalloc(&h->d_wtc, tc_weight_bytes(*cfg, h->D)) == cudaSuccess;
+  if (ok && cfg->net_kind == MAVA_NET_RECURRENT) {
+    const size_t bytes = sizeof(float) * static_cast<size_t>(cfg->n_envs) * cfg->n_agents * cfg->hidden;
+    ok = cudaMalloc(&h->d_hidden, bytes) == cudaSuccess && cudaMemsetAsync(h->d_hidden, 0, bytes, h->stream) == cudaSuccess;
+  }
   if (ok && cfg->precision == MAVA_PRECISION_BF16 && cfg->net_kind == MAVA_NET_CENTRAL_CRITIC)
     ok = cudaMalloc(&h->d_critic, critic_weight_bytes(*cfg)) == cudaSuccess &&
          cudaMalloc(&h->d_obs_last, sizeof(float) * static_cast<size_t>(cfg->n_envs) * cfg->n_agents * h->D) == cudaSuccess;
@@ -202,6 +210,7 @@ void mava_ppo_defaults(mava_ppo_hyper_t *hp) {
 int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, float *grad_dev, float *terms_dev) {
   if (!h || !params_dev || !hp || !grad_dev || h->last_T < 1 || !h->buf.adv || !h->buf.ret) return MAVA_ERR_INVALID_ARG;
   if (!(hp->clip_eps > 0.0f)) return MAVA_ERR_INVALID_ARG;
+  if (h->cfg.net_kind == MAVA_NET_RECURRENT) return MAVA_ERR_UNSUPPORTED;  // no update block for the recurrent policy
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
   return launch_ppo_grad(h, params_dev, *hp, grad_dev, terms_dev, nullptr, 0) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
@@ -212,6 +221,7 @@ int mava_ppo_grad_envs(mava_rollout_t *h, const float *params_dev, const mava_pp
   if (!h || !params_dev || !hp || !grad_dev || !env_ids_dev || n_ids < 1 || h->last_T < 1 || !h->buf.adv || !h->buf.ret)
     return MAVA_ERR_INVALID_ARG;
   if (!(hp->clip_eps > 0.0f)) return MAVA_ERR_INVALID_ARG;
+  if (h->cfg.net_kind == MAVA_NET_RECURRENT) return MAVA_ERR_UNSUPPORTED;
   DeviceGuard guard(h->device);
   if (!guard.ok) return MAVA_ERR_CUDA;
   return launch_ppo_grad(h, params_dev, *hp, grad_dev, terms_dev, env_ids_dev, n_ids) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
@@ -232,6 +242,9 @@ int mava_rollout_reset(mava_rollout_t *h, uint64_t seed) {
   h->cfg.seed = seed;
   h->t_global = 0;
   h->last_T = 0;
+  if (h->d_hidden &&
+      cudaMemsetAsync(h->d_hidden, 0, sizeof(float) * static_cast<size_t>(h->cfg.n_envs) * h->cfg.n_agents * h->cfg.hidden, h->stream) != cudaSuccess)
+    return MAVA_ERR_CUDA;
   return launch_env_init(h) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
 }
 
@@ -297,6 +310,17 @@ int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host) {
   }
   if (cudaStreamSynchronize(h->stream) != cudaSuccess ||
       cudaMemcpy(h->d_state, recs.data(), sizeof(EnvRec) * recs.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+    return MAVA_ERR_CUDA;
+  return MAVA_OK;
+}
+
+int mava_rollout_get_hidden(mava_rollout_t *h, float *hidden_host) {
+  if (!h || !hidden_host || !h->d_hidden) return MAVA_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return MAVA_ERR_CUDA;
+  const size_t bytes = sizeof(float) * static_cast<size_t>(h->cfg.n_envs) * h->cfg.n_agents * h->cfg.hidden;
+  if (cudaMemcpyAsync(hidden_host, h->d_hidden, bytes, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
     return MAVA_ERR_CUDA;
   return MAVA_OK;
 }
@@ -407,6 +431,7 @@ int mava_rollout_run_static(const mava_config_t *cfg, const mava_buffers_t *buff
   const int variant = find_variant(*cfg);
   if (variant < 0) return MAVA_ERR_UNSUPPORTED;
   const bool bf16 = cfg->precision == MAVA_PRECISION_BF16;
+  if (cfg->net_kind == MAVA_NET_RECURRENT) return MAVA_ERR_UNSUPPORTED;  // its hidden vectors are handle state
   if (bf16 && !tc_supported(*cfg)) return MAVA_ERR_UNSUPPORTED;
   if (bf16 && cfg->net_kind == MAVA_NET_CENTRAL_CRITIC) return MAVA_ERR_UNSUPPORTED;  // its scratch is far beyond the array
 
@@ -462,6 +487,7 @@ void mava_rollout_destroy(mava_rollout_t *h) {
   cudaFree(h->d_obs_last);
   cudaFree(h->d_upd);
   cudaFree(h->d_upd_stage);
+  cudaFree(h->d_hidden);
   if (h->copy_ready) {
     cudaStreamSynchronize(h->copy_stream);
     for (int i = 0; i <= kCollectChunks; ++i) cudaEventDestroy(h->chunk_done[i]);

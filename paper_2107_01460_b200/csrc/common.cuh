@@ -110,6 +110,7 @@ struct mava_rollout {
   float *d_obs_last;   //   and the observations after the last step [E][N][D]
   void *d_upd;         // scratch of the update block (made on its first call)
   size_t upd_bytes;
+  float *d_hidden;     // recurrent policy: the agents' hidden vectors [E][N][H]
   void *d_upd_stage;   // staging buffer of the H = 256 tensor-core update (made on its first call)
   size_t upd_stage_bytes;
   uint32_t t_global;
@@ -143,6 +144,11 @@ bool tc_supported(const mava_config_t &cfg);
 bool tc_rollout_is_wide(const mava_rollout *h);  // the next bf16 rollout launch takes the 128-row kernel (not the few-rows form)
 size_t critic_weight_bytes(const mava_config_t &cfg);
 cudaError_t launch_critic_tc(mava_rollout *h, const float *params_dev, int32_t T);
+
+// Recurrent policy (rollout_rec.cu: fp32 SIMT; rollout_rec_tc.cu: bf16 tensor cores).
+cudaError_t launch_rollout_rec_simt(mava_rollout *h, const float *params_dev, const RolloutArgs &args);
+cudaError_t launch_rollout_rec_tc(mava_rollout *h, const float *params_dev, const RolloutArgs &args);
+size_t rec_tc_weight_bytes(const mava_config_t &cfg);
 
 // Update block (fp32).
 cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava_ppo_hyper_t &hp, float *grad_dev, float *terms_dev,

@@ -9,6 +9,7 @@ namespace mava {
 struct ParamLayout {
   size_t W1, b1, W2, b2, Wa, ba, Wv, bv;  // Wv/bv unused with the central critic
   size_t C1, c1, C2, c2, Cv, cv;          // central critic only
+  size_t Wih, bih, Whh, bhh;              // recurrent policy only: the cell's matrices [3H][H] and biases [3H] (gates r, z, n)
   size_t total;
 };
 
@@ -25,6 +26,14 @@ inline ParamLayout param_layout(const mava_config_t &cfg, int D, size_t align) {
     return at;
   };
   L.W1 = take(H * D); L.b1 = take(H);
+  if (cfg.net_kind == MAVA_NET_RECURRENT) {
+    L.Wih = take(3 * H * H); L.bih = take(3 * H);
+    L.Whh = take(3 * H * H); L.bhh = take(3 * H);
+    L.Wa = take(MAVA_N_ACTIONS * H); L.ba = take(MAVA_N_ACTIONS);
+    L.Wv = take(H); L.bv = take(1);
+    L.total = (off + align - 1) / align * align;
+    return L;
+  }
   L.W2 = take(H * H); L.b2 = take(H);
   L.Wa = take(MAVA_N_ACTIONS * H); L.ba = take(MAVA_N_ACTIONS);
   if (cfg.net_kind == MAVA_NET_SHARED_TORSO) {

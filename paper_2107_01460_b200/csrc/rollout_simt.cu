@@ -5,50 +5,11 @@
 #include "common.cuh"
 #include "env.cuh"
 #include "layout.h"
+#include "simt_dense.cuh"
 
 namespace mava {
 
 namespace {
-
-constexpr int kSimtThreads = 256;
-constexpr int kSimtRows = 32;  // agent rows per tile (upper bound; a tile holds floor(32/N) envs)
-
-// y[row][o] = act(sum_k x[row][k] * Wt[k][o] + b[o]) for `ROWS` rows held in shared memory.
-// Thread (rg, cg) owns four consecutive outputs of RPT rows; k runs in ascending order.
-template <int K, int HOUT, int ROWS, bool RELU>
-__device__ __forceinline__ void dense_tile(const float *xs, int x_stride, const float *__restrict__ Wt,
-                                           const float *__restrict__ b, float *ys, int y_stride, int tid) {
-  constexpr int CG = HOUT / 4;
-  constexpr int RG = kSimtThreads / CG;
-  constexpr int RPT = (ROWS + RG - 1) / RG;
-  static_assert(kSimtThreads % CG == 0, "thread layout");
-  const int cg = tid % CG, rg = tid / CG;
-  float acc[RPT][4];
-#pragma unroll
-  for (int i = 0; i < RPT; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0f;
-  for (int k = 0; k < K; ++k) {
-    const float4 w = __ldg(reinterpret_cast<const float4 *>(Wt + static_cast<size_t>(k) * HOUT) + cg);
-#pragma unroll
-    for (int i = 0; i < RPT; ++i) {
-      const int row = rg + i * RG;
-      const float x = row < ROWS ? xs[row * x_stride + k] : 0.0f;
-      acc[i][0] = fmaf(x, w.x, acc[i][0]);
-      acc[i][1] = fmaf(x, w.y, acc[i][1]);
-      acc[i][2] = fmaf(x, w.z, acc[i][2]);
-      acc[i][3] = fmaf(x, w.w, acc[i][3]);
-    }
-  }
-  const float4 bias = __ldg(reinterpret_cast<const float4 *>(b) + cg);
-#pragma unroll
-  for (int i = 0; i < RPT; ++i) {
-    const int row = rg + i * RG;
-    if (row >= ROWS) continue;
-    float v0 = acc[i][0] + bias.x, v1 = acc[i][1] + bias.y, v2 = acc[i][2] + bias.z, v3 = acc[i][3] + bias.w;
-    if (RELU) { v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); v2 = fmaxf(v2, 0.0f); v3 = fmaxf(v3, 0.0f); }
-    float *y = ys + row * y_stride + cg * 4;
-    y[0] = v0; y[1] = v1; y[2] = v2; y[3] = v3;
-  }
-}
 
 template <int N, int F, int H, bool CENTRAL>
 struct SimtSmem {
@@ -260,8 +221,9 @@ cudaError_t launch_simt_variant(mava_rollout *h, const RolloutArgs &args, const 
 // The compiled (N, F, H, net_kind) combinations.
 int find_variant(const mava_config_t &c) {
   struct V { int n, f, h, kind; };
-  static const V table[] = {{2, 2, 64, 0}, {2, 2, 128, 0}, {3, 3, 128, 0}, {4, 5, 256, 1}, {8, 8, 256, 0}};
-  for (int i = 0; i < 5; ++i)
+  static const V table[] = {{2, 2, 64, 0}, {2, 2, 128, 0}, {3, 3, 128, 0}, {4, 5, 256, 1}, {8, 8, 256, 0},
+                            {2, 2, 64, 2}, {3, 3, 64, 2}};  // the last two: the recurrent policy
+  for (int i = 0; i < 7; ++i)
     if (table[i].n == c.n_agents && table[i].f == c.n_food && table[i].h == c.hidden && table[i].kind == c.net_kind)
       return i;
   return -1;
@@ -274,8 +236,8 @@ cudaError_t launch_env_init(mava_rollout *h) {
               static_cast<uint32_t>(h->cfg.seed), static_cast<uint32_t>(h->cfg.seed >> 32)};
   const int threads = 128, blocks = (h->cfg.n_envs + threads - 1) / threads;
   switch (h->variant) {
-    case 0: case 1: env_init_kernel<2, 2><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
-    case 2: env_init_kernel<3, 3><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
+    case 0: case 1: case 5: env_init_kernel<2, 2><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
+    case 2: case 6: env_init_kernel<3, 3><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
     case 3: env_init_kernel<4, 5><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
     case 4: env_init_kernel<8, 8><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
     default: return cudaErrorInvalidValue;

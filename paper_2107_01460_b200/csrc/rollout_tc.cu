@@ -705,7 +705,7 @@ cudaError_t launch_prep_variant(mava_rollout *h, const float *params_dev) {
 // All compiled shapes run on the tensor cores (the centralised critic through critic_tc.cu).
 bool tc_supported(const mava_config_t &cfg) {
   const int v = find_variant(cfg);
-  return v == 0 || v == 1 || v == 2 || v == 3 || v == 4;
+  return v == 0 || v == 1 || v == 2 || v == 3 || v == 4 || v == 5 || v == 6;
 }
 
 // Hidden activations in tensor memory: always for H = 256; for the smaller shapes only when the
@@ -728,6 +728,7 @@ size_t tc_weight_bytes(const mava_config_t &cfg, int) {
     case 2: return TcShape<3, 128, false>::IMAGE_BYTES;
     case 3: return TcShape<4, 256, true>::IMAGE_BYTES;
     case 4: return TcShape<8, 256, true>::IMAGE_BYTES;
+    case 5: case 6: return rec_tc_weight_bytes(cfg);
     default: return 16;
   }
 }
