@@ -48,6 +48,8 @@ def bytes_per_row(w) -> float:
 def flops_per_row(w) -> float:
     """2 * multiply-accumulates of the unpadded network, per agent row."""
     D, H, N = wl.obs_dim(w), w["hidden"], w["n_agents"]
+    if w["net_kind"] == 2:  # recurrent: embedding, the cell's two [3H][H] matrices, the heads
+        return 2.0 * (D * H + 6 * H * H + 7 * H)
     macs = D * H + H * H + 6 * H
     if w["net_kind"] == 0:
         macs += H
@@ -162,7 +164,10 @@ def oracle_sample_run(w, params, n_sample_envs: int, n_threads: int):
     results = [None] * len(chunks)
 
     def work(i):
-        ro = oracle.rollout(ocfg, w["seed"], params, T, chunks[i], want_obs=True)
+        if w["net_kind"] == 2:
+            ro, _ = oracle.rollout_rec(ocfg, w["seed"], params, T, chunks[i], want_obs=True)
+        else:
+            ro = oracle.rollout(ocfg, w["seed"], params, T, chunks[i], want_obs=True)
         adv, ret = oracle.gae(ro.values.astype(np.float32), ro.rewards, ro.dones, wl.GAMMA, wl.LAMBDA)
         results[i] = adv.shape
 
@@ -196,7 +201,7 @@ def oracle_baseline(w, seconds_each: float):
     out = {}
     for label, n_env, n_thr in (("single_thread", n_single, 1), ("all_cores", n_multi, cores)):
         rows, secs, passes, used = 0, 0.0, 0, n_thr
-        while secs < seconds_each and passes < 256:
+        while secs < seconds_each and passes < 4096:
             r_, s_, used = oracle_sample_run(w, params, n_env, n_thr)
             rows += r_; secs += s_; passes += 1
         out[label] = {"value": rows / secs, "unit": UNIT, "cores": used, "kind": "oracle",
@@ -311,7 +316,9 @@ def time_update(torch, binding, ro, params, w, steps, warmup, flush):
         e1.synchronize()
         if i >= warmup:
             times.append(e0.elapsed_time(e1))
-    path = "bf16 tcgen05" if ro.cfg.precision == binding.MAVA_PRECISION_BF16 and binding.update_on_tensor_cores(ro.cfg) else "fp32 SIMT"
+    path = "fp32 SIMT"
+    if binding.update_on_tensor_cores(ro.cfg):
+        path = "bf16 tcgen05" + (" (actor net; the centralised critic's net in fp32 SIMT)" if ro.cfg.net_kind == 1 else "")
     return sum(times) / len(times), path
 
 
@@ -429,11 +436,12 @@ def run_gpu(args):
     # every workload of the table, briefly: device times, roofline fractions, and the oracle beside each
     sweep = []
     if not args.no_sweep and world == 1:
-        for idx in range(5):
+        for idx in range(len(wl.WORKLOAD_NAMES)):
             wi = wl.workload(idx)
             pi = pick_precision(binding, wi)
             r_i, p_i, tr, tg, _ = time_workload(torch, binding, wi, pi, 5, 3, flush=flush)
-            tu_ms, tu_path = time_update(torch, binding, r_i, p_i, wi, 2, 1, flush)
+            recurrent = wi["net_kind"] == 2  # the recurrent policy has a rollout and GAE, no update block
+            tu_ms, tu_path = (None, None) if recurrent else time_update(torch, binding, r_i, p_i, wi, 2, 1, flush)
             del r_i, p_i
             torch.cuda.empty_cache()
             ri = wi["n_envs"] * wi["n_agents"] * wi["T"]
@@ -446,8 +454,10 @@ def run_gpu(args):
                      "rollout_us_per_env_step": 1e3 * tr_ms / wi["T"],
                      "gae_elements_per_s": ri / (tg_ms * 1e-3),
                      "gae_hbm_frac": ri * gae_bytes_per_element(wi) / (tg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                     "update_ms": tu_ms, "update_path": tu_path, "update_rows_per_s": ri / (tu_ms * 1e-3),
-                     "update_tensor_frac": 3 * ri * flops_per_row(wi) / (tu_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+                     "update_ms": tu_ms, "update_path": tu_path}
+            if tu_ms is not None:
+                entry["update_rows_per_s"] = ri / (tu_ms * 1e-3)
+                entry["update_tensor_frac"] = 3 * ri * flops_per_row(wi) / (tu_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]
             if not args.no_oracle:
                 entry["cpu_baseline"] = oracle_baseline(wi, args.oracle_seconds)
             sweep.append(entry)

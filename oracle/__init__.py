@@ -45,6 +45,7 @@ class Config(C.Structure):
         ("episode_cap", C.c_int32),
         ("hidden", C.c_int32),
         ("net_kind", C.c_int32),
+        ("env_kind", C.c_int32),
     ]
 
 
@@ -64,7 +65,7 @@ class EnvState(C.Structure):
 
 def make_config(workload: dict) -> Config:
     """Config from a workload description (keys named like the struct fields)."""
-    return Config(**{name: int(workload[name]) for name, _ in Config._fields_})
+    return Config(**{name: int(workload.get(name, 0)) for name, _ in Config._fields_})
 
 
 _lib = None
@@ -96,6 +97,13 @@ def lib():
         L.orc_env_step.argtypes = [C.POINTER(Config), C.POINTER(EnvState), C.c_void_p, C.POINTER(C.c_float),
                                    C.POINTER(C.c_uint8)]
         L.orc_env_step.restype = None
+        L.orc_wh_reset.argtypes = [C.POINTER(Config), C.c_uint64, C.c_int32, C.c_int32, C.POINTER(EnvState)]
+        L.orc_wh_reset.restype = None
+        L.orc_wh_observe.argtypes = [C.POINTER(Config), C.POINTER(EnvState), C.c_int32, C.c_void_p]
+        L.orc_wh_observe.restype = None
+        L.orc_wh_step.argtypes = [C.POINTER(Config), C.c_uint64, C.c_int32, C.POINTER(EnvState), C.c_void_p,
+                                  C.POINTER(C.c_float), C.POINTER(C.c_uint8)]
+        L.orc_wh_step.restype = None
         L.orc_mlp_forward_env.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_mlp_forward_env.restype = None
         L.orc_sample.argtypes = [C.c_void_p, C.c_float, C.POINTER(C.c_int32), C.c_void_p, C.POINTER(C.c_double)]
@@ -156,6 +164,34 @@ def env_reset(cfg: Config, seed: int, env: int, episode: int) -> EnvState:
     s = EnvState()
     lib().orc_env_reset(C.byref(cfg), C.c_uint64(seed), env, episode, C.byref(s))
     return s
+
+
+def wh_reset(cfg: Config, seed: int, env: int, episode: int) -> EnvState:
+    """Start of a warehouse episode (see orc_wh_reset for how the state's fields are used)."""
+    s = EnvState()
+    lib().orc_wh_reset(C.byref(cfg), C.c_uint64(seed), env, episode, C.byref(s))
+    return s
+
+
+def wh_observe(cfg: Config, state: EnvState, agent: int) -> np.ndarray:
+    out = np.empty(obs_dim(cfg), dtype=np.float32)
+    lib().orc_wh_observe(C.byref(cfg), C.byref(state), agent, _ptr(out))
+    return out
+
+
+def wh_step(cfg: Config, seed: int, env: int, state: EnvState, actions):
+    """Advance a warehouse `state` in place; returns (reward, done)."""
+    a = np.ascontiguousarray(actions, dtype=np.int32)
+    assert a.size == cfg.n_agents
+    r = C.c_float()
+    d = C.c_uint8()
+    lib().orc_wh_step(C.byref(cfg), C.c_uint64(seed), env, C.byref(state), _ptr(a), C.byref(r), C.byref(d))
+    return np.float32(r.value), int(d.value)
+
+
+def initial_state(cfg: Config, seed: int, env: int, episode: int = 0) -> EnvState:
+    """Start-of-episode state of the workload family the config names."""
+    return env_reset(cfg, seed, env, episode) if cfg.env_kind == 0 else wh_reset(cfg, seed, env, episode)
 
 
 def env_observe(cfg: Config, state: EnvState, agent: int) -> np.ndarray:
@@ -221,7 +257,7 @@ def rollout(cfg: Config, seed: int, params, T: int, env_ids, *, forced_actions=N
     n = int(env_ids.size)
     N, D = cfg.n_agents, obs_dim(cfg)
     if states is None:
-        states = [env_reset(cfg, seed, int(e), 0) for e in env_ids]
+        states = [initial_state(cfg, seed, int(e), 0) for e in env_ids]
     st = (EnvState * n)(*states)
     fa = None
     if forced_actions is not None:
@@ -275,7 +311,7 @@ def rollout_rec(cfg: Config, seed: int, params, T: int, env_ids, *, forced_actio
     n = int(env_ids.size)
     N, D, H = cfg.n_agents, obs_dim(cfg), cfg.hidden
     if states is None:
-        states = [env_reset(cfg, seed, int(e), 0) for e in env_ids]
+        states = [initial_state(cfg, seed, int(e), 0) for e in env_ids]
     st = (EnvState * n)(*states)
     hid = np.zeros((n, N, H), dtype=np.float64) if hidden is None else np.array(hidden, dtype=np.float64, order="C", copy=True)
     assert hid.shape == (n, N, H)
@@ -319,7 +355,7 @@ def evaluate(cfg: Config, seed: int, params, T: int, env_ids, *, greedy: bool = 
     n = int(env_ids.size)
     N = cfg.n_agents
     if states is None:
-        states = [env_reset(cfg, seed, int(e), 0) for e in env_ids]
+        states = [initial_state(cfg, seed, int(e), 0) for e in env_ids]
     st = (EnvState * n)(*states)
     fa = None
     if forced_actions is not None:

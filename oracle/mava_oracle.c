@@ -36,6 +36,7 @@
 
 #define ORC_DOMAIN_RESET 0x52534554u  /* key tweak for placement draws  */
 #define ORC_DOMAIN_ACTION 0x41435431u /* key tweak for action uniforms  */
+#define ORC_DOMAIN_REQUEST 0x52455153u /* key tweak for the warehouse's new requests */
 
 typedef struct {
   int32_t grid;            /* G: playable cells are rows/cols 0..G-1            */
@@ -46,7 +47,10 @@ typedef struct {
   int32_t episode_cap;     /* episode ends when step reaches this               */
   int32_t hidden;          /* H: width of both hidden layers                    */
   int32_t net_kind;        /* 0: shared torso + actor/value heads
-                              1: actor net + centralised critic on joint obs    */
+                              1: actor net + centralised critic on joint obs
+                              2: recurrent policy                               */
+  int32_t env_kind;        /* 0: level-based foraging; 1: warehouse;
+                              2: warehouse whose episode ends on a robot conflict */
 } orc_config_t;
 
 typedef struct {
@@ -250,6 +254,201 @@ void orc_env_step(const orc_config_t *cfg, orc_env_state_t *s, const int32_t *ac
 }
 
 /* ------------------------------------------------------------------------- */
+/* Warehouse gridworld (the second workload family; Section 4, "Multi-Robot     */
+/* Warehouse": robots fetch requested shelves, and the variant the report       */
+/* trains on ends the episode on collisions).  The report gives no rules; the   */
+/* ones below were written for this library, sized so that observations,        */
+/* actions and networks are those of the foraging workloads.                    */
+/*                                                                             */
+/* State (in the fields of orc_env_state_t): robot n at (agent_r, agent_c),     */
+/* agent_level[n] = 0 when empty-handed, 1 + f while it carries shelf f;        */
+/* shelf f at (food_r, food_c) -- a carried shelf is at its carrier's cell --   */
+/* food_level[f] = 1 idle, 2 requested; total_food_level counts the deliveries  */
+/* of the episode.  Row 0 is the delivery row.  floor(F/2) shelves (at least    */
+/* one) are requested at all times.                                             */
+/*                                                                             */
+/* Reset (draws i = 0, 1, ... of the episode's reset stream): F shelf cells:    */
+/* draw k picks r in [0, (G-1)*G - k) and shelf k takes the r-th cell, in       */
+/* row-major order over rows 1..G-1, that no earlier shelf took; N robot cells: */
+/* draw picks r in [0, G*G - F - n) and robot n takes the r-th cell of the      */
+/* whole grid that holds neither a shelf nor an earlier robot; then the         */
+/* requests: draw k picks r in [0, F - k) and the r-th still idle shelf in      */
+/* index order becomes requested.                                               */
+/* ------------------------------------------------------------------------- */
+static int wh_requests(const orc_config_t *cfg) { return cfg->n_food / 2 > 0 ? cfg->n_food / 2 : 1; }
+
+void orc_wh_reset(const orc_config_t *cfg, uint64_t seed, int32_t env, int32_t episode, orc_env_state_t *s) {
+  const int G = cfg->grid, N = cfg->n_agents, F = cfg->n_food;
+  memset(s, 0, sizeof(*s));
+  s->episode = episode;
+  uint32_t draw = 0;
+  uint8_t *taken = (uint8_t *)calloc((size_t)G * G, 1);
+  for (int k = 0; k < F; ++k) {
+    uint32_t r = orc_bounded(reset_draw(seed, (uint32_t)env, (uint32_t)episode, draw++), (uint32_t)((G - 1) * G - k));
+    for (int i = G; i < G * G; ++i) {  /* rows 1 .. G-1 */
+      if (taken[i]) continue;
+      if (r == 0) { taken[i] = 1; s->food_r[k] = i / G; s->food_c[k] = i % G; break; }
+      --r;
+    }
+    s->food_level[k] = 1;
+  }
+  for (int n = 0; n < N; ++n) {
+    uint32_t r = orc_bounded(reset_draw(seed, (uint32_t)env, (uint32_t)episode, draw++), (uint32_t)(G * G - F - n));
+    for (int i = 0; i < G * G; ++i) {
+      if (taken[i]) continue;
+      if (r == 0) { taken[i] = 1; s->agent_r[n] = i / G; s->agent_c[n] = i % G; break; }
+      --r;
+    }
+    s->agent_level[n] = 0;
+  }
+  free(taken);
+  for (int k = 0; k < wh_requests(cfg); ++k) {
+    uint32_t r = orc_bounded(reset_draw(seed, (uint32_t)env, (uint32_t)episode, draw++), (uint32_t)(F - k));
+    for (int f = 0; f < F; ++f) {
+      if (s->food_level[f] != 1) continue;
+      if (r == 0) { s->food_level[f] = 2; break; }
+      --r;
+    }
+  }
+}
+
+/* Observation of robot `agent`: the same three 5x5 planes and scalars as the   */
+/* foraging workload, with these meanings: plane 0: 1 at an empty-handed        */
+/* robot's cell, 2 at a carrying robot's (own cell included); plane 1: 1 at an  */
+/* idle shelf's cell, 2 at a requested shelf's (on the ground or carried);      */
+/* plane 2: 1 outside the grid, 0.5 on the delivery row; then 1 or 2 for the    */
+/* robot itself, step/cap, one-hot id.                                          */
+void orc_wh_observe(const orc_config_t *cfg, const orc_env_state_t *s, int32_t agent, float *obs) {
+  const int G = cfg->grid, N = cfg->n_agents, F = cfg->n_food, R = cfg->view_radius;
+  const int W = 2 * R + 1, D = orc_obs_dim(cfg);
+  for (int i = 0; i < D; ++i) obs[i] = 0.0f;
+  const int r0 = s->agent_r[agent], c0 = s->agent_c[agent];
+  for (int dy = -R; dy <= R; ++dy) {
+    for (int dx = -R; dx <= R; ++dx) {
+      const int rr = r0 + dy, cc = c0 + dx, idx = (dy + R) * W + (dx + R);
+      if (rr < 0 || rr >= G || cc < 0 || cc >= G) { obs[2 * W * W + idx] = 1.0f; continue; }
+      if (rr == 0) obs[2 * W * W + idx] = 0.5f;
+      for (int n = 0; n < N; ++n)
+        if (s->agent_r[n] == rr && s->agent_c[n] == cc) obs[idx] = s->agent_level[n] > 0 ? 2.0f : 1.0f;
+      for (int f = 0; f < F; ++f)
+        if (s->food_r[f] == rr && s->food_c[f] == cc) obs[W * W + idx] = (float)s->food_level[f];
+    }
+  }
+  obs[3 * W * W] = s->agent_level[agent] > 0 ? 2.0f : 1.0f;
+  obs[3 * W * W + 1] = (float)s->step / (float)cfg->episode_cap;
+  obs[3 * W * W + 2 + agent] = 1.0f;
+}
+
+/* Transition, all decisions on the start-of-step state.                        */
+/*  Moves (actions 1..4): cancelled if the target is outside the grid, is       */
+/*   another robot's current cell, is another mover's target, or -- for a robot */
+/*   that carries a shelf -- holds a shelf standing on the ground.  The second  */
+/*   and third reasons are robot conflicts.  A carried shelf moves with its     */
+/*   robot; an empty-handed robot may pass under shelves.                       */
+/*  Action 5: an empty-handed robot standing under a shelf on the ground picks  */
+/*   it up; a carrying robot outside the delivery row puts its shelf down.      */
+/*  Delivery: a carrying robot whose cell after the moves is in the delivery    */
+/*   row, with a requested shelf, delivers it: the shelf becomes idle (and      */
+/*   stays on the robot).  For the deliveries in robot order, the d-th one      */
+/*   (d = 0, 1, ...) draws the replacement request: word 0 of the Philox block  */
+/*   with counter (d, env, episode, step) under the request key picks r in      */
+/*   [0, n) and the r-th of the n shelves that are idle and were not delivered  */
+/*   in this step, in index order, becomes requested.                           */
+/*  Reward: the number of deliveries of the step, to every robot.  step += 1;   */
+/*  done when the cap is reached, or (env_kind 2) when a robot conflict         */
+/*  cancelled a move in this step.  No reset happens here.                      */
+void orc_wh_step(const orc_config_t *cfg, uint64_t seed, int32_t env, orc_env_state_t *s, const int32_t *actions,
+                 float *reward, uint8_t *done) {
+  const int G = cfg->grid, N = cfg->n_agents, F = cfg->n_food;
+  static const int dr[ORC_N_ACTIONS] = {0, -1, 1, 0, 0, 0};
+  static const int dc[ORC_N_ACTIONS] = {0, 0, 0, -1, 1, 0};
+  int moving[ORC_MAX_AGENTS], tr[ORC_MAX_AGENTS], tc[ORC_MAX_AGENTS], ok[ORC_MAX_AGENTS];
+  int carried[ORC_MAX_FOOD]; /* shelf f is on a robot at the start of the step */
+  for (int f = 0; f < F; ++f) carried[f] = 0;
+  for (int n = 0; n < N; ++n)
+    if (s->agent_level[n] > 0) carried[s->agent_level[n] - 1] = 1;
+  for (int n = 0; n < N; ++n) {
+    const int a = actions[n];
+    moving[n] = (a >= 1 && a <= 4);
+    tr[n] = s->agent_r[n] + (moving[n] ? dr[a] : 0);
+    tc[n] = s->agent_c[n] + (moving[n] ? dc[a] : 0);
+  }
+  int conflict = 0;
+  for (int n = 0; n < N; ++n) {
+    ok[n] = moving[n];
+    if (!moving[n]) continue;
+    if (tr[n] < 0 || tr[n] >= G || tc[n] < 0 || tc[n] >= G) ok[n] = 0;
+    for (int m = 0; m < N; ++m) {
+      if (m == n) continue;
+      if (s->agent_r[m] == tr[n] && s->agent_c[m] == tc[n]) { ok[n] = 0; conflict = 1; }
+      if (moving[m] && tr[m] == tr[n] && tc[m] == tc[n]) { ok[n] = 0; conflict = 1; }
+    }
+    if (s->agent_level[n] > 0)
+      for (int f = 0; f < F; ++f)
+        if (!carried[f] && s->food_r[f] == tr[n] && s->food_c[f] == tc[n]) ok[n] = 0;
+  }
+  /* pick up / put down, at the start-of-step cell */
+  int new_carry[ORC_MAX_AGENTS];
+  for (int n = 0; n < N; ++n) {
+    new_carry[n] = s->agent_level[n];
+    if (actions[n] != 5) continue;
+    if (s->agent_level[n] == 0) {
+      for (int f = 0; f < F; ++f)
+        if (!carried[f] && s->food_r[f] == s->agent_r[n] && s->food_c[f] == s->agent_c[n]) new_carry[n] = 1 + f;
+    } else if (s->agent_r[n] != 0) {
+      new_carry[n] = 0;
+    }
+  }
+  for (int n = 0; n < N; ++n) {
+    s->agent_level[n] = new_carry[n];
+    if (ok[n]) {
+      s->agent_r[n] = tr[n]; s->agent_c[n] = tc[n];
+      if (s->agent_level[n] > 0) { s->food_r[s->agent_level[n] - 1] = tr[n]; s->food_c[s->agent_level[n] - 1] = tc[n]; }
+    }
+  }
+  int delivered_now[ORC_MAX_FOOD], d = 0;
+  for (int f = 0; f < F; ++f) delivered_now[f] = 0;
+  for (int n = 0; n < N; ++n) {
+    const int f = s->agent_level[n] - 1;
+    if (f >= 0 && s->agent_r[n] == 0 && s->food_level[f] == 2) { s->food_level[f] = 1; delivered_now[f] = 1; ++d; }
+  }
+  for (int k = 0; k < d; ++k) {
+    int n_idle = 0;
+    for (int f = 0; f < F; ++f) n_idle += (s->food_level[f] == 1 && !delivered_now[f]);
+    if (n_idle == 0) break;
+    uint32_t ctr[4] = {(uint32_t)k, (uint32_t)env, (uint32_t)s->episode, (uint32_t)s->step};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32) ^ ORC_DOMAIN_REQUEST};
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    uint32_t r = orc_bounded(out[0], (uint32_t)n_idle);
+    for (int f = 0; f < F; ++f) {
+      if (s->food_level[f] != 1 || delivered_now[f]) continue;
+      if (r == 0) { s->food_level[f] = 2; break; }
+      --r;
+    }
+  }
+  s->total_food_level += d;
+  *reward = (float)d;
+  s->step += 1;
+  *done = (uint8_t)((s->step >= cfg->episode_cap) || (cfg->env_kind == 2 && conflict));
+}
+
+/* The workload family selects the environment's three routines. */
+static void any_reset(const orc_config_t *cfg, uint64_t seed, int32_t env, int32_t episode, orc_env_state_t *s) {
+  if (cfg->env_kind == 0) orc_env_reset(cfg, seed, env, episode, s);
+  else orc_wh_reset(cfg, seed, env, episode, s);
+}
+static void any_observe(const orc_config_t *cfg, const orc_env_state_t *s, int32_t agent, float *obs) {
+  if (cfg->env_kind == 0) orc_env_observe(cfg, s, agent, obs);
+  else orc_wh_observe(cfg, s, agent, obs);
+}
+static void any_step(const orc_config_t *cfg, uint64_t seed, int32_t env, orc_env_state_t *s, const int32_t *actions,
+                     float *reward, uint8_t *done) {
+  if (cfg->env_kind == 0) orc_env_step(cfg, s, actions, reward, done);
+  else orc_wh_step(cfg, seed, env, s, actions, reward, done);
+}
+
+/* ------------------------------------------------------------------------- */
 /* MLP.  Dense layers follow the y = x W^T + b convention with W stored        */
 /* [out][in]; ReLU after both hidden layers, linear heads.  Parameter order    */
 /*   net_kind 0: W1[H][D] b1[H] W2[H][H] b2[H] Wa[6][H] ba[6] Wv[1][H] bv[1]   */
@@ -400,7 +599,7 @@ int orc_rollout(const orc_config_t *cfg, uint64_t seed, const float *params, int
     for (int t = 0; t <= T; ++t) {
       const size_t row0 = ((size_t)t * E_arr + p) * N; /* first agent row of (t, env) */
       if (obs || compute_mlp)
-        for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
+        for (int n = 0; n < N; ++n) any_observe(cfg, s, n, o + (size_t)n * D);
       if (t < T && obs) memcpy(obs + row0 * D, o, sizeof(float) * (size_t)N * D);
       if (compute_mlp) {
         orc_mlp_forward_env(cfg, params, o, emulate_bf16, lg, val);
@@ -426,10 +625,10 @@ int orc_rollout(const orc_config_t *cfg, uint64_t seed, const float *params, int
       }
       float reward;
       uint8_t done;
-      orc_env_step(cfg, s, act, &reward, &done);
+      any_step(cfg, seed, env, s, act, &reward, &done);
       if (rewards) for (int n = 0; n < N; ++n) rewards[row0 + n] = reward;
       if (dones) dones[(size_t)t * E_arr + p] = done;
-      if (done) orc_env_reset(cfg, seed, env, s->episode + 1, s);
+      if (done) any_reset(cfg, seed, env, s->episode + 1, s);
     }
   }
   free(o);
@@ -521,7 +720,7 @@ int orc_rollout_rec(const orc_config_t *cfg, uint64_t seed, const float *params,
     double *h = hidden + (size_t)i * N * H;
     for (int t = 0; t <= T; ++t) {
       const size_t row0 = ((size_t)t * n_local + (size_t)i) * N;
-      for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
+      for (int n = 0; n < N; ++n) any_observe(cfg, s, n, o + (size_t)n * D);
       if (t < T && obs) memcpy(obs + row0 * D, o, sizeof(float) * (size_t)N * D);
       if (t == T) {  /* bootstrap: on a copy of the state */
         memcpy(hb, h, sizeof(double) * (size_t)N * H);
@@ -547,11 +746,11 @@ int orc_rollout_rec(const orc_config_t *cfg, uint64_t seed, const float *params,
       }
       float reward;
       uint8_t done;
-      orc_env_step(cfg, s, act, &reward, &done);
+      any_step(cfg, seed, env, s, act, &reward, &done);
       if (rewards) for (int n = 0; n < N; ++n) rewards[row0 + n] = reward;
       if (dones) dones[(size_t)t * n_local + i] = done;
       if (done) {
-        orc_env_reset(cfg, seed, env, s->episode + 1, s);
+        any_reset(cfg, seed, env, s->episode + 1, s);
         for (int k = 0; k < N * H; ++k) h[k] = 0.0;  /* a new episode starts without memory */
       }
     }
@@ -597,7 +796,7 @@ int orc_evaluate(const orc_config_t *cfg, uint64_t seed, const float *params, in
     ep_count[i] = 0; ret_sum[i] = 0.0f; len_sum[i] = 0;
     for (int t = 0; t < T; ++t) {
       const size_t row0 = ((size_t)t * n_local + (size_t)i) * N;
-      for (int n = 0; n < N; ++n) orc_env_observe(cfg, s, n, o + (size_t)n * D);
+      for (int n = 0; n < N; ++n) any_observe(cfg, s, n, o + (size_t)n * D);
       orc_mlp_forward_env(cfg, params, o, emulate_bf16, lg, val);
       for (int n = 0; n < N; ++n) {
         const double *l = lg + n * ORC_N_ACTIONS;
@@ -618,7 +817,7 @@ int orc_evaluate(const orc_config_t *cfg, uint64_t seed, const float *params, in
       }
       float reward;
       uint8_t done;
-      orc_env_step(cfg, s, act, &reward, &done);
+      any_step(cfg, seed, env, s, act, &reward, &done);
       running += reward;
       length += 1;
       if (done) {
@@ -627,7 +826,7 @@ int orc_evaluate(const orc_config_t *cfg, uint64_t seed, const float *params, in
         len_sum[i] += length;
         running = 0.0f;
         length = 0;
-        orc_env_reset(cfg, seed, env, s->episode + 1, s);
+        any_reset(cfg, seed, env, s->episode + 1, s);
       }
     }
   }

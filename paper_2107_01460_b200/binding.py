@@ -18,6 +18,7 @@ MAVA_ERR_DEVICE_TIMEOUT = -4
 MAVA_ERR_CAPACITY = -5
 MAVA_NET_SHARED_TORSO = 0
 MAVA_NET_CENTRAL_CRITIC = 1
+MAVA_NET_RECURRENT = 2
 MAVA_PRECISION_FP32 = 0
 MAVA_PRECISION_BF16 = 1
 MAVA_FLAG_WRITE_LOGITS = 1
@@ -34,7 +35,7 @@ EXPORTS = [
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
     "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate", "mava_ppo_defaults", "mava_ppo_grad",
-    "mava_adam_step", "mava_ppo_grad_envs", "mava_debug_expire_next_wait",
+    "mava_adam_step", "mava_ppo_grad_envs", "mava_debug_expire_next_wait", "mava_rollout_get_hidden",
 ]
 
 
@@ -95,6 +96,7 @@ def lib():
         L.mava_ppo_grad.argtypes = [vp, vp, hpp, vp, vp]; L.mava_ppo_grad.restype = C.c_int
         L.mava_ppo_grad_envs.argtypes = [vp, vp, hpp, vp, C.c_int32, vp, vp]; L.mava_ppo_grad_envs.restype = C.c_int
         L.mava_adam_step.argtypes = [vp, vp, vp, vp, vp, C.c_int32, hpp]; L.mava_adam_step.restype = C.c_int
+        L.mava_rollout_get_hidden.argtypes = [vp, vp]; L.mava_rollout_get_hidden.restype = C.c_int
         L.mava_debug_expire_next_wait.argtypes = [vp, C.c_int32]; L.mava_debug_expire_next_wait.restype = C.c_int
         _lib = L
     return _lib
@@ -250,6 +252,14 @@ class Rollout:
         n = int(lib().mava_state_record_len(C.byref(self.cfg)))
         out = np.empty((self.cfg.n_envs, n), dtype=np.int32)
         _check(lib().mava_rollout_get_state(self.handle, out.ctypes.data), "mava_rollout_get_state")
+        return out
+
+    def get_hidden(self):
+        """Recurrent policy: the hidden vectors the next run starts from, [E][N][H] float32 (numpy)."""
+        import numpy as np
+
+        out = np.empty((self.cfg.n_envs, self.cfg.n_agents, self.cfg.hidden), dtype=np.float32)
+        _check(lib().mava_rollout_get_hidden(self.handle, out.ctypes.data), "mava_rollout_get_hidden")
         return out
 
     def set_state(self, records):

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmava_rollout.so")
-SOURCES = ["api.cu", "rollout_simt.cu", "rollout_tc.cu", "critic_tc.cu", "gae.cu", "update.cu", "update_tc.cu", "update_tc256.cu"]
+SOURCES = ["api.cu", "rollout_simt.cu", "rollout_tc.cu", "critic_tc.cu", "gae.cu", "update.cu", "update_tc.cu", "update_tc256.cu", "rollout_rec.cu", "rollout_rec_tc.cu"]
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

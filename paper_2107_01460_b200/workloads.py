@@ -45,6 +45,18 @@ WORKLOADS = {
     "rec2_10x10_3p3f_gru64": dict(
         grid=10, n_agents=3, n_food=3, max_agent_level=3, view_radius=2, episode_cap=100,
         hidden=64, net_kind=2, n_envs=8192, T=128, seed=12, precision="bf16"),
+    # Warehouse workloads (Section 4, "Multi-Robot Warehouse"): env_kind 1, or 2 for the variant whose episode ends when
+    # two robots get in each other's way; n_food is the number of shelves.  Observations, actions and networks are
+    # those of the foraging shapes with the same agent count.
+    "wh0_tiny_8x8_2r2s_h64": dict(
+        grid=8, n_agents=2, n_food=2, max_agent_level=2, view_radius=2, episode_cap=50, env_kind=1,
+        hidden=64, net_kind=0, n_envs=16, T=32, seed=20, precision="bf16"),
+    "wh1_10x10_3r3s_h128": dict(
+        grid=10, n_agents=3, n_food=3, max_agent_level=3, view_radius=2, episode_cap=100, env_kind=1,
+        hidden=128, net_kind=0, n_envs=8192, T=128, seed=21, precision="bf16"),
+    "wh2_10x10_3r3s_h128_collisions_end": dict(
+        grid=10, n_agents=3, n_food=3, max_agent_level=3, view_radius=2, episode_cap=100, env_kind=2,
+        hidden=128, net_kind=0, n_envs=8192, T=128, seed=22, precision="bf16"),
 }
 WORKLOAD_NAMES = list(WORKLOADS)
 GAMMA = 0.99
@@ -53,7 +65,7 @@ LAMBDA = 0.95
 
 def workload(name_or_index) -> dict:
     """A copy of one workload description, by name or by index (0..4: the five feed-forward shapes; 5..7: the
-    recurrent variants)."""
+    recurrent variants; 8..10: the warehouse workloads)."""
     if isinstance(name_or_index, int):
         name_or_index = WORKLOAD_NAMES[name_or_index]
     w = dict(WORKLOADS[name_or_index])

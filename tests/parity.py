@@ -149,3 +149,70 @@ def check_against_oracle(w, ro, params, T, precision, mlp_env_ids, obs_env_ids=N
     out["ret"] = float(np.max(np.abs(g["ret"] - ret) / (GAE_TOL * np.maximum(1.0, np.abs(ret)))))
     assert out["adv"] <= 1.0 and out["ret"] <= 1.0, out
     return out
+
+
+def check_recurrent_against_oracle(w, ro, params, T, precision, ids, hidden0=None, t_global0=0, states0=None):
+    """A finished run of a recurrent-policy handle against the oracle replaying the GPU's actions: environment arrays
+    bit for bit (all environments), logits / values / log-probabilities / final hidden vectors of the environments
+    `ids` within the path's tolerance, sampled actions by the margin rule, the sampler exactly on the GPU's own logits."""
+    E, N = ro.cfg.n_envs, ro.cfg.n_agents
+    seed = w["seed"]
+    ocfg = oracle.make_config(w)
+    tol = TOL[precision]
+    g = {k: getattr(ro, k)[:T].cpu().numpy() for k in ("actions", "logp", "rewards", "dones")}
+    g["values"] = ro.values[:T + 1].cpu().numpy()
+    g["logits"] = ro.logits[:T].cpu().numpy()
+    env = oracle_rollout_threaded(ocfg, seed, None, T, np.arange(E, dtype=np.int32), g["actions"], states=states0, compute_mlp=False,
+                                  want_obs=False, t_global0=t_global0)
+    assert np.array_equal(env.rewards.view(np.uint32), g["rewards"].view(np.uint32)), "rewards differ"
+    assert np.array_equal(env.dones, g["dones"]), "dones differ"
+    ids = np.asarray(ids, dtype=np.int32)
+    import torch
+
+    g_obs = ro.obs[:T].index_select(1, torch.from_numpy(ids.astype(np.int64)).cuda()).cpu().numpy()
+    out = {}
+    for emulate in ([False, True] if precision == binding.MAVA_PRECISION_BF16 else [False]):
+        cuts = np.array_split(np.arange(ids.size), min(os.cpu_count() or 1, ids.size))
+        parts = [None] * len(cuts)
+
+        def work(i):
+            c = cuts[i]
+            parts[i] = oracle.rollout_rec(ocfg, seed, params, T, ids[c], forced_actions=g["actions"][:, ids[c]],
+                                          states=None if states0 is None else [states0[j] for j in ids[c]],
+                                          hidden=None if hidden0 is None else hidden0[ids[c]], t_global0=t_global0,
+                                          emulate_bf16=emulate)
+
+        threads = [threading.Thread(target=work, args=(i,)) for i in range(len(cuts))]
+        for th in threads:
+            th.start()
+        for th in threads:
+            th.join()
+        cat = lambda name: np.concatenate([getattr(p[0], name) for p in parts], axis=1)  # noqa: E731
+        ref_hidden = np.concatenate([p[1] for p in parts], axis=0)
+        t_ = TOL_BF16_OPERANDS if emulate else tol
+        tag = "_bf16_operands" if emulate else ""
+        if not emulate:
+            assert np.array_equal(cat("obs").view(np.uint32), g_obs.view(np.uint32)), "obs differ"
+        out["logits" + tag] = close(g["logits"][:, ids], cat("logits"), t_)
+        out["values" + tag] = close(g["values"][:, ids], cat("values"), t_)
+        out["logp" + tag] = close(g["logp"][:, ids], cat("logp"), t_)
+        out["hidden" + tag] = close(ro.get_hidden()[ids], ref_hidden, t_)
+        assert max(out["logits" + tag], out["values" + tag], out["logp" + tag], out["hidden" + tag]) <= 1.0, out
+        eps = 4.0 * t_ * (1.0 + np.max(np.abs(cat("logits")), axis=-1))
+        differ = g["actions"][:, ids] != cat("own_actions")
+        assert not np.any(differ & (cat("margin") > eps)), "an action differs away from a CDF boundary"
+        out["excused_actions" + tag] = int(differ.sum())
+        assert differ.sum() <= max(2, int(10 * t_ * differ.size)), out
+    lg = g["logits"][:, ids].astype(np.float64)
+    for t in range(T):
+        for i, e in enumerate(ids):
+            for n in range(N):
+                u = oracle.lib().orc_action_uniform(seed, t_global0 + t, int(e), n)
+                a, lp, m = oracle.sample(lg[t, i, n], u)
+                if a != g["actions"][t, e, n]:
+                    assert m < 1e-5, ("sampler disagrees with its own logits", t, e, n, m)
+                assert abs(lp[g["actions"][t, e, n]] - g["logp"][t, e, n]) <= 1e-5 * (1 + abs(lp[a]))
+    adv, ret = oracle.gae(g["values"], g["rewards"], g["dones"], float(np.float32(wl.GAMMA)), float(np.float32(wl.LAMBDA)))
+    assert np.max(np.abs(ro.adv[:T].cpu().numpy() - adv) / (GAE_TOL * np.maximum(1.0, np.abs(adv)))) <= 1.0
+    assert np.max(np.abs(ro.ret[:T].cpu().numpy() - ret) / (GAE_TOL * np.maximum(1.0, np.abs(ret)))) <= 1.0
+    return out
