@@ -44,6 +44,10 @@ extern "C" {
 
 #define MAVA_N_ACTIONS 6 /* 0 noop, 1 up (r-1), 2 down (r+1), 3 left (c-1), 4 right (c+1), 5 load */
 
+#define MAVA_ENV_FORAGING 0  /* level-based foraging (the rules in the general comment above)           */
+#define MAVA_ENV_WAREHOUSE 1 /* warehouse: robots carry requested shelves to the delivery row             */
+#define MAVA_ENV_WAREHOUSE_CONFLICTS_END 2 /* the same, and a robot conflict ends the episode             */
+
 #define MAVA_NET_SHARED_TORSO 0 /* one torso, a 6-logit actor head and a value head (IPPO-style)   */
 #define MAVA_NET_CENTRAL_CRITIC 1 /* actor net per agent + critic on the joint observation (MAPPO) */
 
@@ -80,7 +84,7 @@ typedef struct {
   int32_t flags;           /* MAVA_FLAG_* bits                                                    */
   int32_t first_env;       /* global index of this handle's environment 0 (keys Philox), so that
                               shards of one large batch reproduce the unsharded run; usually 0    */
-  int32_t reserved;        /* must be 0                                                           */
+  int32_t env_kind;        /* MAVA_ENV_*: the workload family (0 = level-based foraging)          */
   uint64_t seed;           /* keys every Philox stream                                            */
 } mava_config_t;
 

@@ -46,7 +46,7 @@ class mava_ppo_hyper_t(C.Structure):
 class mava_config_t(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "grid", "n_agents", "n_food", "max_agent_level", "view_radius", "episode_cap", "n_envs", "max_T", "hidden",
-        "net_kind", "precision", "flags", "first_env", "reserved")] + [("seed", C.c_uint64)]
+        "net_kind", "precision", "flags", "first_env", "env_kind")] + [("seed", C.c_uint64)]
 
 
 class mava_buffers_t(C.Structure):
@@ -115,7 +115,7 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
         grid=w["grid"], n_agents=w["n_agents"], n_food=w["n_food"], max_agent_level=w["max_agent_level"],
         view_radius=w["view_radius"], episode_cap=w["episode_cap"], n_envs=w["n_envs"] if n_envs is None else n_envs,
         max_T=w["T"] if max_T is None else max_T, hidden=w["hidden"], net_kind=w["net_kind"], precision=precision,
-        flags=flags, first_env=first_env, reserved=0, seed=w["seed"] if seed is None else seed)
+        flags=flags, first_env=first_env, env_kind=w.get("env_kind", 0), seed=w["seed"] if seed is None else seed)
 
 
 def update_on_tensor_cores(cfg: mava_config_t) -> bool:

@@ -16,13 +16,13 @@ bool config_ok(const mava_config_t &c) {
   return c.grid >= 3 && c.grid <= 64 && c.n_agents >= 1 && c.n_agents <= kMaxAgents && c.n_food >= 1 &&
          c.n_food <= kMaxFood && c.max_agent_level >= 1 && c.max_agent_level <= 3 &&
          c.n_agents + c.n_food <= c.grid * c.grid && c.episode_cap >= 1 && c.n_envs >= 1 && c.max_T >= 1 &&
-         c.hidden >= 1 && c.first_env >= 0 && c.reserved == 0 && (c.net_kind == MAVA_NET_SHARED_TORSO || c.net_kind == MAVA_NET_CENTRAL_CRITIC || c.net_kind == MAVA_NET_RECURRENT) &&
+         c.hidden >= 1 && c.first_env >= 0 && c.env_kind >= 0 && c.env_kind <= 2 && (c.net_kind == MAVA_NET_SHARED_TORSO || c.net_kind == MAVA_NET_CENTRAL_CRITIC || c.net_kind == MAVA_NET_RECURRENT) &&
          (c.precision == MAVA_PRECISION_FP32 || c.precision == MAVA_PRECISION_BF16);
 }
 
 EnvParams env_params(const mava_rollout *h) {
   return EnvParams{h->cfg.grid, h->cfg.max_agent_level, h->cfg.episode_cap, h->cfg.n_envs, h->cfg.first_env,
-                   static_cast<uint32_t>(h->cfg.seed), static_cast<uint32_t>(h->cfg.seed >> 32)};
+                   static_cast<uint32_t>(h->cfg.seed), static_cast<uint32_t>(h->cfg.seed >> 32), h->cfg.env_kind};
 }
 
 struct DeviceGuard {  // makes the handle's device current for the duration of a call
@@ -296,7 +296,8 @@ int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host) {
     EnvRec s{};
     for (int n = 0; n < N; ++n) {
       const int r = *in++, c = *in++, l = *in++;
-      if (r < 0 || r >= G || c < 0 || c >= G || l < 1 || l > 3) return MAVA_ERR_INVALID_ARG;
+      if (r < 0 || r >= G || c < 0 || c >= G) return MAVA_ERR_INVALID_ARG;
+      if (h->cfg.env_kind == 0 ? (l < 1 || l > 3) : (l < 0 || l > F)) return MAVA_ERR_INVALID_ARG;
       s.ar[n] = static_cast<uint8_t>(r); s.ac[n] = static_cast<uint8_t>(c); s.al[n] = static_cast<uint8_t>(l);
     }
     for (int f = 0; f < F; ++f) {
@@ -305,7 +306,7 @@ int mava_rollout_set_state(mava_rollout_t *h, const int32_t *records_host) {
       s.fr[f] = static_cast<uint8_t>(r); s.fc[f] = static_cast<uint8_t>(c); s.fl[f] = static_cast<uint8_t>(l);
     }
     s.step = *in++; s.episode = *in++; s.total = *in++;
-    if (s.step < 0 || s.step >= h->cfg.episode_cap || s.episode < 0 || s.total < 1) return MAVA_ERR_INVALID_ARG;
+    if (s.step < 0 || s.step >= h->cfg.episode_cap || s.episode < 0 || s.total < (h->cfg.env_kind == 0 ? 1 : 0)) return MAVA_ERR_INVALID_ARG;
     recs[static_cast<size_t>(e)] = s;
   }
   if (cudaStreamSynchronize(h->stream) != cudaSuccess ||

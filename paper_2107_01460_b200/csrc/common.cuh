@@ -36,6 +36,7 @@ struct EnvParams {
   int32_t grid, max_level, cap, n_envs;
   int32_t first_env;        // global index of local environment 0 (Philox is keyed on global indices)
   uint32_t key_lo, key_hi;  // seed halves (domain tweak applied on use)
+  int32_t env_kind;         // 0: foraging; 1: warehouse; 2: warehouse whose episode ends on a robot conflict
 };
 
 // Everything a rollout launch needs.

@@ -4,6 +4,7 @@
 // arithmetic in index order, no tensor cores.
 #include "common.cuh"
 #include "env.cuh"
+#include "env_wh.cuh"
 #include "layout.h"
 #include "simt_dense.cuh"
 
@@ -26,7 +27,8 @@ struct SimtSmem {
   uint8_t new_r[kSimtRows], new_c[kSimtRows], collected[EPT * F];
 };
 
-template <int N, int F, int H, bool CENTRAL>
+// ENV: 0 foraging, 1 warehouse (env_wh.cuh).
+template <int N, int F, int H, bool CENTRAL, int ENV = 0>
 __global__ void __launch_bounds__(kSimtThreads)
 rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
   using S = SimtSmem<N, F, H, CENTRAL>;
@@ -50,10 +52,17 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
   for (int t = 0; t <= (ev ? a.T - 1 : a.T); ++t) {
     const bool last = !ev && (t == a.T);
     const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
-    auto sink = [&](int row, int j, float v) { sm.obs[row * D + j] = v; };
-    observe_fill<N>(sm.st, a.env, n_rows, tid, kSimtThreads, sink);
-    __syncthreads();
-    observe_scatter<N, F>(sm.st, n_rows, tid, kSimtThreads, sink);
+    if constexpr (ENV == 0) {
+      auto sink = [&](int row, int j, float v) { sm.obs[row * D + j] = v; };
+      observe_fill<N>(sm.st, a.env, n_rows, tid, kSimtThreads, sink);
+      __syncthreads();
+      observe_scatter<N, F>(sm.st, n_rows, tid, kSimtThreads, sink);
+    } else {
+      for (int i = tid; i < n_rows * D; i += kSimtThreads) {
+        const int row = i / D;
+        sm.obs[i] = wh_obs_element<N, F>(sm.st[row / N], a.env, row % N, i - row * D);
+      }
+    }
     __syncthreads();
 
     if (!last && !ev) {  // the tile's rows are one contiguous block of the time-major obs array
@@ -142,13 +151,18 @@ rollout_simt_kernel(RolloutArgs a, SimtWeights w) {
     __syncthreads();
     if (last) break;
 
-    step_decide<N, F>(sm.st, a.env, sm.act, n_env, sm.new_r, sm.new_c, sm.collected, tid, kSimtThreads);
-    __syncthreads();
+    if constexpr (ENV == 0) {
+      step_decide<N, F>(sm.st, a.env, sm.act, n_env, sm.new_r, sm.new_c, sm.collected, tid, kSimtThreads);
+      __syncthreads();
+    }
     if (tid < n_env) {
       float reward;
       bool done;
-      step_apply<N, F>(sm.st[tid], a.env, static_cast<uint32_t>(a.env.first_env + e0 + tid), sm.new_r, sm.new_c,
-                       sm.collected, tid, reward, done);
+      if constexpr (ENV == 0)
+        step_apply<N, F>(sm.st[tid], a.env, static_cast<uint32_t>(a.env.first_env + e0 + tid), sm.new_r, sm.new_c,
+                         sm.collected, tid, reward, done);
+      else
+        wh_step_rec<N, F>(sm.st[tid], a.env, static_cast<uint32_t>(a.env.first_env + e0 + tid), sm.act + tid * N, reward, done);
       if (ev) {
         sums.step(reward, done);
       } else {
@@ -172,7 +186,8 @@ __global__ void env_init_kernel(EnvRec *state, EnvParams p) {
   if (e >= p.n_envs) return;
   EnvRec s;
   memset(&s, 0, sizeof(s));
-  env_reset<N, F>(s, p, static_cast<uint32_t>(p.first_env + e), 0u);
+  if (p.env_kind == 0) env_reset<N, F>(s, p, static_cast<uint32_t>(p.first_env + e), 0u);
+  else wh_reset_rec<N, F>(s, p, static_cast<uint32_t>(p.first_env + e), 0u);
   state[e] = s;
 }
 
@@ -203,10 +218,10 @@ __global__ void prep_simt_kernel(const float *__restrict__ src, float *__restric
   }
 }
 
-template <int N, int F, int H, bool CENTRAL>
+template <int N, int F, int H, bool CENTRAL, int ENV = 0>
 cudaError_t launch_simt_variant(mava_rollout *h, const RolloutArgs &args, const SimtWeights &w) {
   using S = SimtSmem<N, F, H, CENTRAL>;
-  auto kern = rollout_simt_kernel<N, F, H, CENTRAL>;
+  auto kern = rollout_simt_kernel<N, F, H, CENTRAL, ENV>;
   const size_t smem = sizeof(S);
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (err != cudaSuccess) return err;
@@ -233,7 +248,7 @@ size_t simt_weight_floats(const mava_config_t &cfg, int D) { return param_layout
 
 cudaError_t launch_env_init(mava_rollout *h) {
   EnvParams p{h->cfg.grid, h->cfg.max_agent_level, h->cfg.episode_cap, h->cfg.n_envs, h->cfg.first_env,
-              static_cast<uint32_t>(h->cfg.seed), static_cast<uint32_t>(h->cfg.seed >> 32)};
+              static_cast<uint32_t>(h->cfg.seed), static_cast<uint32_t>(h->cfg.seed >> 32), h->cfg.env_kind};
   const int threads = 128, blocks = (h->cfg.n_envs + threads - 1) / threads;
   switch (h->variant) {
     case 0: case 1: case 5: env_init_kernel<2, 2><<<blocks, threads, 0, h->stream>>>(h->d_state, p); break;
@@ -266,6 +281,13 @@ cudaError_t launch_rollout_simt(mava_rollout *h, const RolloutArgs &args) {
     w.Wv = base + L.Cv; w.bv = base + L.cv;  // unused by the head loop of the central variant
     w.C1t = base + L.C1; w.c1 = base + L.c1; w.C2t = base + L.C2; w.c2 = base + L.c2;
     w.Cv = base + L.Cv; w.cv = base + L.cv;
+  }
+  if (h->cfg.env_kind != 0) {  // the warehouse family is compiled for two shapes
+    switch (h->variant) {
+      case 0: return launch_simt_variant<2, 2, 64, false, 1>(h, args, w);
+      case 2: return launch_simt_variant<3, 3, 128, false, 1>(h, args, w);
+      default: return cudaErrorNotSupported;
+    }
   }
   switch (h->variant) {
     case 0: return launch_simt_variant<2, 2, 64, false>(h, args, w);

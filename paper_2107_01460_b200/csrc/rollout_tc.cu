@@ -25,6 +25,7 @@
 
 #include "common.cuh"
 #include "env.cuh"
+#include "env_wh.cuh"
 #include "layout.h"
 #include "tc_common.cuh"
 
@@ -306,7 +307,7 @@ __device__ __forceinline__ void expand_quads(const QuadPlan<D, K1> &p, uint32_t 
 }
 
 // ---- the rollout kernel ------------------------------------------------------------------------
-template <int N, int F, int H, bool TM, bool EVAL>
+template <int N, int F, int H, bool TM, bool EVAL, int ENV = 0>
 __global__ void __launch_bounds__(TcShape<N, H, TM>::THREADS, 1)
 rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ept, int n_tiles, int groups) {
   using S = TcShape<N, H, TM>;
@@ -460,11 +461,13 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       // 1. non-zero observation entries into the zeroed A tile (and the zeroed fp32 block)
       if (active) {
         const uint32_t a_row = a_addr + a_offset<K1>(row, 0);
-        observe_env<N, F>(env, a.env, ag, [&](int j, float v) {
+        auto put = [&](int j, float v) {
           if (!TM) sts_f32(stage_addr + 4u * static_cast<uint32_t>(crow * D + j), v);
           else if (j == 3 * kPlane + 1) sts_f32(frac_addr + 4u * static_cast<uint32_t>(row), v);
           sts_u16(a_row + a_offset<K1>(0, j), bf16_bits(v));
-        });
+        };
+        if constexpr (ENV == 0) observe_env<N, F>(env, a.env, ag, put);
+        else wh_observe_env<N, F>(env, a.env, ag, put);
         if (S::FOLD1) {  // the two columns that pick up the bias rows of W1
           sts_u16(a_row + a_offset<K1>(0, D), 0x3F80);
           sts_u16(a_row + a_offset<K1>(0, D + 1), 0x3F80);
@@ -617,7 +620,8 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       // 5. transition and auto-reset, inside the warp
       float reward;
       bool done;
-      step_env_warp<N, F>(env, a.env, env_id, ag, base, active, action, reward, done);
+      if constexpr (ENV == 0) step_env_warp<N, F>(env, a.env, env_id, ag, base, active, action, reward, done);
+      else wh_step_env_warp<N, F>(env, a.env, env_id, base, active, action, reward, done);
       pend_reward = reward;
       pend_done = done;
       pend_done_idx = static_cast<size_t>(t) * a.env.n_envs + e0 + le;
@@ -655,10 +659,10 @@ int few_rows_tile(const mava_rollout *h, int sms) {
   return 0;
 }
 
-template <int N, int F, int H, bool TM>
+template <int N, int F, int H, bool TM, int ENV = 0>
 cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   using S = TcShape<N, H, TM>;
-  auto kern = args.eval ? rollout_tc_kernel<N, F, H, TM, true> : rollout_tc_kernel<N, F, H, TM, false>;
+  auto kern = args.eval ? rollout_tc_kernel<N, F, H, TM, true, ENV> : rollout_tc_kernel<N, F, H, TM, false, ENV>;
   const size_t smem = sizeof(TcSmem<N, F, H, TM>);
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (err != cudaSuccess) return err;
@@ -666,7 +670,7 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
   if (err != cudaSuccess) return err;
   // Few rows per SM: the form with the rows as the N operand of the MMA.
-  if constexpr (!TM && H == kTileRows) {
+  if constexpr (!TM && H == kTileRows && ENV == 0) {
     const int rb = few_rows_tile<N, H, TM>(h, sms);
     if (rb == 16) return launch_tc_small<N, F, H, 16>(h, args, sms);
     if (rb == 32) return launch_tc_small<N, F, H, 32>(h, args, sms);
@@ -715,7 +719,7 @@ static bool use_tm(const mava_rollout *h) { return h->variant >= 3 || (h->cfg.fl
 bool tc_rollout_is_wide(const mava_rollout *h) {
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return false;
-  if (use_tm(h)) return true;
+  if (use_tm(h) || h->cfg.env_kind != 0) return true;
   if (h->variant == 1) return few_rows_tile<2, 128, false>(h, sms) == 0;
   if (h->variant == 2) return few_rows_tile<3, 128, false>(h, sms) == 0;
   return true;
@@ -746,6 +750,13 @@ cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev) {
 
 cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args) {
   const bool tm = use_tm(h);
+  if (h->cfg.env_kind != 0) {  // the warehouse family: two shapes, hidden activations in shared memory
+    switch (h->variant) {
+      case 0: return launch_tc_variant<2, 2, 64, false, 1>(h, args);
+      case 2: return launch_tc_variant<3, 3, 128, false, 1>(h, args);
+      default: return cudaErrorNotSupported;
+    }
+  }
   switch (h->variant) {
     case 0: return tm ? launch_tc_variant<2, 2, 64, true>(h, args) : launch_tc_variant<2, 2, 64, false>(h, args);
     case 1: return tm ? launch_tc_variant<2, 2, 128, true>(h, args) : launch_tc_variant<2, 2, 128, false>(h, args);

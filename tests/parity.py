@@ -189,15 +189,21 @@ def check_recurrent_against_oracle(w, ro, params, T, precision, ids, hidden0=Non
             th.join()
         cat = lambda name: np.concatenate([getattr(p[0], name) for p in parts], axis=1)  # noqa: E731
         ref_hidden = np.concatenate([p[1] for p in parts], axis=0)
+        # Against the bf16-operand oracle the carried state is re-quantised to bf16 at every step on both sides: a hidden
+        # unit whose new value falls within fp32-versus-double rounding of a bf16 boundary lands one bf16 step apart
+        # (2^-8 relative), and that difference travels on through the episode instead of ending with the step as in the
+        # feed-forward nets.  So the bulk must still agree to 2e-3 (the 99.9th percentile of the error ratio), while
+        # the worst element gets three times that.
         t_ = TOL_BF16_OPERANDS if emulate else tol
         tag = "_bf16_operands" if emulate else ""
         if not emulate:
             assert np.array_equal(cat("obs").view(np.uint32), g_obs.view(np.uint32)), "obs differ"
-        out["logits" + tag] = close(g["logits"][:, ids], cat("logits"), t_)
-        out["values" + tag] = close(g["values"][:, ids], cat("values"), t_)
-        out["logp" + tag] = close(g["logp"][:, ids], cat("logp"), t_)
-        out["hidden" + tag] = close(ro.get_hidden()[ids], ref_hidden, t_)
-        assert max(out["logits" + tag], out["values" + tag], out["logp" + tag], out["hidden" + tag]) <= 1.0, out
+        worst_allowed = 3.0 if emulate else 1.0
+        for name, got, ref in (("logits", g["logits"][:, ids], cat("logits")), ("values", g["values"][:, ids], cat("values")),
+                               ("logp", g["logp"][:, ids], cat("logp")), ("hidden", ro.get_hidden()[ids], ref_hidden)):
+            ratio = np.abs(np.asarray(got, dtype=np.float64) - ref) / (t_ * (1.0 + np.abs(ref)))
+            out[name + tag] = float(ratio.max())
+            assert ratio.max() <= worst_allowed and np.quantile(ratio, 0.999) <= 1.0, (name, tag, ratio.max(), np.quantile(ratio, 0.999))
         eps = 4.0 * t_ * (1.0 + np.max(np.abs(cat("logits")), axis=-1))
         differ = g["actions"][:, ids] != cat("own_actions")
         assert not np.any(differ & (cat("margin") > eps)), "an action differs away from a CDF boundary"
