@@ -353,24 +353,29 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
 }
 
 // ---- weight kernel ---------------------------------------------------------------------------------------------------
-// CTAs [0, n_w2) sum d W2 and d b2; the others d W1, d b1 and d Wh.  A CTA's work items are half tiles (64 rows) of
-// the tiles it owns; an item's operands come in by bulk copies into a ring of stages.
-constexpr int kHalfRows = 64;
-constexpr uint32_t kQ = 16384;                                // 64 rows of a [128][128] unit-half tile
-constexpr uint32_t kW2Stage = 4 * kQ, kW2Stages = 3;          // d z2 (two unit halves), h1 (two unit halves)
-constexpr uint32_t kXHalf = kHalfRows * kK1 * 2, kDhHalf = kHalfRows * kHeads * 2;
-constexpr uint32_t kW1Stage = 4 * kQ + kXHalf + kDhHalf, kW1Stages = 2;  // d z1, h2 (two unit halves each), x, dhead
+// CTAs [0, n_w2) sum d W2 and d b2; the others d W1, d b1 and d Wh.  A CTA's work items are 32-row pieces of the tiles it
+// owns; an item's operands come in by bulk copies into a ring of stages.  Roles inside the CTA, connected by mbarriers
+// only: one producer thread (copies), one MMA thread, eight consumer warps (thread j sums column j of the d z tile for
+// the bias gradient).  A stage is free again when its MMAs have completed and every consumer warp has let go of it.
+constexpr int kItemRows = 32;
+constexpr int kItemsPerTile = kR / kItemRows;
+constexpr uint32_t kQ = kItemRows * 128 * 2;                  // an item's rows of a [128][128] unit-half tile: 8 KB
+constexpr uint32_t kW2Stage = 4 * kQ, kW2Stages = 6;          // d z2 (two unit halves), h1 (two unit halves)
+constexpr uint32_t kXPart = kItemRows * kK1 * 2, kDhPart = kItemRows * kHeads * 2;
+constexpr uint32_t kW1Stage = 4 * kQ + kXPart + kDhPart, kW1Stages = 5;  // d z1, h2 (two unit halves each), x, dhead
 constexpr uint32_t kRingBytes = kW2Stage * kW2Stages > kW1Stage * kW1Stages ? kW2Stage * kW2Stages : kW1Stage * kW1Stages;
+constexpr int kMaxStages = 6;
+constexpr int kWgtThreads = 320, kConsumerWarps = 8;
 
 struct WgtSmem {
   alignas(128) unsigned char ring[kRingBytes];
-  alignas(8) uint64_t full[3], empty[3], done;
+  alignas(8) uint64_t full[kMaxStages], empty[kMaxStages], done;
   uint32_t tmem_base;
 };
 
 struct WgtOffsets { size_t W1, b1, W2, b2, Wa, Wv; };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kWgtThreads, 1)
 ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, int n_w2, float *__restrict__ partial, size_t n_params,
                       int *status, WgtOffsets off, int D, int has_value) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -384,9 +389,9 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
   const uint32_t ring = smem_u32(sm.ring), full0 = smem_u32(&sm.full[0]), empty0 = smem_u32(&sm.empty[0]), done_bar = smem_u32(&sm.done);
   constexpr uint32_t kCols = 512;
   if (tid == 0) {
-    for (int s = 0; s < 3; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(full0 + 8u * s, 1);
-      mbar_init(empty0 + 8u * s, 1 + kThreads / 32);  // the MMAs' commit and every warp's column sums
+      mbar_init(empty0 + 8u * s, 1 + kConsumerWarps);  // the MMAs' commit and every consumer warp
     }
     mbar_init(done_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -400,75 +405,87 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   const int my_tiles = rank < n_tiles ? (n_tiles - rank + peers - 1) / peers : 0;
-  const int n_items = 2 * my_tiles;
-  auto request = [&](int u) {  // thread 0: item u into stage u % S
-    const int lt = rank + (u >> 1) * peers, rh = u & 1;
-    const unsigned char *st = staging + static_cast<size_t>(lt) * kStTile;
-    const uint32_t dst = ring + static_cast<uint32_t>(u % S) * stage_bytes, bar = full0 + 8u * (u % S);
-    mbar_expect_tx(bar, stage_bytes);
-    const size_t a = role_w2 ? kStDz2 : kStDz1, b = role_w2 ? kStH1 : kStH2;
-    bulk_load(dst, st + a + static_cast<size_t>(rh) * kQ, kQ, bar);
-    bulk_load(dst + kQ, st + a + kHalfBytes + static_cast<size_t>(rh) * kQ, kQ, bar);
-    bulk_load(dst + 2 * kQ, st + b + static_cast<size_t>(rh) * kQ, kQ, bar);
-    bulk_load(dst + 3 * kQ, st + b + kHalfBytes + static_cast<size_t>(rh) * kQ, kQ, bar);
-    if (!role_w2) {
-      bulk_load(dst + 4 * kQ, st + kStX + static_cast<size_t>(rh) * kXHalf, kXHalf, bar);
-      bulk_load(dst + 4 * kQ + kXHalf, st + kStDh + static_cast<size_t>(rh) * kDhHalf, kDhHalf, bar);
-    }
-  };
+  const int n_items = kItemsPerTile * my_tiles;
   bool timed_out = false;
-  int issued = 0;
-  if (tid == 0)
-    for (; issued < S && issued < n_items; ++issued) request(issued);
-  float db = 0.0f;  // thread j: bias gradient of out unit j (d b2 or d b1)
-  const uint32_t my_col = static_cast<uint32_t>(tid >> 7) * kQ + static_cast<uint32_t>(((tid & 127) >> 3) * 128 + (tid & 7) * 2);
-#pragma unroll 1
-  for (int u = 0; u < n_items; ++u) {
-    const int s = u % S;
-    const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
-    timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
-    if (__syncthreads_or(timed_out)) { timed_out = true; break; }
-    if (tid == 0) {
-      tc_fence_after();
-      const uint32_t keep = u > 0 ? 1u : 0u;
-      if (role_w2) {  // d W2 [out half a][in half b] += d z2[:, a]^T . h1[:, b] over the item's 64 rows
-#pragma unroll
-        for (int k = 0; k < kHalfRows / 16; ++k)
-#pragma unroll
-          for (int ab = 0; ab < 4; ++ab)
-            mma_bf16(tmem + static_cast<uint32_t>(ab * 128), desc_mn(base + (ab >> 1) * kQ, 128, k), desc_mn(base + 2 * kQ + (ab & 1) * kQ, 128, k),
-                     instr_desc(128, 128) | kAmn | kBmn, keep | (k > 0));
-      } else {        // d W1 [out half a][in] += d z1[:, a]^T . x;  d Wh^T [unit half a][head] += h2[:, a]^T . dhead
-#pragma unroll
-        for (int k = 0; k < kHalfRows / 16; ++k)
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * kQ, 128, k), desc_mn(base + 4 * kQ, kK1, k),
-                     instr_desc(128, kK1) | kAmn | kBmn, keep | (k > 0));
-            mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * kQ, 128, k), desc_mn(base + 4 * kQ + kXHalf, kHeads, k),
-                     instr_desc(128, kHeads) | kAmn | kBmn, keep | (k > 0));
-          }
+  float db = 0.0f;  // consumer thread j: bias gradient of out unit j (d b2 or d b1)
+
+  if (warp == kConsumerWarps) {
+    // ---- producer
+    if (lane == 0) {
+      int issued = 0;
+      for (int u = 0; u < n_items && !timed_out; ++u) {
+        const int s = u % S;
+        if (u >= S) timed_out |= !mbar_wait(empty0 + 8u * s, ((u / S) - 1) & 1);
+        if (timed_out) break;
+        const int lt = rank + (u / kItemsPerTile) * peers, q = u % kItemsPerTile;
+        const unsigned char *st = staging + static_cast<size_t>(lt) * kStTile;
+        const uint32_t dst = ring + static_cast<uint32_t>(s) * stage_bytes, bar = full0 + 8u * s;
+        mbar_expect_tx(bar, stage_bytes);
+        const size_t a = role_w2 ? kStDz2 : kStDz1, b = role_w2 ? kStH1 : kStH2;
+        bulk_load(dst, st + a + static_cast<size_t>(q) * kQ, kQ, bar);
+        bulk_load(dst + kQ, st + a + kHalfBytes + static_cast<size_t>(q) * kQ, kQ, bar);
+        bulk_load(dst + 2 * kQ, st + b + static_cast<size_t>(q) * kQ, kQ, bar);
+        bulk_load(dst + 3 * kQ, st + b + kHalfBytes + static_cast<size_t>(q) * kQ, kQ, bar);
+        if (!role_w2) {
+          bulk_load(dst + 4 * kQ, st + kStX + static_cast<size_t>(q) * kXPart, kXPart, bar);
+          bulk_load(dst + 4 * kQ + kXPart, st + kStDh + static_cast<size_t>(q) * kDhPart, kDhPart, bar);
+        }
+        issued = u + 1;
       }
-      mma_commit(empty0 + 8u * s);  // the stage is free once these MMAs have read it
+      if (timed_out)  // let the copies still in flight land before the block goes away
+        for (int u = issued > S ? issued - S : 0; u < issued; ++u) mbar_wait(full0 + 8u * (u % S), (u / S) & 1);
     }
-    // bias gradient: this thread's unit, summed over the item's rows in row order
+  } else if (warp == kConsumerWarps + 1) {
+    // ---- MMA issue
+    if (lane == 0) {
+      for (int u = 0; u < n_items && !timed_out; ++u) {
+        const int s = u % S;
+        const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
+        timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
+        if (timed_out) break;
+        tc_fence_after();
+        const uint32_t keep = u > 0 ? 1u : 0u;
+        if (role_w2) {  // d W2 [out half a][in half b] += d z2[:, a]^T . h1[:, b] over the item's rows
+#pragma unroll
+          for (int k = 0; k < kItemRows / 16; ++k)
+#pragma unroll
+            for (int ab = 0; ab < 4; ++ab)
+              mma_bf16(tmem + static_cast<uint32_t>(ab * 128), desc_mn(base + (ab >> 1) * kQ, 128, k), desc_mn(base + 2 * kQ + (ab & 1) * kQ, 128, k),
+                       instr_desc(128, 128) | kAmn | kBmn, keep | (k > 0));
+        } else {        // d W1 [out half a][in] += d z1[:, a]^T . x;  d Wh^T [unit half a][head] += h2[:, a]^T . dhead
+#pragma unroll
+          for (int k = 0; k < kItemRows / 16; ++k)
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {
+              mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * kQ, 128, k), desc_mn(base + 4 * kQ, kK1, k),
+                       instr_desc(128, kK1) | kAmn | kBmn, keep | (k > 0));
+              mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * kQ, 128, k), desc_mn(base + 4 * kQ + kXPart, kHeads, k),
+                       instr_desc(128, kHeads) | kAmn | kBmn, keep | (k > 0));
+            }
+        }
+        mma_commit(empty0 + 8u * s);  // the stage is free once these MMAs have read it
+      }
+      if (!timed_out && n_items > 0) mma_commit(done_bar);  // covers every MMA issued above
+    }
+  } else {
+    // ---- consumers: this thread's unit, summed over the item's rows in row order
+    const uint32_t my_col = static_cast<uint32_t>(tid >> 7) * kQ + static_cast<uint32_t>(((tid & 127) >> 3) * 128 + (tid & 7) * 2);
+    for (int u = 0; u < n_items && !timed_out; ++u) {
+      const int s = u % S;
+      const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
+      timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
+      if (__any_sync(0xFFFFFFFFu, timed_out)) { timed_out = true; break; }
 #pragma unroll 8
-    for (int r = 0; r < kHalfRows; ++r)
-      db += __uint_as_float(lds_u16(base + my_col + static_cast<uint32_t>((r >> 3) * 2048 + (r & 7) * 16)) << 16);
-    __syncwarp();
-    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8u * s) : "memory");
-    if (tid == 0 && u >= 1 && issued < n_items) {
-      // the previous item's stage (its MMAs are done and every warp has summed it) takes the item S - 1 ahead
-      timed_out |= !mbar_wait(empty0 + 8u * ((u - 1) % S), ((u - 1) / S) & 1);
-      if (!timed_out) { request(issued); ++issued; }
+      for (int r = 0; r < kItemRows; ++r)
+        db += __uint_as_float(lds_u16(base + my_col + static_cast<uint32_t>((r >> 3) * 2048 + (r & 7) * 16)) << 16);
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8u * s) : "memory");
     }
   }
-  if (tid == 0 && !timed_out) {  // one more commit covers every MMA issued so far
-    mma_commit(done_bar);
-    timed_out |= !mbar_wait(done_bar, 0);
-  }
+  // the consumer warps read the accumulators below; the other two warps go straight to the block-wide barrier
+  if (warp < kConsumerWarps && n_items > 0 && !timed_out) timed_out |= !mbar_wait(done_bar, 0);
   timed_out = __syncthreads_or(timed_out) != 0;
-  if (!timed_out && my_tiles > 0) {
+  if (!timed_out && my_tiles > 0 && warp < kConsumerWarps) {
     tc_fence_after();
     float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -495,10 +512,7 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
       part[off.b1 + tid] += db;
     }
   }
-  if (timed_out && tid == 0) {
-    atomicExch(status, kStatusTimeout);
-    for (int u = issued > S ? issued - S : 0; u < issued; ++u) mbar_wait(full0 + 8u * (u % S), (u / S) & 1);  // copies in flight land first
-  }
+  if (timed_out && tid == 0) atomicExch(status, kStatusTimeout);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
@@ -534,7 +548,7 @@ cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const
     ppo_rows256_kernel<<<slices, kThreads, sizeof(RowSmem), h->stream>>>(static_cast<const unsigned char *>(image), rows, hp, adv_stats,
                                                                          static_cast<unsigned char *>(staging), t0, nt, partial, n_params,
                                                                          term_partial, h->d_status, ho, h->D, has_value ? 1 : 0);
-    ppo_weights256_kernel<<<slices, kThreads, sizeof(WgtSmem), h->stream>>>(static_cast<const unsigned char *>(staging), nt, n_w2, partial,
+    ppo_weights256_kernel<<<slices, kWgtThreads, sizeof(WgtSmem), h->stream>>>(static_cast<const unsigned char *>(staging), nt, n_w2, partial,
                                                                             n_params, h->d_status, wo, h->D, has_value ? 1 : 0);
     h->launches += 2;
   }

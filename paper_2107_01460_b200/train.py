@@ -1,5 +1,6 @@
 """The whole on-device loop the report describes (Section 2, Figure 2): roll out, estimate advantages, update,
-repeat, with evaluation blocks in between -- every step a call into the C ABI, nothing computed in Python.
+repeat, with evaluation blocks in between -- every step of the method is a call into the C ABI; Python drives the
+loop, draws the minibatch permutations, averages the printed returns and, across ranks, sums the gradient.
 
     python -m paper_2107_01460_b200.train [--workload 1] [--envs 1024] [--steps 64] [--iters 200] [--epochs 4]
                                           [--lr 1e-3] [--eval-every 25] [--minibatches 1]
