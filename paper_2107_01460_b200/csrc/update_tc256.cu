@@ -137,42 +137,58 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
 
   // 128 accumulator columns of this thread (+ bias, ReLU) -> bf16 -> tensor memory (A operand of the next product) and
   // the staged tile; gate bits out
+  // (the load of the next 32 columns is in flight while the current 32 are converted; biases come in as 16-byte reads)
+  auto fwd_batch = [&](const uint32_t *ra, const float *bias, int c0, unsigned char *stage_act, uint32_t &g_out) {
+    uint32_t pk[16], g = 0;
+#pragma unroll
+    for (int e4 = 0; e4 < 8; ++e4) {
+      const float4 b = *reinterpret_cast<const float4 *>(bias + 128 * half + c0 + 4 * e4);
+      const float v0 = __uint_as_float(ra[4 * e4]) + b.x, v1 = __uint_as_float(ra[4 * e4 + 1]) + b.y;
+      const float v2 = __uint_as_float(ra[4 * e4 + 2]) + b.z, v3 = __uint_as_float(ra[4 * e4 + 3]) + b.w;
+      g |= (static_cast<uint32_t>(v0 > 0.0f) << (4 * e4)) | (static_cast<uint32_t>(v1 > 0.0f) << (4 * e4 + 1)) |
+           (static_cast<uint32_t>(v2 > 0.0f) << (4 * e4 + 2)) | (static_cast<uint32_t>(v3 > 0.0f) << (4 * e4 + 3));
+      pk[2 * e4] = relu_pack_bf16(__float_as_uint(v0), __float_as_uint(v1));
+      pk[2 * e4 + 1] = relu_pack_bf16(__float_as_uint(v2), __float_as_uint(v3));
+    }
+    g_out = g;
+    tmem_st16(tmem + kColHid + lane_off + static_cast<uint32_t>((128 * half + c0) / 2), pk);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      stg_v4(stage_act + act_row_off + static_cast<size_t>((c0 / 8 + q) * 128), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+  };
   auto fwd_epilogue = [&](const float *bias, unsigned char *stage_act, uint32_t gate[4]) {
-#pragma unroll
-    for (int c0 = 0; c0 < 128; c0 += 32) {
-      uint32_t ra[32], pk[16];
-      tmem_ld32_nowait(tmem + kColAcc + lane_off + 128u * half + c0, ra);
+    uint32_t ra[32], rb[32];
+    const uint32_t acc = tmem + kColAcc + lane_off + 128u * half;
+    tmem_ld32_nowait(acc, ra);
+#pragma unroll 1
+    for (int c0 = 0; c0 < 128; c0 += 64) {
+      tmem_ld_wait(); tmem_ld32_nowait(acc + static_cast<uint32_t>(c0 + 32), rb); fwd_batch(ra, bias, c0, stage_act, gate[c0 / 32]);
       tmem_ld_wait();
-      uint32_t g = 0;
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const float v0 = __uint_as_float(ra[2 * e]) + bias[128 * half + c0 + 2 * e];
-        const float v1 = __uint_as_float(ra[2 * e + 1]) + bias[128 * half + c0 + 2 * e + 1];
-        g |= (static_cast<uint32_t>(v0 > 0.0f) << (2 * e)) | (static_cast<uint32_t>(v1 > 0.0f) << (2 * e + 1));
-        pk[e] = relu_pack_bf16(__float_as_uint(v0), __float_as_uint(v1));
-      }
-      gate[c0 / 32] = g;
-      tmem_st16(tmem + kColHid + lane_off + static_cast<uint32_t>((128 * half + c0) / 2), pk);
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        stg_v4(stage_act + act_row_off + static_cast<size_t>((c0 / 8 + q) * 128), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+      if (c0 == 0) tmem_ld32_nowait(acc + 64u, ra);
+      fwd_batch(rb, bias, c0 + 32, stage_act, gate[c0 / 32 + 1]);
     }
     tmem_st_wait();
   };
+  auto bwd_batch = [&](const uint32_t *ra, uint32_t g, int c0, unsigned char *stage_act, bool to_tmem) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      pk[e] = pack_bf16(((g >> (2 * e)) & 1u) ? __uint_as_float(ra[2 * e]) : 0.0f, ((g >> (2 * e + 1)) & 1u) ? __uint_as_float(ra[2 * e + 1]) : 0.0f);
+    if (to_tmem) tmem_st16(tmem + kColHid + lane_off + static_cast<uint32_t>((128 * half + c0) / 2), pk);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      stg_v4(stage_act + act_row_off + static_cast<size_t>((c0 / 8 + q) * 128), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+  };
   auto bwd_epilogue = [&](const uint32_t gate[4], unsigned char *stage_act, bool to_tmem) {
-#pragma unroll
-    for (int c0 = 0; c0 < 128; c0 += 32) {
-      uint32_t ra[32], pk[16];
-      tmem_ld32_nowait(tmem + kColAcc + lane_off + 128u * half + c0, ra);
+    uint32_t ra[32], rb[32];
+    const uint32_t acc = tmem + kColAcc + lane_off + 128u * half;
+    tmem_ld32_nowait(acc, ra);
+#pragma unroll 1
+    for (int c0 = 0; c0 < 128; c0 += 64) {
+      tmem_ld_wait(); tmem_ld32_nowait(acc + static_cast<uint32_t>(c0 + 32), rb); bwd_batch(ra, gate[c0 / 32], c0, stage_act, to_tmem);
       tmem_ld_wait();
-      const uint32_t g = gate[c0 / 32];
-#pragma unroll
-      for (int e = 0; e < 16; ++e)
-        pk[e] = pack_bf16(((g >> (2 * e)) & 1u) ? __uint_as_float(ra[2 * e]) : 0.0f, ((g >> (2 * e + 1)) & 1u) ? __uint_as_float(ra[2 * e + 1]) : 0.0f);
-      if (to_tmem) tmem_st16(tmem + kColHid + lane_off + static_cast<uint32_t>((128 * half + c0) / 2), pk);
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        stg_v4(stage_act + act_row_off + static_cast<size_t>((c0 / 8 + q) * 128), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+      if (c0 == 0) tmem_ld32_nowait(acc + 64u, ra);
+      bwd_batch(rb, gate[c0 / 32 + 1], c0 + 32, stage_act, to_tmem);
     }
     if (to_tmem) tmem_st_wait();
   };
@@ -193,7 +209,14 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
         if (has_value) { v_old = rows.value_old[my_row * rows.vstride]; ret = rows.ret[my_row * rows.vstride]; }
       }
     }
-    if (tid == 0) bulk_store_wait_read();  // the copies of the previous tile's x and dhead tiles have read them
+    if (tid == 0) {
+      bulk_store_wait_read();  // the copies of the previous tile's x and dhead tiles have read them
+      // the next tile's rows on their way into L2 (a full tile of consecutive rows is one 16-byte aligned block)
+      if (rows.env_ids == nullptr && i + 1 < my_tiles && (tile0 + lt + static_cast<long long>(gridDim.x) + 1) * kR <= rows.n)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(rows.x + static_cast<size_t>(tile0 + lt + gridDim.x) * kR * D),
+                     "r"(static_cast<uint32_t>(kR * D * 4))
+                     : "memory");
+    }
     tc_fence_before();
     __syncthreads();
     // ---- the tile's rows as bf16 into x: a warp per row, consecutive lanes consecutive features

@@ -72,3 +72,47 @@ def test_hand_worked_warehouse_steps_on_the_gpu(precision):
     assert after[5, :6].tolist() == [3, 2, 0, 3, 4, 0]
     assert ro.dones[0].cpu().numpy().tolist() == [0] * 6
     assert float(ro.rewards[0].sum()) == 2.0
+
+
+@pytest.mark.parametrize("precision", [FP32, BF16])
+@pytest.mark.parametrize("name,n_envs", [(WH0, 16), (WH2, 130)])
+def test_warehouse_evaluation_block(name, n_envs, precision):
+    """A greedy evaluation block of the warehouse family: episode counts, return sums, length sums and final states bit
+    for bit against the oracle's transition under the GPU's own actions."""
+    import torch
+
+    from test_gpu_evaluate import _episode_sums, _state_records
+
+    w = wl.workload(name)
+    T = 130
+    params = torch.from_numpy(wl.make_params(w, bias_scale=0.1)).cuda()
+    ro = binding.Rollout(binding.make_config(w, precision=precision, max_T=4, n_envs=n_envs))
+    cnt, ret, ln, acts = ro.evaluate(params, T, greedy=True, want_actions=True)
+    assert ro.status() == binding.MAVA_OK
+    acts = acts.cpu().numpy()
+    env = oracle.rollout(oracle.make_config(w), w["seed"], None, T, np.arange(n_envs), forced_actions=acts, compute_mlp=False,
+                         want_obs=False)
+    c0, r0, l0 = _episode_sums(env.rewards, env.dones)
+    assert np.array_equal(cnt.cpu().numpy(), c0) and np.array_equal(ln.cpu().numpy(), l0)
+    assert np.array_equal(ret.cpu().numpy().view(np.uint32), r0.view(np.uint32))
+    assert np.array_equal(ro.get_state(), _state_records(env.states, w["n_agents"], w["n_food"]))
+    assert c0.sum() >= n_envs  # at least the cap ends an episode per environment
+    ro.close()
+
+
+def test_warehouse_shards_reproduce_the_whole_batch():
+    """Two handles with first_env offsets give the bytes of one handle over all environments (Philox, the replacement
+    requests included, is keyed on global environment indices)."""
+    import torch
+
+    w = wl.workload(WH2)
+    T, n, cut = 40, 90, 37
+    params = torch.from_numpy(wl.make_params(w)).cuda()
+    whole = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=n))
+    lo = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=cut))
+    hi = binding.Rollout(binding.make_config(w, precision=BF16, max_T=T, n_envs=n - cut, first_env=cut))
+    for r in (whole, lo, hi):
+        r.run(params, T)
+    for name in ("obs", "actions", "rewards", "dones", "logp", "values"):
+        full = getattr(whole, name)
+        assert torch.equal(full[:, :cut], getattr(lo, name)) and torch.equal(full[:, cut:], getattr(hi, name)), name

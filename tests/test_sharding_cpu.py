@@ -34,6 +34,13 @@ def _worker(rank, world, port, out_dir):
     ro = oracle.rollout(oracle.make_config(w), w["seed"], wl.make_params(w), 12, ids)
     np.save(os.path.join(out_dir, f"obs{rank}.npy"), ro.obs)
     np.save(os.path.join(out_dir, f"act{rank}.npy"), ro.actions)
+    # the warehouse family (its replacement requests are keyed on global indices too) and the recurrent policy
+    ww = wl.workload("wh2_10x10_3r3s_h128_collisions_end")
+    wh = oracle.rollout(oracle.make_config(ww), ww["seed"], wl.make_params(ww), 30, ids)
+    np.save(os.path.join(out_dir, f"wh{rank}.npy"), np.concatenate([wh.obs.reshape(30, per_rank, -1), wh.rewards], axis=2))
+    wr = wl.workload("rec0_tiny_8x8_2p2f_gru64")
+    rec, hid = oracle.rollout_rec(oracle.make_config(wr), wr["seed"], wl.make_params(wr), 12, ids)
+    np.save(os.path.join(out_dir, f"rec{rank}.npy"), rec.logits)
     t = torch.tensor([1.0 + rank, 10.0 - rank], dtype=torch.float64)  # (step ms, e2e s) of this rank
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     assert t.tolist() == [float(world), 10.0]
@@ -49,6 +56,14 @@ def test_env_shards_reproduce_the_unsharded_batch(tmp_path):
     obs = np.concatenate([np.load(tmp_path / f"obs{r}.npy") for r in range(world)], axis=1)
     act = np.concatenate([np.load(tmp_path / f"act{r}.npy") for r in range(world)], axis=1)
     assert np.array_equal(obs, whole.obs) and np.array_equal(act, whole.actions)
+    ids = np.arange(10, dtype=np.int32)
+    ww = wl.workload("wh2_10x10_3r3s_h128_collisions_end")
+    wh = oracle.rollout(oracle.make_config(ww), ww["seed"], wl.make_params(ww), 30, ids)
+    got = np.concatenate([np.load(tmp_path / f"wh{r}.npy") for r in range(world)], axis=1)
+    assert np.array_equal(got, np.concatenate([wh.obs.reshape(30, 10, -1), wh.rewards], axis=2))
+    wr = wl.workload("rec0_tiny_8x8_2p2f_gru64")
+    rec, _ = oracle.rollout_rec(oracle.make_config(wr), wr["seed"], wl.make_params(wr), 12, ids)
+    assert np.array_equal(np.concatenate([np.load(tmp_path / f"rec{r}.npy") for r in range(world)], axis=1), rec.logits)
 
 
 def _shard_gradient(rank, per_rank, T):
