@@ -212,6 +212,19 @@ int mava_ppo_grad_envs(mava_rollout_t *h, const float *params_dev, const mava_pp
 int mava_adam_step(mava_rollout_t *h, float *params_dev, const float *grad_dev, float *m_dev, float *v_dev, int32_t step,
                    const mava_ppo_hyper_t *hp);
 
+/* The update loop of one training iteration behind one call (Section 2, Figure 2: each update function turns its
+ * rolled-out experience into new parameters): `epochs` passes over the last run's rows, each pass cut into
+ * `minibatches` minibatches of environments, every minibatch one mava_ppo_grad_envs followed by one mava_adam_step
+ * (step numbers first_step, first_step + 1, ...).  The shuffling is the caller's: perm_dev is [epochs][n_envs] int32
+ * (device pointer), row e a permutation of 0..n_envs-1 (any list of valid indices works; it is not checked beyond the
+ * range check of mava_ppo_grad_envs); minibatch k of pass e is the slice [k * n_envs / minibatches, (k + 1) * n_envs /
+ * minibatches) of that row.  params_dev, m_dev, v_dev are updated in place; grad_dev is workspace of
+ * mava_params_count floats; terms_dev, if not NULL, receives [epochs * minibatches][4] loss terms in the order the
+ * minibatches were taken.  Asynchronous: everything is enqueued on the handle's stream, nothing is copied to the host.
+ * Errors: as mava_ppo_grad_envs and mava_adam_step; INVALID_ARG for epochs < 1, minibatches < 1 or > n_envs. */
+int mava_ppo_update(mava_rollout_t *h, float *params_dev, float *m_dev, float *v_dev, float *grad_dev, const mava_ppo_hyper_t *hp,
+                    int32_t epochs, int32_t minibatches, const int32_t *perm_dev, int32_t first_step, float *terms_dev);
+
 /* Back to episode 0 and global step 0 under a new seed.  Asynchronous. */
 int mava_rollout_reset(mava_rollout_t *h, uint64_t seed);
 

@@ -35,7 +35,7 @@ EXPORTS = [
     "mava_rollout_reset", "mava_rollout_status", "mava_state_record_len", "mava_rollout_get_state",
     "mava_rollout_set_state", "mava_rollout_collect_host", "mava_rollout_launch_count", "mava_rollout_destroy",
     "mava_strerror", "mava_rollout_run_static", "mava_rollout_evaluate", "mava_ppo_defaults", "mava_ppo_grad",
-    "mava_adam_step", "mava_ppo_grad_envs", "mava_debug_expire_next_wait", "mava_rollout_get_hidden",
+    "mava_adam_step", "mava_ppo_grad_envs", "mava_debug_expire_next_wait", "mava_rollout_get_hidden", "mava_ppo_update",
 ]
 
 
@@ -96,6 +96,8 @@ def lib():
         L.mava_ppo_grad.argtypes = [vp, vp, hpp, vp, vp]; L.mava_ppo_grad.restype = C.c_int
         L.mava_ppo_grad_envs.argtypes = [vp, vp, hpp, vp, C.c_int32, vp, vp]; L.mava_ppo_grad_envs.restype = C.c_int
         L.mava_adam_step.argtypes = [vp, vp, vp, vp, vp, C.c_int32, hpp]; L.mava_adam_step.restype = C.c_int
+        L.mava_ppo_update.argtypes = [vp, vp, vp, vp, vp, hpp, C.c_int32, C.c_int32, vp, C.c_int32, vp]
+        L.mava_ppo_update.restype = C.c_int
         L.mava_rollout_get_hidden.argtypes = [vp, vp]; L.mava_rollout_get_hidden.restype = C.c_int
         L.mava_debug_expire_next_wait.argtypes = [vp, C.c_int32]; L.mava_debug_expire_next_wait.restype = C.c_int
         _lib = L
@@ -233,6 +235,19 @@ class Rollout:
         hp = ppo_defaults() if hp is None else hp
         _check(lib().mava_adam_step(self.handle, params.data_ptr(), grad.data_ptr(), m.data_ptr(), v.data_ptr(), step,
                                     C.byref(hp)), "mava_adam_step")
+
+    def ppo_update(self, params, m, v, perm, minibatches: int, first_step: int, hp: "mava_ppo_hyper_t | None" = None):
+        """`perm.shape[0]` passes of `minibatches` minibatches each over the last run's rows (mava_ppo_update): params, m,
+        v change in place; returns the loss terms [passes * minibatches][4] (device tensor)."""
+        import torch
+
+        hp = ppo_defaults() if hp is None else hp
+        assert perm.is_cuda and perm.dtype == torch.int32 and perm.is_contiguous() and perm.shape[1] == self.cfg.n_envs
+        grad = torch.empty_like(params)
+        terms = torch.empty((perm.shape[0] * minibatches, 4), dtype=torch.float32, device=params.device)
+        _check(lib().mava_ppo_update(self.handle, params.data_ptr(), m.data_ptr(), v.data_ptr(), grad.data_ptr(), C.byref(hp),
+                                     perm.shape[0], minibatches, perm.data_ptr(), first_step, terms.data_ptr()), "mava_ppo_update")
+        return terms
 
     def reset(self, seed: int):
         _check(lib().mava_rollout_reset(self.handle, seed), "mava_rollout_reset")

@@ -235,6 +235,24 @@ int mava_adam_step(mava_rollout_t *h, float *params_dev, const float *grad_dev, 
   return launch_adam_step(h, params_dev, grad_dev, m_dev, v_dev, step, *hp) == cudaSuccess ? MAVA_OK : MAVA_ERR_CUDA;
 }
 
+int mava_ppo_update(mava_rollout_t *h, float *params_dev, float *m_dev, float *v_dev, float *grad_dev, const mava_ppo_hyper_t *hp,
+                    int32_t epochs, int32_t minibatches, const int32_t *perm_dev, int32_t first_step, float *terms_dev) {
+  if (!h || !params_dev || !m_dev || !v_dev || !grad_dev || !hp || !perm_dev || epochs < 1 || minibatches < 1 || first_step < 1 ||
+      minibatches > h->cfg.n_envs)
+    return MAVA_ERR_INVALID_ARG;
+  const int E = h->cfg.n_envs;
+  int step = first_step;
+  for (int e = 0; e < epochs; ++e)
+    for (int k = 0; k < minibatches; ++k) {
+      const int lo = static_cast<int>(static_cast<int64_t>(E) * k / minibatches), hi = static_cast<int>(static_cast<int64_t>(E) * (k + 1) / minibatches);
+      float *terms = terms_dev ? terms_dev + 4 * (static_cast<size_t>(e) * minibatches + k) : nullptr;
+      int rc = mava_ppo_grad_envs(h, params_dev, hp, perm_dev + static_cast<size_t>(e) * E + lo, hi - lo, grad_dev, terms);
+      if (rc == MAVA_OK) rc = mava_adam_step(h, params_dev, grad_dev, m_dev, v_dev, step++, hp);
+      if (rc != MAVA_OK) return rc;
+    }
+  return MAVA_OK;
+}
+
 int mava_rollout_reset(mava_rollout_t *h, uint64_t seed) {
   if (!h) return MAVA_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);

@@ -68,8 +68,18 @@ def train(workload: int = 1, n_envs: int = 1024, T: int = 64, iters: int = 200, 
             break
         ro.run(params, T)
         ro.gae(wl.GAMMA, wl.LAMBDA)
+        import torch.distributed as dist
+
+        if not (dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1):
+            # one process: the passes and minibatches of the iteration in one library call; the shuffling (a fresh
+            # permutation per pass, seeded, same on every run) is drawn here and handed over
+            perm = torch.stack([torch.randperm(n_envs, generator=shuffle, device="cuda") if minibatches > 1
+                                else torch.arange(n_envs, device="cuda") for _ in range(epochs)]).to(torch.int32).contiguous()
+            ro.ppo_update(params, m, v, perm, max(1, minibatches), step + 1, hp)
+            step += epochs * max(1, minibatches)
+            continue
         for _ in range(epochs):
-            # an epoch: every environment once, in `minibatches` pieces of a fresh permutation (seeded, same on every run)
+            # several ranks: the gradient is averaged between the gradient call and the optimiser call
             pieces = [None] if minibatches <= 1 else torch.randperm(n_envs, generator=shuffle, device="cuda").to(torch.int32).chunk(minibatches)
             for ids in pieces:
                 step += 1

@@ -275,3 +275,32 @@ def test_at_unchanged_parameters_the_ratios_of_a_bf16_handle_stay_near_one():
     print(out)
     assert out["tensor"] < 1e-3
     assert out["fp32"] < 3e-2
+
+
+@pytest.mark.parametrize("idx,precision", [(1, BF16), (0, FP32), (3, BF16)])
+def test_update_loop_in_one_call_equals_the_calls_it_stands_for(idx, precision):
+    """mava_ppo_update (passes x minibatches of gradient + Adam inside the library) against the same sequence issued call
+    by call: same kernels on the same inputs, so parameters, moments and loss terms must be the same bytes."""
+    import torch
+
+    n_envs, T, epochs, mbs = 96, 12, 2, 3
+    w, ro, params = _rolled_out(idx, n_envs, T, precision, flags=0)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    perm = torch.stack([torch.randperm(n_envs, generator=g, device="cuda") for _ in range(epochs)]).to(torch.int32).contiguous()
+    hp = binding.ppo_defaults()
+    p1, m1, v1 = params.clone(), torch.zeros_like(params), torch.zeros_like(params)
+    terms1 = ro.ppo_update(p1, m1, v1, perm, mbs, 1, hp)
+    p2, m2, v2 = params.clone(), torch.zeros_like(params), torch.zeros_like(params)
+    terms2, step = [], 0
+    for e in range(epochs):
+        for k in range(mbs):
+            ids = perm[e, n_envs * k // mbs: n_envs * (k + 1) // mbs].contiguous()
+            t, grad = ro.ppo_grad(p2, hp, env_ids=ids)
+            step += 1
+            ro.adam_step(p2, grad, m2, v2, step, hp)
+            terms2.append(t.clone())
+    assert ro.status() == binding.MAVA_OK
+    assert torch.equal(p1, p2) and torch.equal(m1, m2) and torch.equal(v1, v2)
+    assert torch.equal(terms1, torch.stack(terms2))
+    assert not torch.equal(p1, params)
+    ro.close()
