@@ -4,8 +4,8 @@ TEST INFRASTRUCTURE ONLY, like the rest of this package: plain numpy in float64,
 fusion, one statement per formula.  Nothing under the CUDA package imports it.
 
 What it follows.  The report (Section 2, "Strong baseline algorithms and training architectures",
-Figure 2) says that every update function takes the rolled-out experience and minimises "multi-agent
-PPO" losses, for independent learners (a critic head on the shared torso) and for a centralised
+Figure 2) says that every update function takes the rolled-out experience and minimises multi-agent
+PPO losses, for independent learners (a critic head on the shared torso) and for a centralised
 critic; it prints no formula and no coefficient.  The reading taken here is the clipped-surrogate
 objective of Schulman et al. (2017) as multi-agent PPO systems commonly use it, over ONE minibatch of
 rows (a row = one agent at one environment-step):
