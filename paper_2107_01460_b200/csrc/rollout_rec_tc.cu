@@ -78,7 +78,12 @@ __global__ void prep_rec_tc_kernel(const float *__restrict__ params, unsigned ch
 }
 
 __device__ __forceinline__ uint64_t rdesc(uint32_t tile, int C, int k) { return smem_desc(tile + k * 256, 128, C * 16); }
-__device__ __forceinline__ float sigm(float v) { return 1.0f / (1.0f + expf(-v)); }
+// Branch-free forms (ex2.approx and rcp.approx: a few 1e-7, far below the bf16 step the result is rounded to), so
+// that the compiler can interleave the units of a row: with one warp per scheduler the gate epilogue is bound by
+// the latency of dependent instructions, not by their number.
+// The arguments are clamped to where the functions have long saturated in binary32, which keeps the exponential finite.
+__device__ __forceinline__ float sigm(float v) { return __fdividef(1.0f, 1.0f + __expf(-fminf(fmaxf(v, -30.0f), 30.0f))); }
+__device__ __forceinline__ float tanh_fast(float v) { return 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * fminf(fmaxf(v, -15.0f), 15.0f))); }
 __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -254,7 +259,7 @@ rollout_rec_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, fl
                 const float hprev = __uint_as_float(s == 0 ? (hw[e] << 16) : (hw[e] & 0xFFFF0000u));
                 const float r = sigm(gr[q] + brz[j]);
                 const float z = sigm(gz[q] + brz[H + j]);
-                const float n = tanhf(gi[q] + bin[j] + r * (gh[q] + bhn[j]));
+                const float n = tanh_fast(gi[q] + bin[j] + r * (gh[q] + bhn[j]));
                 hn[s] = (1.0f - z) * n + z * hprev;
               }
               pk[e] = pack_bf16(hn[0], hn[1]);
