@@ -318,7 +318,7 @@ def time_update(torch, binding, ro, params, w, steps, warmup, flush):
             times.append(e0.elapsed_time(e1))
     path = "fp32 SIMT"
     if binding.update_on_tensor_cores(ro.cfg):
-        path = "bf16 tcgen05" + (" (actor net; the centralised critic's net in fp32 SIMT)" if ro.cfg.net_kind == 1 else "")
+        path = "bf16 tcgen05"
     return sum(times) / len(times), path
 
 

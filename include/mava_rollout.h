@@ -193,13 +193,13 @@ void mava_ppo_defaults(mava_ppo_hyper_t *hp);
  * mean entropy, value term (device pointers).
  * Arithmetic: an fp32 handle computes in fp32 on the plain ALUs.  A bf16 handle takes tensor-core kernels (bf16
  * operands, fp32 accumulation; the derivatives with respect to the hidden pre-activations are rounded to bf16 before
- * they enter a product) for the shared-torso shapes with H <= 128 and for H = 256 (with the centralised critic: the
- * actor net; the critic's net stays in fp32), unless MAVA_FLAG_UPDATE_FP32 is set.  The rollout of a bf16 handle
+ * they enter a product) for the shared-torso shapes with H <= 128 and for H = 256 (with the centralised critic: both
+ * nets), unless MAVA_FLAG_UPDATE_FP32 is set.  The rollout of a bf16 handle
  * stored logp and values from bf16 arithmetic: re-evaluated at unchanged parameters by the tensor-core kernels (same
  * operand rounding) the ratio rho is 1 to about 1e-3; re-evaluated in fp32 (the flag) the rollout's rounding shows as
  * a policy change of up to a few 1e-2 in rho and in V - values, which the clips then see.
  * The library allocates its scratch on the first call and keeps it until destroy: one gradient slice of params_count
- * floats per resident CTA (up to three per SM), and for H = 256 on the tensor cores a staging buffer of 1.2 GB.
+ * floats per resident CTA (up to three per SM), and for H = 256 on the tensor cores a staging buffer of up to 1.5 GB.
  * The recurrent policy has no update block (MAVA_ERR_UNSUPPORTED).  Asynchronous.
  * Errors: INVALID_ARG (NULL pointers, no run yet, adv/ret NULL), UNSUPPORTED, CUDA. */
 int mava_ppo_grad(mava_rollout_t *h, const float *params_dev, const mava_ppo_hyper_t *hp, float *grad_dev, float *terms_dev);

@@ -123,7 +123,7 @@ def make_config(w: dict, precision: int | None = None, flags: int = 0, max_T: in
 def update_on_tensor_cores(cfg: mava_config_t) -> bool:
     """Whether mava_ppo_grad takes the bf16 tensor-core kernels for a handle of this configuration: the shared-torso
     shapes with H <= 128 and D <= 80 (one fused kernel), and H = 256 with 64 < D <= 96 (row kernel + weight kernel; with
-    a centralised critic only the actor net, the critic net stays on the fp32 kernel)."""
+    a centralised critic both nets)."""
     if cfg.precision != MAVA_PRECISION_BF16 or cfg.flags & MAVA_FLAG_UPDATE_FP32:
         return False
     D = 77 + cfg.n_agents

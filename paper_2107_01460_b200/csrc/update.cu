@@ -377,7 +377,7 @@ struct UpdScratch {
   int slices;
 };
 size_t image_room() {
-  const size_t a = ppo_tc_image_bytes(), b = ppo_tc256_image_bytes();
+  const size_t a = ppo_tc_image_bytes(), b = ppo_tc256_image_bytes(kMaxAgents);
   return ((a > b ? a : b) + 255) / 256 * 256;
 }
 UpdScratch carve(mava_rollout *h, size_t n_params, int slices) {
@@ -463,9 +463,10 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
     return cudaGetLastError();
   }
 
-  // H = 256 on the tensor cores: the actor / shared-torso net; a centralised critic stays on the fp32 kernel below
+  // H = 256 on the tensor cores: the actor / shared-torso net and, one input slab per agent, the centralised critic's
   const bool tc256 = update_takes_tensor_cores_256(cfg, D);
-  const int slices_tc = tc256 ? static_cast<int>(tiles128 < sms ? (tiles128 < 2 ? 2 : tiles128) : sms) : 0;
+  const int min_slices = 1 + (central ? N : 1);  // the weight kernel needs a CTA for d W2 and one per input slab
+  const int slices_tc = tc256 ? static_cast<int>(tiles128 < sms ? (tiles128 < min_slices ? min_slices : tiles128) : sms) : 0;
   const long long tiles = (R + kUpdRows - 1) / kUpdRows;
   // fp32 kernel: as many CTAs (= gradient slices) as are resident at once with the larger of the two nets' shared-memory needs
   const int joint = N * D;
@@ -485,7 +486,7 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   if (err != cudaSuccess) return err;
   const int chunk_tiles = static_cast<int>(tiles128 < kChunkTiles ? tiles128 : kChunkTiles);
   if (tc256) {
-    err = ensure_update_staging(h, ppo_tc256_staging_bytes(chunk_tiles));
+    err = ensure_update_staging(h, ppo_tc256_staging_bytes(chunk_tiles, central ? N : 1));
     if (err != cudaSuccess) return err;
   }
   const UpdScratch sc = carve(h, P, slices);
@@ -494,8 +495,10 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
     transpose_kernel<<<64, 256, 0, st>>>(params_dev + off, sc.wt + off, out, in);
     h->launches += 1;
   };
-  if (!tc256) { tr(L.W1, H, D); tr(L.W2, H, H); }
-  if (central) { tr(L.C1, H, joint); tr(L.C2, H, H); }
+  if (!tc256) {
+    tr(L.W1, H, D); tr(L.W2, H, H);
+    if (central) { tr(L.C1, H, joint); tr(L.C2, H, H); }
+  }
   stat_partial_kernel<<<kStatBlocks, 256, 0, st>>>(h->buf.adv, R, sc.stat_part, rows);
   stat_final_kernel<<<1, 32, 0, st>>>(sc.stat_part, kStatBlocks, R, sc.stats);
   h->launches += 2;
@@ -518,12 +521,14 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
   actor.oW1 = L.W1; actor.ob1 = L.b1; actor.oW2 = L.W2; actor.ob2 = L.b2; actor.oWa = L.Wa; actor.oba = L.ba;
   if (!central) {
     actor.Wv = params_dev + L.Wv; actor.bv = params_dev + L.bv; actor.oWv = L.Wv; actor.obv = L.bv;
-    err = tc256 ? launch_ppo_net_tc256(h, params_dev, L, rows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P, sc.term_part,
-                                       slices_tc, true)
+    const Tc256Net net{L.W1, L.b1, L.W2, L.b2, L.Wa, L.ba, L.Wv, L.bv, 1, true, true};
+    err = tc256 ? launch_ppo_net_tc256(h, params_dev, net, rows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P,
+                                       sc.term_part, slices_tc)
                 : run_net(actor, rows);
   } else {
-    err = tc256 ? launch_ppo_net_tc256(h, params_dev, L, rows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P, sc.term_part,
-                                       slices_tc, false)
+    const Tc256Net anet{L.W1, L.b1, L.W2, L.b2, L.Wa, L.ba, 0, 0, 1, true, false};
+    err = tc256 ? launch_ppo_net_tc256(h, params_dev, anet, rows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P,
+                                       sc.term_part, slices_tc)
                 : run_net(actor, rows);
     if (err != cudaSuccess) return err;
     UpdNet critic{};
@@ -535,7 +540,10 @@ cudaError_t launch_ppo_grad(mava_rollout *h, const float *params_dev, const mava
     UpdRows crows{};
     crows.x = h->buf.obs; crows.value_old = h->buf.values; crows.ret = h->buf.ret; crows.vstride = N; crows.n = S;
     crows.env_ids = env_ids_dev; crows.n_ids = n_env; crows.E = E; crows.per_env = 1;
-    err = run_net(critic, crows);
+    const Tc256Net cnet{L.C1, L.c1, L.C2, L.c2, 0, 0, L.Cv, L.cv, N, false, true};
+    err = tc256 ? launch_ppo_net_tc256(h, params_dev, cnet, crows, hp, sc.stats, sc.image, h->d_upd_stage, chunk_tiles, sc.partial, P,
+                                       sc.term_part, slices_tc)
+                : run_net(critic, crows);
   }
   if (err != cudaSuccess) return err;
   reduce_partials_kernel<<<128, 256, 0, st>>>(sc.partial, P, slices, grad_dev, sc.term_part, 8 * slices, R, central ? S : R, hp,

@@ -48,14 +48,21 @@ cudaError_t launch_ppo_net_tc(mava_rollout *h, const float *params_dev, const Pa
                               const double *adv_stats, void *image, float *partial, size_t n_params, double *term_partial, int slices);
 
 
-// Tensor-core path for H = 256 (update_tc256.cu): the actor / shared-torso net with 64 < D <= 96, a chunk of
-// `chunk_tiles` 128-row tiles at a time through `staging` (ppo_tc256_staging_bytes(chunk_tiles) bytes).  Adds into the
-// slices of `partial` and into `term_partial` (both zeroed by the caller); needs slices >= 2.
+// Tensor-core path for H = 256 (update_tc256.cu): a net with hidden width 256 whose first layer takes `slabs` observation
+// slabs of width 64 < D <= 96 side by side (1: the actor / shared-torso net; n_agents: the centralised critic), a chunk
+// of `chunk_tiles` 128-row tiles at a time through `staging` (ppo_tc256_staging_bytes bytes).  Offsets are those of the
+// net's layers in the flat parameter array.  Adds into the slices of `partial` and into `term_partial` (both zeroed by
+// the caller); needs slices >= 1 + slabs.
+struct Tc256Net {
+  size_t W1, b1, W2, b2, Wa, ba, Wv, bv;
+  int slabs;
+  bool has_actor, has_value;
+};
 bool ppo_tc256_supported(const mava_config_t &cfg, int D);
-size_t ppo_tc256_image_bytes();
-size_t ppo_tc256_staging_bytes(int chunk_tiles);
-cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const ParamLayout &L, const UpdRows &rows, const UpdHyper &hp,
+size_t ppo_tc256_image_bytes(int slabs);
+size_t ppo_tc256_staging_bytes(int chunk_tiles, int slabs);
+cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const Tc256Net &net, const UpdRows &rows, const UpdHyper &hp,
                                  const double *adv_stats, void *image, void *staging, int chunk_tiles, float *partial, size_t n_params,
-                                 double *term_partial, int slices, bool has_value);
+                                 double *term_partial, int slices);
 
 }  // namespace mava

@@ -45,7 +45,8 @@ constexpr uint32_t kTmemCols = 512;
 
 struct UtcSmem {
   alignas(128) unsigned char img[(kImgBytes + 127) / 128 * 128];
-  alignas(128) unsigned char x[kUR * kUK1 * 2];
+  alignas(128) unsigned char x[(kUR / 8) * (kUK1 / 8) * kALbo];  // feature chunks 144 bytes apart (see a_offset): the
+                                                                 // converter's 2-byte stores then spread over the banks
   alignas(128) unsigned char h1[kUR * kUH * 2];
   alignas(128) unsigned char h2[kUR * kUH * 2];   // d z1 once h2's last reader is done
   alignas(128) unsigned char dz2[kUR * kUH * 2];
@@ -242,7 +243,7 @@ ppo_net_tc_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHype
 #pragma unroll
           for (int q = 0; q < 3; ++q) {
             const int k = lane + 32 * q;
-            if (k < D) sts_u16(xt + canon_offset(r, k, kUK1), bf16_bits(v[g][q]));
+            if (k < D) sts_u16(xt + a_offset<kUK1>(r, k), bf16_bits(v[g][q]));
           }
         }
       }
@@ -254,7 +255,8 @@ ppo_net_tc_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHype
       if (bulk_ok(i + 1)) { request_stage(i + 1); stage_pending = true; }
       tc_fence_after();
 #pragma unroll
-      for (int k = 0; k < kUK1 / 16; ++k) mma_bf16(tmem + kColAcc, desc_k(xt, kUK1, k), desc_k(w1, kUK1, k), instr_desc(kUR, kUH), k > 0);
+      for (int k = 0; k < kUK1 / 16; ++k)
+        mma_bf16(tmem + kColAcc, smem_desc(xt + k * 2 * kALbo, kALbo, (kUK1 / 8) * kALbo), desc_k(w1, kUK1, k), instr_desc(kUR, kUH), k > 0);
       mma_commit(bar_mma);
     }
     timed_out |= !mbar_wait(bar_mma, ph_mma); ph_mma ^= 1;
@@ -369,7 +371,8 @@ ppo_net_tc_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHype
       tc_fence_after();
 #pragma unroll
       for (int k = 0; k < kUR / 16; ++k)
-        mma_bf16(tmem + kColDW1, desc_mn(dz1t, kUH, k), desc_mn(xt, kUK1, k), instr_desc(kUH, kUK1) | kAmn | kBmn, keep | (k > 0));
+        mma_bf16(tmem + kColDW1, desc_mn(dz1t, kUH, k), smem_desc(xt + k * 2 * (kUK1 / 8) * kALbo, (kUK1 / 8) * kALbo, kALbo),
+                 instr_desc(kUH, kUK1) | kAmn | kBmn, keep | (k > 0));
 #pragma unroll
       for (int k = 0; k < kUR / 16; ++k)
         mma_bf16(tmem + kColDB1, desc_mn(dz1t, kUH, k), desc_mn(dht, kUHeads, k), instr_desc(kUH, kUHeads) | kAmn | kBmn, keep | (k > 0));

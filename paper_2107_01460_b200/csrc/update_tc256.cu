@@ -28,77 +28,107 @@ constexpr int kK1 = 96;       // input width, padded (D = 81, 85)
 constexpr int kHeads = 16;
 constexpr int kThreads = 256;
 
+// Image in shared memory: W1 (one input slab) | W2 | Wh | b1 | b2 | bh.  In global memory the image holds all slabs of
+// W1 first (kImgW2 bytes each), then the rest in the same order.
 constexpr uint32_t kImgW1 = 0, kImgW2 = kImgW1 + kH * kK1 * 2, kImgWh = kImgW2 + kH * kH * 2;
 constexpr uint32_t kImgB1 = kImgWh + kHeads * kH * 2, kImgB2 = kImgB1 + kH * 4, kImgBh = kImgB2 + kH * 4;
 constexpr uint32_t kImgBytes = kImgBh + 32;
 static_assert(kImgBytes % 16 == 0, "bulk copies");
 
-// staging buffer, per tile: x [128][96]; h1, h2, d z2, d z1 as two unit halves [128][128] each; dhead [128][16]
-constexpr size_t kStX = 0, kStXBytes = kR * kK1 * 2;
+// staging buffer, per tile: one x tile [128][96] per input slab; h1, h2, d z2, d z1 as two unit halves [128][128] each;
+// dhead [128][16].  An input slab is one agent's observation: the actor / shared-torso net has one, the centralised
+// critic (input = the agents' observations side by side) one per agent.
+constexpr uint32_t kXLbo = kALbo, kXSbo = (kK1 / 8) * kALbo;  // x tile: feature chunks 144 bytes apart (the converter's
+                                                               // 2-byte stores then spread over the banks), row groups 1728
+constexpr size_t kStXBytes = (kR / 8) * kXSbo;
 constexpr size_t kHalfBytes = kR * 128 * 2, kActBytes = 2 * kHalfBytes;
-constexpr size_t kStH1 = kStX + kStXBytes, kStH2 = kStH1 + kActBytes, kStDz2 = kStH2 + kActBytes, kStDz1 = kStDz2 + kActBytes;
-constexpr size_t kStDh = kStDz1 + kActBytes, kStDhBytes = kR * kHeads * 2;
-constexpr size_t kStTile = kStDh + kStDhBytes;  // 290 816 bytes
+constexpr size_t kStDhBytes = kR * kHeads * 2;
+struct StageLayout {
+  size_t x, h1, h2, dz2, dz1, dh, tile;
+};
+__host__ __device__ inline StageLayout stage_layout(int slabs) {
+  StageLayout L;
+  L.x = 0; L.h1 = static_cast<size_t>(slabs) * kStXBytes; L.h2 = L.h1 + kActBytes; L.dz2 = L.h2 + kActBytes; L.dz1 = L.dz2 + kActBytes;
+  L.dh = L.dz1 + kActBytes; L.tile = L.dh + kStDhBytes;  // 290 816 bytes with one slab
+  return L;
+}
 
 constexpr uint32_t kColAcc = 0, kColHid = 256, kColHead = 384, kTmemRow = 512;
 
 struct RowSmem {
   alignas(128) unsigned char img[(kImgBytes + 127) / 128 * 128];
-  alignas(128) unsigned char x[kR * kK1 * 2];
+  alignas(128) unsigned char x[kStXBytes];
   alignas(128) unsigned char dhead[kR * kHeads * 2];
   long long rmap[kR];
   float red[4][8];
-  alignas(8) uint64_t bar_load, bar_mma;
+  alignas(8) uint64_t bar_load, bar_mma, bar_mmb, bar_w1;  // bar_mmb: the second column half of a product issued in halves
   uint32_t tmem_base;
 };
 
-__global__ void prep_upd256_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, ParamLayout L, int D, int has_value) {
-  auto bf = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(image + off); };
+// Which net the kernels work on: offsets of its layers in the flat parameter (= gradient) array and its input shape.
+struct Net256 {
+  size_t W1, b1, W2, b2, Wa, ba, Wv, bv;
+  int D;          // width of one input slab (an agent's observation)
+  int slabs;      // 1, or the number of agents for the centralised critic
+  int w1_ld;      // input width of the first layer = slabs * D
+  int has_actor, has_value;
+};
+
+__global__ void prep_upd256_kernel(const float *__restrict__ params, unsigned char *__restrict__ image, Net256 net) {
   const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-  for (int i = tid; i < kH * kK1; i += nth) {
-    const int n = i / kK1, k = i - n * kK1;
-    bf(kImgW1)[canon_offset(n, k, kK1) / 2] = __float2bfloat16_rn(k < D ? params[L.W1 + static_cast<size_t>(n) * D + k] : 0.0f);
+  const int D = net.D;
+  for (int i = tid; i < net.slabs * kH * kK1; i += nth) {
+    const int a = i / (kH * kK1), r = i - a * (kH * kK1), n = r / kK1, k = r - n * kK1;
+    reinterpret_cast<__nv_bfloat16 *>(image + static_cast<size_t>(a) * kImgW2)[canon_offset(n, k, kK1) / 2] =
+        __float2bfloat16_rn(k < D ? params[net.W1 + static_cast<size_t>(n) * net.w1_ld + a * D + k] : 0.0f);
   }
+  unsigned char *rest = image + static_cast<size_t>(net.slabs) * kImgW2 - kImgW2;  // so that rest + kImgX is where X lies
+  auto bf = [&](uint32_t off) { return reinterpret_cast<__nv_bfloat16 *>(rest + off); };
   for (int i = tid; i < kH * kH; i += nth) {
     const int n = i / kH, k = i - n * kH;
-    bf(kImgW2)[canon_offset(n, k, kH) / 2] = __float2bfloat16_rn(params[L.W2 + static_cast<size_t>(n) * kH + k]);
+    bf(kImgW2)[canon_offset(n, k, kH) / 2] = __float2bfloat16_rn(params[net.W2 + static_cast<size_t>(n) * kH + k]);
   }
   for (int i = tid; i < kHeads * kH; i += nth) {
     const int n = i / kH, k = i - n * kH;
     float v = 0.0f;
-    if (n < kActions) v = params[L.Wa + static_cast<size_t>(n) * kH + k];
-    else if (n == kActions && has_value) v = params[L.Wv + k];
+    if (n < kActions && net.has_actor) v = params[net.Wa + static_cast<size_t>(n) * kH + k];
+    else if (n == kActions && net.has_value) v = params[net.Wv + k];
     bf(kImgWh)[canon_offset(n, k, kH) / 2] = __float2bfloat16_rn(v);
   }
-  float *b1 = reinterpret_cast<float *>(image + kImgB1), *b2 = reinterpret_cast<float *>(image + kImgB2),
-        *bh = reinterpret_cast<float *>(image + kImgBh);
-  for (int i = tid; i < kH; i += nth) { b1[i] = params[L.b1 + i]; b2[i] = params[L.b2 + i]; }
-  if (tid < 8) bh[tid] = tid < kActions ? params[L.ba + tid] : ((tid == kActions && has_value) ? params[L.bv] : 0.0f);
+  float *b1 = reinterpret_cast<float *>(rest + kImgB1), *b2 = reinterpret_cast<float *>(rest + kImgB2), *bh = reinterpret_cast<float *>(rest + kImgBh);
+  for (int i = tid; i < kH; i += nth) { b1[i] = params[net.b1 + i]; b2[i] = params[net.b2 + i]; }
+  if (tid < 8) bh[tid] = (tid < kActions && net.has_actor) ? params[net.ba + tid] : ((tid == kActions && net.has_value) ? params[net.bv] : 0.0f);
 }
 
 __device__ __forceinline__ uint64_t desc_k(uint32_t tile, int C, int k) { return smem_desc(tile + k * 256, 128, C * 16); }
 __device__ __forceinline__ uint64_t desc_mn(uint32_t tile, int C, int k) { return smem_desc(tile + k * 2 * C * 16, C * 16, 128); }
 constexpr uint32_t kAmn = 1u << 15, kBmn = 1u << 16;
 
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ void stg_v4(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
-
-struct HeadOffsets { size_t ba, bv; };
 
 // ---- row kernel ------------------------------------------------------------------------------------------------------
 // Tiles [tile0, tile0 + n_tiles) of the minibatch; tile t's staging record is number t - tile0.
 __global__ void __launch_bounds__(kThreads, 1)
 ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyper hp, const double *__restrict__ adv_stats,
                    unsigned char *__restrict__ staging, long long tile0, int n_tiles, float *__restrict__ partial, size_t n_params,
-                   double *__restrict__ term_partial, int *status, HeadOffsets off, int D, int has_value) {
+                   double *__restrict__ term_partial, int *status, Net256 net) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   RowSmem &sm = *reinterpret_cast<RowSmem *>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row = tid & (kR - 1), half = tid >> 7;
-  const uint32_t bar_load = smem_u32(&sm.bar_load), bar_mma = smem_u32(&sm.bar_mma);
+  const uint32_t bar_load = smem_u32(&sm.bar_load), bar_mma = smem_u32(&sm.bar_mma), bar_mmb = smem_u32(&sm.bar_mmb), bar_w1 = smem_u32(&sm.bar_w1);
+  const int D = net.D, slabs = net.slabs, has_value = net.has_value, has_actor = net.has_actor;
+  const StageLayout SL = stage_layout(slabs);
+  const unsigned char *image_rest = image + static_cast<size_t>(slabs) * kImgW2;  // W2 | Wh | biases
   if (tid == 0) {
-    mbar_init(bar_load, 1); mbar_init(bar_mma, 1);
+    mbar_init(bar_load, 1); mbar_init(bar_mma, 1); mbar_init(bar_mmb, 1); mbar_init(bar_w1, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -110,10 +140,12 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (tid == 0) {
-    mbar_expect_tx(bar_load, kImgBytes);
+  if (tid == 0) {  // everything but W1 stays for the whole run; with one slab W1 does too
     constexpr uint32_t kChunk = 16384;
-    for (uint32_t o = 0; o < kImgBytes; o += kChunk) bulk_load(smem_u32(sm.img + o), image + o, min(kChunk, kImgBytes - o), bar_load);
+    const uint32_t first = slabs == 1 ? 0u : kImgW2;
+    mbar_expect_tx(bar_load, kImgBytes - first);
+    for (uint32_t o = first; o < kImgBytes; o += kChunk)
+      bulk_load(smem_u32(sm.img + o), (o < kImgW2 ? image : image_rest - kImgW2) + o, min(kChunk, kImgBytes - o), bar_load);
   }
   bool timed_out = !mbar_wait(bar_load, 0);
   timed_out = __syncthreads_or(timed_out) != 0;
@@ -129,7 +161,7 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
   const float inv_n = 1.0f / static_cast<float>(rows.n);
   const int my_tiles = static_cast<int>(blockIdx.x) < n_tiles ? (n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
 
-  uint32_t ph = 0;
+  uint32_t ph = 0, phb = 0, ph_w1 = 0;
   double t_actor = 0.0, t_ent = 0.0, t_value = 0.0;
   float gbh = 0.0f;
   // this thread's 16-byte pieces of a staged activation: unit half `half`, its own row
@@ -196,7 +228,7 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
   for (int i = 0; i < my_tiles && !timed_out; ++i) {
     const int lt = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);  // tile inside the chunk
     const long long row0 = (tile0 + lt) * kR;
-    unsigned char *st = staging + static_cast<size_t>(lt) * kStTile;
+    unsigned char *st = staging + static_cast<size_t>(lt) * SL.tile;
     const int n_valid = static_cast<int>(min(static_cast<long long>(kR), rows.n - row0));
     const long long my_row = row < n_valid ? real_row(rows, row0 + row) : -1;
     int action = 0;
@@ -205,56 +237,77 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
       sm.rmap[row] = my_row;
       if (row < n_valid && my_row < 0) atomicExch(status, kStatusBadIndex);
       if (my_row >= 0) {
-        action = rows.actions[my_row]; logp_old = rows.logp_old[my_row]; adv = rows.adv[my_row];
+        if (has_actor) { action = rows.actions[my_row]; logp_old = rows.logp_old[my_row]; adv = rows.adv[my_row]; }
         if (has_value) { v_old = rows.value_old[my_row * rows.vstride]; ret = rows.ret[my_row * rows.vstride]; }
       }
     }
-    if (tid == 0) {
-      bulk_store_wait_read();  // the copies of the previous tile's x and dhead tiles have read them
-      // the next tile's rows on their way into L2 (a full tile of consecutive rows is one 16-byte aligned block)
-      if (rows.env_ids == nullptr && i + 1 < my_tiles && (tile0 + lt + static_cast<long long>(gridDim.x) + 1) * kR <= rows.n)
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(rows.x + static_cast<size_t>(tile0 + lt + gridDim.x) * kR * D),
-                     "r"(static_cast<uint32_t>(kR * D * 4))
-                     : "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    // ---- the tile's rows as bf16 into x: a warp per row, consecutive lanes consecutive features
-    {
-      constexpr int G = 8;
-      for (int g0 = warp; g0 < kR; g0 += 8 * G) {
-        float v[G][3];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-          const long long src = sm.rmap[g0 + 8 * g];
-#pragma unroll
-          for (int q = 0; q < 3; ++q) {
-            const int k = lane + 32 * q;
-            v[g][q] = (k < D && src >= 0) ? rows.x[src * D + k] : 0.0f;
-          }
+    // ---- layer 1, one input slab at a time: z1 = sum over slabs of x_a . W1_a^T
+    for (int a = 0; a < slabs; ++a) {
+      if (a > 0) {  // the previous slab's MMAs (both column halves) have read the x tile and the W1 slab
+        timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+        timed_out |= !mbar_wait(bar_mmb, phb); phb ^= 1;
+      }
+      if (tid == 0) {
+        bulk_store_wait_read();  // the copies of the x tile (and of the previous tile's dhead tile) have read them
+        if (slabs > 1) {         // this slab of W1 comes in while the rows are converted
+          mbar_expect_tx(bar_w1, kImgW2);
+          for (uint32_t o = 0; o < kImgW2; o += 16384)
+            bulk_load(smem_u32(sm.img + o), image + static_cast<size_t>(a) * kImgW2 + o, 16384, bar_w1);
         }
+        // the next tile's rows on their way into L2 (a full tile of consecutive rows is one 16-byte aligned block)
+        if (a == 0 && rows.env_ids == nullptr && i + 1 < my_tiles && (tile0 + lt + static_cast<long long>(gridDim.x) + 1) * kR <= rows.n)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(rows.x + static_cast<size_t>(tile0 + lt + gridDim.x) * kR * net.w1_ld),
+                       "r"(static_cast<uint32_t>(kR * net.w1_ld * 4))
+                       : "memory");
+      }
+      tc_fence_before();
+      __syncthreads();
+      // the tile's rows (slab a of each) as bf16 into x: a warp per row, consecutive lanes consecutive features
+      {
+        constexpr int G = 16;  // all of a warp's rows at once: one round trip to L2
+        for (int g0 = warp; g0 < kR; g0 += 8 * G) {
+          float v[G][3];
 #pragma unroll
-        for (int g = 0; g < G; ++g)
+          for (int g = 0; g < G; ++g) {
+            const long long src = sm.rmap[g0 + 8 * g];
 #pragma unroll
-          for (int q = 0; q < 3; ++q) {
-            const int k = lane + 32 * q;
-            if (k < D) sts_u16(xt + canon_offset(g0 + 8 * g, k, kK1), bf16_bits(v[g][q]));
+            for (int q = 0; q < 3; ++q) {
+              const int k = lane + 32 * q;
+              v[g][q] = (k < D && src >= 0) ? rows.x[src * net.w1_ld + a * D + k] : 0.0f;
+            }
           }
+#pragma unroll
+          for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int q = 0; q < 3; ++q) {
+              const int k = lane + 32 * q;
+              if (k < D) sts_u16(xt + a_offset<kK1>(g0 + 8 * g, k), bf16_bits(v[g][q]));
+            }
+        }
+      }
+      fence_async_smem();
+      __syncthreads();
+      if (tid == 0) {
+        bulk_store(st + SL.x + static_cast<size_t>(a) * kStXBytes, xt, static_cast<uint32_t>(kStXBytes));
+        if (slabs > 1) { timed_out |= !mbar_wait(bar_w1, ph_w1); ph_w1 ^= 1; }
+        tc_fence_after();
+#pragma unroll
+        // the product in two column halves with a commit each: a thread's epilogue needs its own half only
+#pragma unroll
+        for (int nh = 0; nh < 2; ++nh) {
+#pragma unroll
+          for (int k = 0; k < kK1 / 16; ++k)
+            mma_bf16(tmem + kColAcc + 128u * nh, smem_desc(xt + k * 2 * kXLbo, kXLbo, kXSbo), desc_k(w1 + nh * 16 * (kK1 * 16), kK1, k),
+                     instr_desc(kR, kH / 2), (a > 0) | (k > 0));
+          mma_commit(nh == 0 ? bar_mma : bar_mmb);
+        }
       }
     }
-    fence_async_smem();
-    __syncthreads();
-    if (tid == 0) {
-      bulk_store(st + kStX, xt, static_cast<uint32_t>(kStXBytes));
-      tc_fence_after();
-#pragma unroll
-      for (int k = 0; k < kK1 / 16; ++k) mma_bf16(tmem + kColAcc, desc_k(xt, kK1, k), desc_k(w1, kK1, k), instr_desc(kR, kH), k > 0);
-      mma_commit(bar_mma);
-    }
-    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    if (half == 0) { timed_out |= !mbar_wait(bar_mma, ph); } else { timed_out |= !mbar_wait(bar_mmb, phb); }
+    ph ^= 1; phb ^= 1;
     tc_fence_after();
     uint32_t gate1[4], gate2[4];
-    fwd_epilogue(b1, st + kStH1, gate1);
+    fwd_epilogue(b1, st + SL.h1, gate1);
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
@@ -265,7 +318,7 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
     }
     timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
     tc_fence_after();
-    fwd_epilogue(b2, st + kStH2, gate2);
+    fwd_epilogue(b2, st + SL.h2, gate2);
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
@@ -281,7 +334,7 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
       tmem_ld16(tmem + kColHead + lane_off, hv);
 #pragma unroll
       for (int k = 0; k < 8; ++k) d[k] = 0.0f;
-      if (my_row >= 0) {
+      if (my_row >= 0 && has_actor) {
         float l[kActions], m = -INFINITY, sum = 0.0f;
 #pragma unroll
         for (int k = 0; k < kActions; ++k) { l[k] = hv[k] + bh[k]; m = fmaxf(m, l[k]); }
@@ -305,7 +358,9 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
           d[k] = d_logp * ((k == action ? 1.0f : 0.0f) - p[k]) + hp.ent_coef * inv_n * p[k] * (lp[k] + ent);
         t_actor += fminf(s1, s2);
         t_ent += ent;
-        if (has_value) {
+      }
+      if (my_row >= 0 && has_value) {
+        {
           const float v = hv[kActions] + bh[kActions];
           const float u = v - ret, uc = v_old + fminf(fmaxf(v - v_old, -hp.clip_eps), hp.clip_eps) - ret;
           const bool in_range = fabsf(v - v_old) <= hp.clip_eps;
@@ -325,7 +380,7 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
     fence_async_smem(); tc_fence_before();
     __syncthreads();
     if (tid == 0) {
-      bulk_store(st + kStDh, dht, static_cast<uint32_t>(kStDhBytes));
+      bulk_store(st + SL.dh, dht, static_cast<uint32_t>(kStDhBytes));
       tc_fence_after();
       mma_bf16(tmem + kColAcc, desc_k(dht, kHeads, 0), desc_mn(wh, kH, 0), instr_desc(kR, kH) | kBmn, 0);  // d h2 = dhead . Wh
       mma_commit(bar_mma);
@@ -333,25 +388,29 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
     if (tid <= kActions) gbh += (sm.red[0][tid] + sm.red[1][tid]) + (sm.red[2][tid] + sm.red[3][tid]);
     timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
     tc_fence_after();
-    bwd_epilogue(gate2, st + kStDz2, true);
+    bwd_epilogue(gate2, st + SL.dz2, true);
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
       tc_fence_after();
 #pragma unroll
-      for (int k = 0; k < kH / 16; ++k)  // d h1 = d z2 . W2
-        mma_bf16_ts(tmem + kColAcc, tmem + kColHid + k * 8, desc_mn(w2, kH, k), instr_desc(kR, kH) | kBmn, k > 0);
-      mma_commit(bar_mma);
+      for (int nh = 0; nh < 2; ++nh) {  // d h1 = d z2 . W2, again in two column halves
+#pragma unroll
+        for (int k = 0; k < kH / 16; ++k)
+          mma_bf16_ts(tmem + kColAcc + 128u * nh, tmem + kColHid + k * 8, desc_mn(w2 + nh * 16 * 128, kH, k), instr_desc(kR, kH / 2) | kBmn, k > 0);
+        mma_commit(nh == 0 ? bar_mma : bar_mmb);
+      }
     }
-    timed_out |= !mbar_wait(bar_mma, ph); ph ^= 1;
+    if (half == 0) { timed_out |= !mbar_wait(bar_mma, ph); } else { timed_out |= !mbar_wait(bar_mmb, phb); }
+    ph ^= 1; phb ^= 1;
     tc_fence_after();
-    bwd_epilogue(gate1, st + kStDz1, false);
+    bwd_epilogue(gate1, st + SL.dz1, false);
     timed_out = __syncthreads_or(timed_out) != 0;
   }
   if (!timed_out) {
     float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
-    if (tid < kActions) part[off.ba + tid] += gbh;
-    if (tid == kActions && has_value) part[off.bv] += gbh;
+    if (tid < kActions && has_actor) part[net.ba + tid] += gbh;
+    if (tid == kActions && has_value) part[net.bv] += gbh;
   }
   {
     double s[3] = {t_actor, t_ent, t_value};
@@ -376,15 +435,15 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
 }
 
 // ---- weight kernel ---------------------------------------------------------------------------------------------------
-// CTAs [0, n_w2) sum d W2 and d b2; the others d W1, d b1 and d Wh.  A CTA's work items are 32-row pieces of the tiles it
-// owns; an item's operands come in by bulk copies into a ring of stages.  Roles inside the CTA, connected by mbarriers
+// CTAs [0, n_w2) sum d W2 and d b2; the others d W1 (one input slab each; CTA index modulo the slab count picks the
+// slab), and those of slab 0 also d b1 and d Wh.  A CTA's work items are 32-row pieces of the tiles it owns; an item's operands come in by bulk copies into a ring of stages.  Roles inside the CTA, connected by mbarriers
 // only: one producer thread (copies), one MMA thread, eight consumer warps (thread j sums column j of the d z tile for
 // the bias gradient).  A stage is free again when its MMAs have completed and every consumer warp has let go of it.
 constexpr int kItemRows = 32;
 constexpr int kItemsPerTile = kR / kItemRows;
 constexpr uint32_t kQ = kItemRows * 128 * 2;                  // an item's rows of a [128][128] unit-half tile: 8 KB
 constexpr uint32_t kW2Stage = 4 * kQ, kW2Stages = 6;          // d z2 (two unit halves), h1 (two unit halves)
-constexpr uint32_t kXPart = kItemRows * kK1 * 2, kDhPart = kItemRows * kHeads * 2;
+constexpr uint32_t kXPart = (kItemRows / 8) * kXSbo, kDhPart = kItemRows * kHeads * 2;
 constexpr uint32_t kW1Stage = 4 * kQ + kXPart + kDhPart, kW1Stages = 5;  // d z1, h2 (two unit halves each), x, dhead
 constexpr uint32_t kRingBytes = kW2Stage * kW2Stages > kW1Stage * kW1Stages ? kW2Stage * kW2Stages : kW1Stage * kW1Stages;
 constexpr int kMaxStages = 6;
@@ -396,17 +455,20 @@ struct WgtSmem {
   uint32_t tmem_base;
 };
 
-struct WgtOffsets { size_t W1, b1, W2, b2, Wa, Wv; };
-
 __global__ void __launch_bounds__(kWgtThreads, 1)
 ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, int n_w2, float *__restrict__ partial, size_t n_params,
-                      int *status, WgtOffsets off, int D, int has_value) {
+                      int *status, Net256 net) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   WgtSmem &sm = *reinterpret_cast<WgtSmem *>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool role_w2 = static_cast<int>(blockIdx.x) < n_w2;
-  const int rank = role_w2 ? static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x) - n_w2;
-  const int peers = role_w2 ? n_w2 : static_cast<int>(gridDim.x) - n_w2;
+  const int D = net.D, slabs = net.slabs, has_value = net.has_value, has_actor = net.has_actor;
+  const StageLayout SL = stage_layout(slabs);
+  const int rest = static_cast<int>(gridDim.x) - n_w2;                                  // CTAs of the d W1 group
+  const int slab = role_w2 ? 0 : (static_cast<int>(blockIdx.x) - n_w2) % slabs;          // input slab of this CTA
+  const int rank = role_w2 ? static_cast<int>(blockIdx.x) : (static_cast<int>(blockIdx.x) - n_w2) / slabs;
+  const int peers = role_w2 ? n_w2 : rest / slabs + (slab < rest % slabs ? 1 : 0);
+  const bool heads_too = !role_w2 && slab == 0;                                          // d Wh and d b1 ride with slab 0
   const int S = role_w2 ? kW2Stages : kW1Stages;
   const uint32_t stage_bytes = role_w2 ? kW2Stage : kW1Stage;
   const uint32_t ring = smem_u32(sm.ring), full0 = smem_u32(&sm.full[0]), empty0 = smem_u32(&sm.empty[0]), done_bar = smem_u32(&sm.done);
@@ -440,18 +502,19 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
         const int s = u % S;
         if (u >= S) timed_out |= !mbar_wait(empty0 + 8u * s, ((u / S) - 1) & 1);
         if (timed_out) break;
-        const int lt = rank + (u / kItemsPerTile) * peers, q = u % kItemsPerTile;
-        const unsigned char *st = staging + static_cast<size_t>(lt) * kStTile;
+        // the chunk's last tiles first: the row kernel wrote them last, so they are the ones still in L2
+        const int lt = n_tiles - 1 - (rank + (u / kItemsPerTile) * peers), q = u % kItemsPerTile;
+        const unsigned char *st = staging + static_cast<size_t>(lt) * SL.tile;
         const uint32_t dst = ring + static_cast<uint32_t>(s) * stage_bytes, bar = full0 + 8u * s;
         mbar_expect_tx(bar, stage_bytes);
-        const size_t a = role_w2 ? kStDz2 : kStDz1, b = role_w2 ? kStH1 : kStH2;
+        const size_t a = role_w2 ? SL.dz2 : SL.dz1, b = role_w2 ? SL.h1 : SL.h2;
         bulk_load(dst, st + a + static_cast<size_t>(q) * kQ, kQ, bar);
         bulk_load(dst + kQ, st + a + kHalfBytes + static_cast<size_t>(q) * kQ, kQ, bar);
         bulk_load(dst + 2 * kQ, st + b + static_cast<size_t>(q) * kQ, kQ, bar);
         bulk_load(dst + 3 * kQ, st + b + kHalfBytes + static_cast<size_t>(q) * kQ, kQ, bar);
         if (!role_w2) {
-          bulk_load(dst + 4 * kQ, st + kStX + static_cast<size_t>(q) * kXPart, kXPart, bar);
-          bulk_load(dst + 4 * kQ + kXPart, st + kStDh + static_cast<size_t>(q) * kDhPart, kDhPart, bar);
+          bulk_load(dst + 4 * kQ, st + SL.x + static_cast<size_t>(slab) * kStXBytes + static_cast<size_t>(q) * kXPart, kXPart, bar);
+          bulk_load(dst + 4 * kQ + kXPart, st + SL.dh + static_cast<size_t>(q) * kDhPart, kDhPart, bar);
         }
         issued = u + 1;
       }
@@ -480,10 +543,11 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
           for (int k = 0; k < kItemRows / 16; ++k)
 #pragma unroll
             for (int a = 0; a < 2; ++a) {
-              mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * kQ, 128, k), desc_mn(base + 4 * kQ, kK1, k),
+              mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * kQ, 128, k), smem_desc(base + 4 * kQ + k * 2 * kXSbo, kXSbo, kXLbo),
                        instr_desc(128, kK1) | kAmn | kBmn, keep | (k > 0));
-              mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * kQ, 128, k), desc_mn(base + 4 * kQ + kXPart, kHeads, k),
-                       instr_desc(128, kHeads) | kAmn | kBmn, keep | (k > 0));
+              if (heads_too)
+                mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * kQ, 128, k), desc_mn(base + 4 * kQ + kXPart, kHeads, k),
+                         instr_desc(128, kHeads) | kAmn | kBmn, keep | (k > 0));
             }
         }
         mma_commit(empty0 + 8u * s);  // the stage is free once these MMAs have read it
@@ -491,16 +555,36 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
       if (!timed_out && n_items > 0) mma_commit(done_bar);  // covers every MMA issued above
     }
   } else {
-    // ---- consumers: this thread's unit, summed over the item's rows in row order
-    const uint32_t my_col = static_cast<uint32_t>(tid >> 7) * kQ + static_cast<uint32_t>(((tid & 127) >> 3) * 128 + (tid & 7) * 2);
+    // ---- consumers: column sums of the d z tile for the bias gradient.  Warp w covers feature chunks 4 w .. 4 w + 3 (units
+    // 32 w .. 32 w + 31); lane l reads row l's 16-byte piece of a chunk (a warp's 32 pieces are 512 contiguous-by-group
+    // bytes: no bank conflict beyond the four wavefronts 512 bytes need), the eight values are summed over the lanes by
+    // a butterfly, and lane l keeps the sum of unit 32 w + l.  Fixed order: the same bytes on every call.
+    const uint32_t row_off = static_cast<uint32_t>((lane >> 3) * 2048 + (lane & 7) * 16);
     for (int u = 0; u < n_items && !timed_out; ++u) {
       const int s = u % S;
       const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
       timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
       if (__any_sync(0xFFFFFFFFu, timed_out)) { timed_out = true; break; }
-#pragma unroll 8
-      for (int r = 0; r < kItemRows; ++r)
-        db += __uint_as_float(lds_u16(base + my_col + static_cast<uint32_t>((r >> 3) * 2048 + (r & 7) * 16)) << 16);
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const int chunk = 4 * warp + cc;  // 0..31: unit half chunk >> 4, chunk inside it chunk & 15
+        const uint4 q = lds_v4(base + static_cast<uint32_t>(chunk >> 4) * kQ + static_cast<uint32_t>(chunk & 15) * 128u + row_off);
+        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { v[2 * e] = __uint_as_float(w4[e] << 16); v[2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u); }
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v[e] += __shfl_xor_sync(0xFFFFFFFFu, v[e], o);
+        float pick = v[0];
+#pragma unroll
+        for (int e = 1; e < 8; ++e) pick = ((lane & 7) == e) ? v[e] : pick;
+        if ((lane >> 3) == cc) db += pick;
+      }
+      // the stage's next writer is a bulk copy (async proxy); these were generic-proxy reads.  Without the proxy fence
+      // the copy may land before the reads have been performed (seen on the GPU as bias sums that changed from call to call).
+      fence_async_smem();
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8u * s) : "memory");
     }
@@ -518,21 +602,24 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
       for (int b = 0; b < 2; ++b)
         for (int c0 = 0; c0 < 128; c0 += 16) {
           tmem_ld16(tmem + lane_off + static_cast<uint32_t>((a * 2 + b) * 128 + c0), v);
-          float *dst = part + off.W2 + static_cast<size_t>(unit) * kH + b * 128 + c0;
+          float *dst = part + net.W2 + static_cast<size_t>(unit) * kH + b * 128 + c0;
 #pragma unroll
           for (int c = 0; c < 16; ++c) dst[c] += v[c];
         }
-      part[off.b2 + tid] += db;
+      part[net.b2 + tid] += db;
     } else {
       for (int c0 = 0; c0 < kK1; c0 += 16) {
         tmem_ld16(tmem + lane_off + static_cast<uint32_t>(a * kK1 + c0), v);
         for (int c = 0; c < 16; ++c)
-          if (c0 + c < D) part[off.W1 + static_cast<size_t>(unit) * D + c0 + c] += v[c];
+          if (c0 + c < D) part[net.W1 + static_cast<size_t>(unit) * net.w1_ld + slab * D + c0 + c] += v[c];
       }
-      tmem_ld16(tmem + lane_off + static_cast<uint32_t>(192 + a * 32), v);
-      for (int k = 0; k < kActions; ++k) part[off.Wa + static_cast<size_t>(k) * kH + unit] += v[k];
-      if (has_value) part[off.Wv + unit] += v[kActions];
-      part[off.b1 + tid] += db;
+      if (heads_too) {
+        tmem_ld16(tmem + lane_off + static_cast<uint32_t>(192 + a * 32), v);
+        if (has_actor)
+          for (int k = 0; k < kActions; ++k) part[net.Wa + static_cast<size_t>(k) * kH + unit] += v[k];
+        if (has_value) part[net.Wv + unit] += v[kActions];
+        part[net.b1 + tid] += db;
+      }
     }
   }
   if (timed_out && tid == 0) atomicExch(status, kStatusTimeout);
@@ -547,13 +634,16 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
 }  // namespace
 
 bool ppo_tc256_supported(const mava_config_t &cfg, int D) { return cfg.hidden == kH && D <= kK1 && D > 64; }
-size_t ppo_tc256_image_bytes() { return kImgBytes; }
-size_t ppo_tc256_staging_bytes(int chunk_tiles) { return static_cast<size_t>(chunk_tiles) * kStTile; }
+size_t ppo_tc256_image_bytes(int slabs) { return static_cast<size_t>(slabs - 1) * kImgW2 + kImgBytes; }
+size_t ppo_tc256_staging_bytes(int chunk_tiles, int slabs) { return static_cast<size_t>(chunk_tiles) * stage_layout(slabs).tile; }
 
-cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const ParamLayout &L, const UpdRows &rows, const UpdHyper &hp,
+cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const Tc256Net &desc, const UpdRows &rows, const UpdHyper &hp,
                                  const double *adv_stats, void *image, void *staging, int chunk_tiles, float *partial, size_t n_params,
-                                 double *term_partial, int slices, bool has_value) {
-  prep_upd256_kernel<<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(image), L, h->D, has_value ? 1 : 0);
+                                 double *term_partial, int slices) {
+  Net256 net{};
+  net.W1 = desc.W1; net.b1 = desc.b1; net.W2 = desc.W2; net.b2 = desc.b2; net.Wa = desc.Wa; net.ba = desc.ba; net.Wv = desc.Wv; net.bv = desc.bv;
+  net.D = h->D; net.slabs = desc.slabs; net.w1_ld = desc.slabs * h->D; net.has_actor = desc.has_actor ? 1 : 0; net.has_value = desc.has_value ? 1 : 0;
+  prep_upd256_kernel<<<64, 256, 0, h->stream>>>(params_dev, static_cast<unsigned char *>(image), net);
   h->launches += 1;
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
@@ -562,17 +652,17 @@ cudaError_t launch_ppo_net_tc256(mava_rollout *h, const float *params_dev, const
     err = cudaFuncSetAttribute(ppo_weights256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(WgtSmem)));
   if (err != cudaSuccess) return err;
   const long long tiles = (rows.n + kR - 1) / kR;
-  const HeadOffsets ho{L.ba, L.bv};
-  const WgtOffsets wo{L.W1, L.b1, L.W2, L.b2, L.Wa, L.Wv};
-  // CTAs of the weight kernel by the bytes each group streams per tile (128 KB against 156 KB)
-  const int n_w2 = slices >= 2 ? (slices * 128 + 142) / 284 : 1;
+  // CTAs of the weight kernel by the bytes each group streams per tile: 128 KB for d W2 against 156 KB per input slab
+  int n_w2 = (slices * 128 + (128 + 156 * net.slabs) / 2) / (128 + 156 * net.slabs);
+  if (n_w2 < 1) n_w2 = 1;
+  if (slices - n_w2 < net.slabs) return cudaErrorInvalidConfiguration;  // every slab needs a CTA
   for (long long t0 = 0; t0 < tiles; t0 += chunk_tiles) {
     const int nt = static_cast<int>(tiles - t0 < chunk_tiles ? tiles - t0 : chunk_tiles);
     ppo_rows256_kernel<<<slices, kThreads, sizeof(RowSmem), h->stream>>>(static_cast<const unsigned char *>(image), rows, hp, adv_stats,
                                                                          static_cast<unsigned char *>(staging), t0, nt, partial, n_params,
-                                                                         term_partial, h->d_status, ho, h->D, has_value ? 1 : 0);
+                                                                         term_partial, h->d_status, net);
     ppo_weights256_kernel<<<slices, kWgtThreads, sizeof(WgtSmem), h->stream>>>(static_cast<const unsigned char *>(staging), nt, n_w2, partial,
-                                                                            n_params, h->d_status, wo, h->D, has_value ? 1 : 0);
+                                                                               n_params, h->d_status, net);
     h->launches += 2;
   }
   return cudaGetLastError();

@@ -178,23 +178,17 @@ def test_minibatches_of_environments(idx, n_envs, T):
 # operand, logits good to 2e-2): 5e-2 * max|grad| and 2e-2 * (1 + |ref|).
 
 def _tensor_path_reference(w, shapes, p64, batch, hp, emulate):
-    """Oracle loss terms and gradient for the tensor-core path.  With a centralised critic only the actor net runs on
-    the tensor cores; the critic's net stays on the fp32 kernel, so in bf16-operand mode its loss term and its layers'
-    gradients are the exact oracle's (the two nets share no parameter)."""
+    """Oracle loss terms and gradient for the tensor-core path (with a centralised critic both nets take it)."""
     ref = ppo.ppo_loss(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
     ref_grad = ppo.ppo_grad(p64, shapes, w["net_kind"], batch, emulate_bf16=emulate)
-    if emulate and w["net_kind"] == 1:
-        exact = ppo.ppo_loss(p64, shapes, 1, batch)
-        ref = dict(ref, value=exact["value"], total=ref["actor"] - hp.ent_coef * ref["entropy"] + hp.vf_coef * exact["value"])
-        n_actor = sum(o * i + o for _, (o, i) in shapes[:3])
-        ref_grad = np.concatenate([ref_grad[:n_actor], ppo.ppo_grad(p64, shapes, 1, batch)[n_actor:]])
     return ref, ref_grad
 
 
 @pytest.mark.parametrize("idx,n_envs,T", [(0, 16, 32), (1, 77, 20), (2, 50, 33), (2, 300, 40), (0, 1, 3),
                                           (1, 1024, 128),  # the size the benchmark times
-                                          # H = 256: row kernel + weight kernel (with the centralised critic: the actor net)
-                                          (4, 21, 11), (4, 150, 40), (3, 45, 17), (3, 300, 20), (4, 1, 2)])
+                                          # H = 256: row kernel + weight kernel (with the centralised critic: both nets,
+                                          # the critic's first layer one agent's observation at a time)
+                                          (4, 21, 11), (4, 150, 40), (3, 45, 17), (3, 300, 20), (4, 1, 2), (3, 2, 3)])
 def test_tensor_core_update_matches_the_bf16_operand_oracle(idx, n_envs, T):
     import torch
 
@@ -214,12 +208,20 @@ def test_tensor_core_update_matches_the_bf16_operand_oracle(idx, n_envs, T):
         ref, ref_grad = _tensor_path_reference(w, shapes, p64, batch, hp, emulate)
         for k, name in enumerate(("total", "actor", "entropy", "value")):
             assert abs(t[k] - ref[name]) <= l_tol * (1 + abs(ref[name])), (emulate, name, t[k], ref[name])
+        if not emulate and n_envs * T * w["n_agents"] < 1024:
+            # a few dozen rows: one row whose ratio lands on the other side of a clip boundary once the operands are
+            # rounded is several percent of the gradient, so the comparison with exact arithmetic says nothing here
+            continue
         worst = np.max(np.abs(gg - ref_grad)) / np.max(np.abs(ref_grad))
         assert worst <= g_tol, (emulate, worst)
-        # layer by layer as well: a layer with small gradients must not hide behind the largest one
+        # layer by layer as well: a layer with small gradients must not hide behind the largest one.  Against exact
+        # arithmetic only the weight matrices are judged this way: a head's bias gradient is one number, the sum of
+        # the rows' signed derivatives, which nearly cancels, so its own size is no scale for the operands' rounding.
         off = 0
         for name, (o, i) in shapes:
             for lo, hi in ((off, off + o * i), (off + o * i, off + o * i + o)):
+                if not emulate and hi - lo < 8:
+                    continue
                 seg = np.max(np.abs(ref_grad[lo:hi]))
                 assert np.max(np.abs(gg[lo:hi] - ref_grad[lo:hi])) <= 5 * g_tol * seg + 1e-12, (emulate, name, lo)
             off += o * i + o
