@@ -74,7 +74,13 @@ struct TcShape {
   // that one group's environment phase (sampler, transition, observation) overlaps the other's
   // network phase (the three MMAs and their epilogues).
   static constexpr bool PINGPONG = TM && GROUPS == 1;
-  static constexpr int THREADS = 2 * kGroupThreads;
+  // In ping-pong mode a third warpgroup sends the observation blocks out (bf16 A tile -> fp32 rows of the obs array):
+  // on the two thread groups' own time that copy was a quarter of the step.
+  static constexpr bool HELPERS = PINGPONG;
+  static constexpr int THREADS = (HELPERS ? 3 : 2) * kGroupThreads;
+  // Registers: the block starts with 65536 / 384 rounded down to a multiple of 8 per thread; the helpers give theirs
+  // back (kHelperRegs) and the two groups take kGroupRegs each: 256 * 200 + 128 * 72 = 60416 <= 384 * 160.
+  static constexpr int kGroupRegs = 200, kHelperRegs = 72;
 };
 
 template <int N, int F, int H, bool TM>
@@ -96,6 +102,7 @@ struct TcSmem {
   alignas(8) uint64_t load_bar;
   uint32_t tmem_base;
   int abort;  // ping-pong mode: a group gave up; both finish their barrier protocol without work
+  int copy_rows[2];  // ping-pong mode, per group: rows of the step's observation block the helpers send out (0: none)
 };
 
 
@@ -313,10 +320,13 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   using S = TcShape<N, H, TM>;
   constexpr int D = S::D, K1 = S::K1;
   constexpr bool PP = S::PINGPONG;
+  constexpr bool HP = S::HELPERS;       // the third warpgroup sends the observation blocks out
+  constexpr int TP = HP ? 3 : 2;        // parties of the A tile's hand-over barrier
   extern __shared__ __align__(128) unsigned char smem_raw[];
   TcSmem<N, F, H, TM> &sm = *reinterpret_cast<TcSmem<N, F, H, TM> *>(smem_raw);
   const int tid = threadIdx.x;
-  const int g = tid / kGroupThreads;   // thread group
+  const bool helper = HP && tid >= 2 * kGroupThreads;
+  const int g = helper ? 0 : tid / kGroupThreads;   // thread group
   const int dg = PP ? 0 : g;           // the set of tile resources it uses
   const int row = tid % kGroupThreads; // row of the tile this thread owns; also its TMEM lane
   const int warp = tid / 32, lane = tid & 31;
@@ -337,7 +347,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (!PP || g == 0) {  // zero the observation block and the A operand once
+  if ((!PP || g == 0) && !helper) {  // zero the observation block and the A operand once
     uint4 *z = reinterpret_cast<uint4 *>(gs.x);
     for (int i = row; i < static_cast<int>(S::X_BYTES / 16); i += kGroupThreads) z[i] = make_uint4(0, 0, 0, 0);
     z = reinterpret_cast<uint4 *>(gs.a);
@@ -378,10 +388,45 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
   const int ag = lane % N;                // its agent
   const int crow = le * N + ag;           // compact row inside the tile's block
 
+  if (helper) {
+    if constexpr (HP) {
+      // ---- helper warpgroup: for every step of either group, in the order in which the groups use the A tile, wait
+      // until the step's observations are in the tile, expand the rows the group asks for to fp32 in the obs array
+      // (warp w the rows of the group's warp w), and let go of the tile.  The loop bounds are those of the groups,
+      // which in ping-pong mode walk through every step's barriers whatever happens to them.
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(S::kHelperRegs));
+      QuadPlan<D, K1> quad_plan;
+      if (N % 4 == 0) plan_quads<D, K1>(quad_plan, lane);
+      pair_arrive(kBarTile + 0, TP);  // group 0 goes first
+      const volatile int *copy_rows = sm.copy_rows;
+      for (int it = 0;; ++it) {
+        const int tile0 = (it * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x)) * groups;
+        if (tile0 >= n_tiles) break;
+        for (int t = 0; t <= (EVAL ? a.T - 1 : a.T); ++t) {
+          for (int hg = 0; hg < 2; ++hg) {
+            pair_sync(kBarReady + hg);
+            const int n_rows = copy_rows[hg];
+            if (n_rows > 0) {
+              const int e0 = (tile0 + hg) * ept;
+              float *dst = (t == a.T) ? a.obs_last + static_cast<size_t>(e0) * N * D
+                                      : a.buf.obs + (static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N) * D;
+              if constexpr (N % 4 == 0)
+                expand_quads<D, K1>(quad_plan, a_addr, frac_addr, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+              else
+                expand_rows<D, K1>(a_addr, frac_addr, dst, wg * S::RPW, min(S::RPW, n_rows - wg * S::RPW), wg * 32, lane);
+            }
+            pair_arrive(kBarTile + (1 - hg), TP);
+          }
+        }
+      }
+    }
+  } else {
+  // ---- the two thread groups (everything up to the common exit) ------------------------------------------------
+  if constexpr (HP) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(S::kGroupRegs));
   QuadPlan<D, K1> quad_plan;
-  if (PP && N % 4 == 0) plan_quads<D, K1>(quad_plan, lane);
+  if (PP && !HP && N % 4 == 0) plan_quads<D, K1>(quad_plan, lane);
   if (PP && g == 1) {  // group 0 goes first on both shared resources
-    pair_arrive(kBarTile + 0);
+    pair_arrive(kBarTile + 0, TP);
     pair_arrive(kBarTmem + 0);
     pair_arrive(kBarHid + 0);
   }
@@ -442,14 +487,18 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       const bool last = !ev && (t == a.T);
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
       if (PP) {
-        pair_sync(kBarTile + g);  // the other group is done with the A tile
+        pair_sync(kBarTile + g, TP);  // the other group (and the helpers' copy of its rows) is done with the A tile
         // one verdict for the whole group (its threads may see the flag at different times); the flag
         // is looked at every eighth step only: the load would queue behind the partner's copy-out
         idle = group_any(g, idle || ((t & 7) == 0 && lds_s32(abort_addr) != 0));
         if (idle) {  // keep the hand-over order of a working step: three acquisitions, then three releases
+          if (HP) {    // nothing for the helpers to copy
+            if (row == 0) *reinterpret_cast<volatile int *>(&sm.copy_rows[g]) = 0;
+            pair_arrive(kBarReady + g);
+          }
           pair_sync(kBarTmem + g);
           pair_sync(kBarHid + g);
-          pair_arrive(kBarTile + (1 - g));
+          pair_arrive(kBarTile + (1 - g), TP);
           pair_arrive(kBarTmem + (1 - g));
           pair_arrive(kBarHid + (1 - g));
           continue;
@@ -472,6 +521,12 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
           sts_u16(a_row + a_offset<K1>(0, D), 0x3F80);
           sts_u16(a_row + a_offset<K1>(0, D + 1), 0x3F80);
         }
+      }
+      if (HP) {  // the helpers take the rows from here (the observation after the last step feeds a centralised critic)
+        if (row == 0)
+          *reinterpret_cast<volatile int *>(&sm.copy_rows[g]) = (!EVAL && (t < a.T || a.obs_last != nullptr)) ? n_rows : 0;
+        __threadfence_block();
+        pair_arrive(kBarReady + g);
       }
       fence_async_smem();
       tc_fence_before();
@@ -510,6 +565,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
         if (bulk_pending) { bulk_store_wait_read(); bulk_pending = false; }
         group_sync(g);
       }
+      if (HP) pair_arrive(kBarTile + (1 - g), TP);  // layer 1 has read the A tile; the helpers let go of it on their own
       if (PP) pair_sync(kBarHid + g);  // the other group's heads MMA has read the hidden-activation columns
       tc_fence_after();
       hidden_epilogue<H, TM>(acc_col + lane_off, hid_col + lane_off, stage_addr, row);
@@ -532,7 +588,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       } else if (!TM) {
         for (int i = row; i < static_cast<int>(S::A_BYTES / 16); i += kGroupThreads) sts_zero16(a_addr + 16u * i);
       }
-      if (PP) {
+      if (PP && !HP) {
         if (!ev && (!last || a.obs_last != nullptr)) {  // the observation after the last step feeds a centralised critic
           float *dst = last ? a.obs_last + static_cast<size_t>(e0) * N * D : obs_dst;
           if constexpr (N % 4 == 0)
@@ -634,6 +690,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
     }
   }
   if (timed_out && row == 0) atomicExch(a.status, kStatusTimeout);
+  }  // thread groups
 
   bulk_store_wait_all();  // bulk stores of this thread, if any, have landed
   // ---- common exit: every thread arrives here; tensor memory is returned ----------------------

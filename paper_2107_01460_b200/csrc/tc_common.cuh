@@ -92,16 +92,20 @@ __device__ __forceinline__ void group_sync(int g) {
   asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "r"(kGroupThreads) : "memory");
 }
 // Producer/consumer halves of a named barrier shared by the two thread groups of a CTA.
-__device__ __forceinline__ void pair_arrive(int id) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
+__device__ __forceinline__ void pair_arrive(int id, int parties = 2) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(parties * kGroupThreads) : "memory");
 }
-__device__ __forceinline__ void pair_sync(int id) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(2 * kGroupThreads) : "memory");
+__device__ __forceinline__ void pair_sync(int id, int parties = 2) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(parties * kGroupThreads) : "memory");
 }
 // Ping-pong hand-over barriers (ids 1..2 belong to the groups): group g waits on kBar* + g for
 // the A tile / the accumulator columns / the hidden-activation columns of tensor memory, and the
 // other group arrives there when it lets go.
 constexpr int kBarTile = 8, kBarTmem = 10, kBarHid = 12;
+// With a helper warpgroup for the observation copy-out: group g arrives on kBarReady + g when its observations are in
+// the A tile, the helpers wait there; and the A tile changes hands (kBarTile) when the group's layer-1 MMA and the
+// helpers' copy have both read it: three parties of 128 threads.
+constexpr int kBarReady = 14;
 // Barrier of the group that also ORs a predicate over its threads.
 __device__ __forceinline__ bool group_any(int g, bool pred) {
   uint32_t out;
