@@ -58,8 +58,9 @@ extern "C" {
 #define MAVA_PRECISION_BF16 1 /* bf16 operands, fp32 accumulation on the tcgen05 tensor cores      */
 
 #define MAVA_FLAG_WRITE_LOGITS 1 /* also write the six logits of every row to buffers.logits       */
-#define MAVA_FLAG_HIDDEN_IN_TMEM 2 /* bf16 path, H <= 128: keep hidden activations in tensor memory
-                                      (the layout H = 256 always uses); results are identical     */
+#define MAVA_FLAG_HIDDEN_IN_TMEM 2 /* bf16 path, H = 64: keep hidden activations in tensor memory (the layout the 128-row
+                                      kernel always uses from H = 128 on); at H = 128 the flag only selects the 128-row
+                                      kernel like MAVA_FLAG_WIDE_TILES; results are identical */
 #define MAVA_FLAG_WIDE_TILES 4 /* bf16 path: always use 128-row tiles, also for batches small
                                   enough for the few-rows form of the kernel; results are identical */
 

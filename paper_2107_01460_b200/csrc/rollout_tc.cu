@@ -58,13 +58,16 @@ struct TcShape {
   static constexpr uint32_t IMAGE_BYTES = ONES_OFF + ONES_BYTES;
   static constexpr uint32_t A_BYTES = (kTileRows / 8) * (K1 / 8) * 144;  // padded core-matrix pitch, see a_offset
   static constexpr uint32_t STAGE_BYTES = (kTileRows * D * 4 + 15) / 16 * 16;
-  static constexpr uint32_t X_BYTES =
-      TM ? 16 : (STAGE_BYTES > kTileRows * H * 2 ? STAGE_BYTES : kTileRows * H * 2);
   // Tensor-memory columns of one group: accumulator (reused by both hidden layers), the bf16
   // hidden activations (two per column) when TM, the heads accumulator.
   static constexpr int HID_COL = H;
   static constexpr int HEAD_COL = H + (TM ? H / 2 : 0);
   static constexpr int GROUP_COLS = HEAD_COL + 64;  // two heads accumulators: one per thread group in ping-pong mode
+  // TM with room for two groups' columns (H <= 128): the fp32 observation block is kept as well and leaves as a bulk
+  // copy.  Nothing else lives in its memory, so the copy has a whole step to read it.
+  static constexpr bool STG = TM && 2 * GROUP_COLS <= 512;
+  static constexpr uint32_t X_BYTES =
+      TM ? (STG ? STAGE_BYTES : 16) : (STAGE_BYTES > kTileRows * H * 2 ? STAGE_BYTES : kTileRows * H * 2);
   // independent sets of tile resources (A tile, block, tensor-memory columns) per CTA
   static constexpr int GROUPS = (2 * GROUP_COLS <= 512 && 2 * (A_BYTES + X_BYTES) + IMAGE_BYTES <= 220 * 1024) ? 2 : 1;
   static constexpr int TMEM_COLS = GROUPS * GROUP_COLS <= 256 ? 256 : 512;
@@ -511,7 +514,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       if (active) {
         const uint32_t a_row = a_addr + a_offset<K1>(row, 0);
         auto put = [&](int j, float v) {
-          if (!TM) sts_f32(stage_addr + 4u * static_cast<uint32_t>(crow * D + j), v);
+          if (!TM || S::STG) sts_f32(stage_addr + 4u * static_cast<uint32_t>(crow * D + j), v);
           else if (j == 3 * kPlane + 1) sts_f32(frac_addr + 4u * static_cast<uint32_t>(row), v);
           sts_u16(a_row + a_offset<K1>(0, j), bf16_bits(v));
         };
@@ -542,7 +545,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       flush_outputs();  // the previous step's rows
       float *obs_dst = a.buf.obs + row0 * D;
       if (!last && !PP && !ev) {
-        if (!TM) {  // one contiguous piece of the time-major array
+        if (!TM || S::STG) {  // one contiguous piece of the time-major array
           // by the bulk-copy engine when alignment allows: it leaves the load/store pipe to the
           // other group; the block was fenced for the async proxy together with the A tile
           const int count = n_rows * D;
@@ -606,12 +609,15 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       if (!TM) fence_async_smem();
       tc_fence_before();
       if (PP) pair_arrive(kBarTmem + (1 - g));  // this thread is done with the accumulator columns
+      if (S::STG && bulk_pending) { bulk_store_wait_read(); bulk_pending = false; }  // the block is zeroed after this barrier
       group_sync(g);
       // 4. heads: six logits and the value, N padded to 16
       if (row == 0) {
         tc_fence_after();
         issue_layer<H, kHeadRows, false, TM>(head_col, h_addr, w_addr + S::WH_OFF, 0u, 0u, bar);
       }
+      if (S::STG)  // while the heads run: zero the observation block for the next step (its copy has read it)
+        for (int i = row; i < static_cast<int>(S::STAGE_BYTES / 16); i += kGroupThreads) sts_zero16(stage_addr + 16u * i);
       timed_out |= !mbar_wait(bar, phase);
       phase ^= 1;
       if (PP) pair_arrive(kBarHid + (1 - g));  // the heads MMA is done reading the hidden-activation columns
@@ -708,7 +714,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
 template <int N, int H, bool TM>
 int few_rows_tile(const mava_rollout *h, int sms) {
   if constexpr (!TM && H == kTileRows) {
-    if ((h->cfg.flags & MAVA_FLAG_WIDE_TILES) == 0) {
+    if ((h->cfg.flags & (MAVA_FLAG_WIDE_TILES | MAVA_FLAG_HIDDEN_IN_TMEM)) == 0) {  // either flag asks for the 128-row kernel
       if (h->cfg.n_envs <= sms * SmallShape<N, H, 16>::EPT_MAX) return 16;
       if (h->cfg.n_envs <= sms * SmallShape<N, H, 32>::EPT_MAX) return 32;
     }
@@ -719,19 +725,19 @@ int few_rows_tile(const mava_rollout *h, int sms) {
 template <int N, int F, int H, bool TM, int ENV = 0>
 cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   using S = TcShape<N, H, TM>;
-  auto kern = args.eval ? rollout_tc_kernel<N, F, H, TM, true, ENV> : rollout_tc_kernel<N, F, H, TM, false, ENV>;
-  const size_t smem = sizeof(TcSmem<N, F, H, TM>);
-  cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (err != cudaSuccess) return err;
   int sms = 0;
-  err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+  cudaError_t err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
   if (err != cudaSuccess) return err;
   // Few rows per SM: the form with the rows as the N operand of the MMA.
-  if constexpr (!TM && H == kTileRows && ENV == 0) {
-    const int rb = few_rows_tile<N, H, TM>(h, sms);
+  if constexpr (H == kTileRows && ENV == 0) {
+    const int rb = few_rows_tile<N, H, false>(h, sms);
     if (rb == 16) return launch_tc_small<N, F, H, 16>(h, args, sms);
     if (rb == 32) return launch_tc_small<N, F, H, 32>(h, args, sms);
   }
+  auto kern = args.eval ? rollout_tc_kernel<N, F, H, TM, true, ENV> : rollout_tc_kernel<N, F, H, TM, false, ENV>;
+  const size_t smem = sizeof(TcSmem<N, F, H, TM>);
+  err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (err != cudaSuccess) return err;
   // Environments per tile: full tiles when there is enough work for every group of every SM,
   // otherwise smaller tiles so that all groups have one (the per-step chain is latency-bound).
   // Two thread groups per CTA, unless one group per SM already holds all environments: alone on
@@ -741,7 +747,7 @@ cudaError_t launch_tc_variant(mava_rollout *h, const RolloutArgs &args) {
   int ept = (h->cfg.n_envs + slots - 1) / slots;
   if (ept > S::EPT_MAX) ept = S::EPT_MAX;
   if (ept < 1) ept = 1;
-  if (!TM) {  // tiles whose observation block is a whole number of 16-byte pieces leave as one bulk copy
+  if (!TM || S::STG) {  // tiles whose observation block is a whole number of 16-byte pieces leave as one bulk copy
     for (int e = ept; e <= S::EPT_MAX; ++e)
       if ((e * N * S::D) % 4 == 0) { ept = e; break; }
   }
@@ -769,14 +775,18 @@ bool tc_supported(const mava_config_t &cfg) {
   return v == 0 || v == 1 || v == 2 || v == 3 || v == 4 || v == 5 || v == 6;
 }
 
-// Hidden activations in tensor memory: always for H = 256; for the smaller shapes only when the
-// handle asks for it (MAVA_FLAG_HIDDEN_IN_TMEM), which lets small cases exercise that path.
-static bool use_tm(const mava_rollout *h) { return h->variant >= 3 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0; }
+// Hidden activations in tensor memory: always for H >= 128 (at H = 128 the fp32 observation block keeps its shared
+// memory to itself and its bulk copy has a whole step to read it: 6 % faster than sharing that memory with the
+// activations); at H = 64 only when the handle asks for it (MAVA_FLAG_HIDDEN_IN_TMEM), which keeps both layouts
+// of the 128-row kernel in use.
+static bool use_tm(const mava_rollout *h) {
+  return h->cfg.hidden >= 128 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0;
+}
 
 bool tc_rollout_is_wide(const mava_rollout *h) {
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return false;
-  if (use_tm(h) || h->cfg.env_kind != 0) return true;
+  if (h->cfg.env_kind != 0 || (h->cfg.flags & MAVA_FLAG_HIDDEN_IN_TMEM) != 0) return true;
   if (h->variant == 1) return few_rows_tile<2, 128, false>(h, sms) == 0;
   if (h->variant == 2) return few_rows_tile<3, 128, false>(h, sms) == 0;
   return true;
@@ -807,17 +817,17 @@ cudaError_t launch_prep_tc(mava_rollout *h, const float *params_dev) {
 
 cudaError_t launch_rollout_tc(mava_rollout *h, const RolloutArgs &args) {
   const bool tm = use_tm(h);
-  if (h->cfg.env_kind != 0) {  // the warehouse family: two shapes, hidden activations in shared memory
+  if (h->cfg.env_kind != 0) {  // the warehouse family: two shapes
     switch (h->variant) {
       case 0: return launch_tc_variant<2, 2, 64, false, 1>(h, args);
-      case 2: return launch_tc_variant<3, 3, 128, false, 1>(h, args);
+      case 2: return launch_tc_variant<3, 3, 128, true, 1>(h, args);
       default: return cudaErrorNotSupported;
     }
   }
   switch (h->variant) {
     case 0: return tm ? launch_tc_variant<2, 2, 64, true>(h, args) : launch_tc_variant<2, 2, 64, false>(h, args);
-    case 1: return tm ? launch_tc_variant<2, 2, 128, true>(h, args) : launch_tc_variant<2, 2, 128, false>(h, args);
-    case 2: return tm ? launch_tc_variant<3, 3, 128, true>(h, args) : launch_tc_variant<3, 3, 128, false>(h, args);
+    case 1: return launch_tc_variant<2, 2, 128, true>(h, args);
+    case 2: return launch_tc_variant<3, 3, 128, true>(h, args);
     case 3: return launch_tc_variant<4, 5, 256, true>(h, args);
     case 4: return launch_tc_variant<8, 8, 256, true>(h, args);
     default: return cudaErrorNotSupported;
