@@ -555,33 +555,22 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
       if (!timed_out && n_items > 0) mma_commit(done_bar);  // covers every MMA issued above
     }
   } else {
-    // ---- consumers: column sums of the d z tile for the bias gradient.  Warp w covers feature chunks 4 w .. 4 w + 3 (units
-    // 32 w .. 32 w + 31); lane l reads row l's 16-byte piece of a chunk (a warp's 32 pieces are 512 contiguous-by-group
-    // bytes: no bank conflict beyond the four wavefronts 512 bytes need), the eight values are summed over the lanes by
-    // a butterfly, and lane l keeps the sum of unit 32 w + l.  Fixed order: the same bytes on every call.
-    const uint32_t row_off = static_cast<uint32_t>((lane >> 3) * 2048 + (lane & 7) * 16);
+    // ---- consumers: column sums of the d z tile for the bias gradient; thread j sums unit j over the item's rows.
+    // A warp's 32 units are four 16-byte chunks 128 bytes apart, i.e. on the same four banks: each chunk's eight lanes
+    // therefore start at a different row of the 8-row group (row offset 16 bytes = four banks) and the warp's loads
+    // touch 16 distinct banks.  The order of a thread's additions is fixed: the same bytes on every call.
+    const uint32_t my_col = static_cast<uint32_t>(tid >> 7) * kQ + static_cast<uint32_t>(((tid & 127) >> 3) * 128 + (tid & 7) * 2);
+    const int rot = (lane >> 3) * 2;
     for (int u = 0; u < n_items && !timed_out; ++u) {
       const int s = u % S;
       const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
       timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
       if (__any_sync(0xFFFFFFFFu, timed_out)) { timed_out = true; break; }
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int chunk = 4 * warp + cc;  // 0..31: unit half chunk >> 4, chunk inside it chunk & 15
-        const uint4 q = lds_v4(base + static_cast<uint32_t>(chunk >> 4) * kQ + static_cast<uint32_t>(chunk & 15) * 128u + row_off);
-        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
-        float v[8];
+      for (int rg = 0; rg < kItemRows / 8; ++rg)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) { v[2 * e] = __uint_as_float(w4[e] << 16); v[2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u); }
-#pragma unroll
-        for (int e = 0; e < 8; ++e)
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v[e] += __shfl_xor_sync(0xFFFFFFFFu, v[e], o);
-        float pick = v[0];
-#pragma unroll
-        for (int e = 1; e < 8; ++e) pick = ((lane & 7) == e) ? v[e] : pick;
-        if ((lane >> 3) == cc) db += pick;
-      }
+        for (int j = 0; j < 8; ++j)
+          db += __uint_as_float(lds_u16(base + my_col + static_cast<uint32_t>(rg * 2048) + static_cast<uint32_t>(((j + rot) & 7) * 16)) << 16);
       // the stage's next writer is a bulk copy (async proxy); these were generic-proxy reads.  Without the proxy fence
       // the copy may land before the reads have been performed (seen on the GPU as bias sums that changed from call to call).
       fence_async_smem();
