@@ -109,6 +109,11 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ void stg_v4(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -165,7 +170,9 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
   double t_actor = 0.0, t_ent = 0.0, t_value = 0.0;
   float gbh = 0.0f;
   // this thread's 16-byte pieces of a staged activation: unit half `half`, its own row
-  const size_t act_row_off = static_cast<size_t>(half) * kHalfBytes + static_cast<size_t>((row >> 3) * 2048 + (row & 7) * 16);
+  // a staged activation tile is [128 rows][256 units] in the canonical layout: 8-row groups 4096 bytes apart, a row's
+  // 16-byte pieces (8 units) 128 bytes apart; this thread's units start at piece 16 * half
+  const size_t act_row_off = static_cast<size_t>((row >> 3) * 4096 + (row & 7) * 16) + static_cast<size_t>(half) * 2048;
 
   // 128 accumulator columns of this thread (+ bias, ReLU) -> bf16 -> tensor memory (A operand of the next product) and
   // the staged tile; gate bits out
@@ -441,10 +448,10 @@ ppo_rows256_kernel(const unsigned char *__restrict__ image, UpdRows rows, UpdHyp
 // the bias gradient).  A stage is free again when its MMAs have completed and every consumer warp has let go of it.
 constexpr int kItemRows = 32;
 constexpr int kItemsPerTile = kR / kItemRows;
-constexpr uint32_t kQ = kItemRows * 128 * 2;                  // an item's rows of a [128][128] unit-half tile: 8 KB
-constexpr uint32_t kW2Stage = 4 * kQ, kW2Stages = 6;          // d z2 (two unit halves), h1 (two unit halves)
+constexpr uint32_t kQ = kItemRows * 128 * 2;                  // half of an item's rows of a [128][256] tile: 8 KB
+constexpr uint32_t kW2Stage = 4 * kQ, kW2Stages = 6;          // d z2, h1 (16 KB each: 32 rows x 256 units)
 constexpr uint32_t kXPart = (kItemRows / 8) * kXSbo, kDhPart = kItemRows * kHeads * 2;
-constexpr uint32_t kW1Stage = 4 * kQ + kXPart + kDhPart, kW1Stages = 5;  // d z1, h2 (two unit halves each), x, dhead
+constexpr uint32_t kW1Stage = 4 * kQ + kXPart + kDhPart, kW1Stages = 5;  // d z1, h2 (16 KB each), x, dhead
 constexpr uint32_t kRingBytes = kW2Stage * kW2Stages > kW1Stage * kW1Stages ? kW2Stage * kW2Stages : kW1Stage * kW1Stages;
 constexpr int kMaxStages = 6;
 constexpr int kWgtThreads = 320, kConsumerWarps = 8;
@@ -492,7 +499,7 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
   const int my_tiles = rank < n_tiles ? (n_tiles - rank + peers - 1) / peers : 0;
   const int n_items = kItemsPerTile * my_tiles;
   bool timed_out = false;
-  float db = 0.0f;  // consumer thread j: bias gradient of out unit j (d b2 or d b1)
+  float db0 = 0.0f, db1 = 0.0f;  // consumer thread: bias gradient (d b2 or d b1) of its two units over its half of the rows
 
   if (warp == kConsumerWarps) {
     // ---- producer
@@ -508,10 +515,11 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
         const uint32_t dst = ring + static_cast<uint32_t>(s) * stage_bytes, bar = full0 + 8u * s;
         mbar_expect_tx(bar, stage_bytes);
         const size_t a = role_w2 ? SL.dz2 : SL.dz1, b = role_w2 ? SL.h1 : SL.h2;
-        bulk_load(dst, st + a + static_cast<size_t>(q) * kQ, kQ, bar);
-        bulk_load(dst + kQ, st + a + kHalfBytes + static_cast<size_t>(q) * kQ, kQ, bar);
-        bulk_load(dst + 2 * kQ, st + b + static_cast<size_t>(q) * kQ, kQ, bar);
-        bulk_load(dst + 3 * kQ, st + b + kHalfBytes + static_cast<size_t>(q) * kQ, kQ, bar);
+        // an item's 32 rows of a staged tile are four 8-row groups = 16 KB in one piece (two copies of 8 KB each)
+        bulk_load(dst, st + a + static_cast<size_t>(q) * 2 * kQ, kQ, bar);
+        bulk_load(dst + kQ, st + a + static_cast<size_t>(q) * 2 * kQ + kQ, kQ, bar);
+        bulk_load(dst + 2 * kQ, st + b + static_cast<size_t>(q) * 2 * kQ, kQ, bar);
+        bulk_load(dst + 3 * kQ, st + b + static_cast<size_t>(q) * 2 * kQ + kQ, kQ, bar);
         if (!role_w2) {
           bulk_load(dst + 4 * kQ, st + SL.x + static_cast<size_t>(slab) * kStXBytes + static_cast<size_t>(q) * kXPart, kXPart, bar);
           bulk_load(dst + 4 * kQ + kXPart, st + SL.dh + static_cast<size_t>(q) * kDhPart, kDhPart, bar);
@@ -531,22 +539,23 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
         if (timed_out) break;
         tc_fence_after();
         const uint32_t keep = u > 0 ? 1u : 0u;
-        if (role_w2) {  // d W2 [out half a][in half b] += d z2[:, a]^T . h1[:, b] over the item's rows
+        if (role_w2) {  // d W2 [out half a][all 256 in] += d z2[:, a]^T . h1 over the item's rows: each operand piece is
+                        // read from shared memory 1.5 times per product instead of twice with four 128 x 128 products
 #pragma unroll
           for (int k = 0; k < kItemRows / 16; ++k)
 #pragma unroll
-            for (int ab = 0; ab < 4; ++ab)
-              mma_bf16(tmem + static_cast<uint32_t>(ab * 128), desc_mn(base + (ab >> 1) * kQ, 128, k), desc_mn(base + 2 * kQ + (ab & 1) * kQ, 128, k),
-                       instr_desc(128, 128) | kAmn | kBmn, keep | (k > 0));
+            for (int a = 0; a < 2; ++a)
+              mma_bf16(tmem + static_cast<uint32_t>(a * 256), desc_mn(base + a * 2048, 256, k), desc_mn(base + 2 * kQ, 256, k),
+                       instr_desc(128, 256) | kAmn | kBmn, keep | (k > 0));
         } else {        // d W1 [out half a][in] += d z1[:, a]^T . x;  d Wh^T [unit half a][head] += h2[:, a]^T . dhead
 #pragma unroll
           for (int k = 0; k < kItemRows / 16; ++k)
 #pragma unroll
             for (int a = 0; a < 2; ++a) {
-              mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * kQ, 128, k), smem_desc(base + 4 * kQ + k * 2 * kXSbo, kXSbo, kXLbo),
+              mma_bf16(tmem + static_cast<uint32_t>(a * kK1), desc_mn(base + a * 2048, 256, k), smem_desc(base + 4 * kQ + k * 2 * kXSbo, kXSbo, kXLbo),
                        instr_desc(128, kK1) | kAmn | kBmn, keep | (k > 0));
               if (heads_too)
-                mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * kQ, 128, k), desc_mn(base + 4 * kQ + kXPart, kHeads, k),
+                mma_bf16(tmem + static_cast<uint32_t>(192 + a * 32), desc_mn(base + 2 * kQ + a * 2048, 256, k), desc_mn(base + 4 * kQ + kXPart, kHeads, k),
                          instr_desc(128, kHeads) | kAmn | kBmn, keep | (k > 0));
             }
         }
@@ -555,22 +564,27 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
       if (!timed_out && n_items > 0) mma_commit(done_bar);  // covers every MMA issued above
     }
   } else {
-    // ---- consumers: column sums of the d z tile for the bias gradient; thread j sums unit j over the item's rows.
-    // A warp's 32 units are four 16-byte chunks 128 bytes apart, i.e. on the same four banks: each chunk's eight lanes
-    // therefore start at a different row of the 8-row group (row offset 16 bytes = four banks) and the warp's loads
-    // touch 16 distinct banks.  The order of a thread's additions is fixed: the same bytes on every call.
-    const uint32_t my_col = static_cast<uint32_t>(tid >> 7) * kQ + static_cast<uint32_t>(((tid & 127) >> 3) * 128 + (tid & 7) * 2);
-    const int rot = (lane >> 3) * 2;
+    // ---- consumers: column sums of the d z tile for the bias gradient.  Thread (w, l): units 2p, 2p + 1 with
+    // p = 32 (w & 3) + l, over the item's rows 16 (w >> 2) .. + 15, by 4-byte loads.  A warp's 32 unit pairs are eight
+    // 16-byte pieces 128 bytes apart, i.e. on the same four banks: each piece's four lanes therefore start at a
+    // different row of the 8-row group (row offset 16 bytes = four banks) and a load touches all 32 banks once.  The
+    // two row halves are added at the end, in a fixed order: the same bytes on every call.
+    const int p = (warp & 3) * 32 + lane;
+    const uint32_t my_col = static_cast<uint32_t>((p >> 2) * 128 + (p & 3) * 4) + static_cast<uint32_t>(warp >> 2) * 2 * 4096;
+    const int rot = lane >> 2;
     for (int u = 0; u < n_items && !timed_out; ++u) {
       const int s = u % S;
       const uint32_t base = ring + static_cast<uint32_t>(s) * stage_bytes;
       timed_out |= !mbar_wait(full0 + 8u * s, (u / S) & 1);
       if (__any_sync(0xFFFFFFFFu, timed_out)) { timed_out = true; break; }
 #pragma unroll
-      for (int rg = 0; rg < kItemRows / 8; ++rg)
+      for (int rg = 0; rg < 2; ++rg)
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          db += __uint_as_float(lds_u16(base + my_col + static_cast<uint32_t>(rg * 2048) + static_cast<uint32_t>(((j + rot) & 7) * 16)) << 16);
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t w2 = lds_u32(base + my_col + static_cast<uint32_t>(rg * 4096) + static_cast<uint32_t>(((j + rot) & 7) * 16));
+          db0 += __uint_as_float(w2 << 16);
+          db1 += __uint_as_float(w2 & 0xFFFF0000u);
+        }
       // the stage's next writer is a bulk copy (async proxy); these were generic-proxy reads.  Without the proxy fence
       // the copy may land before the reads have been performed (seen on the GPU as bias sums that changed from call to call).
       fence_async_smem();
@@ -581,6 +595,13 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
   // the consumer warps read the accumulators below; the other two warps go straight to the block-wide barrier
   if (warp < kConsumerWarps && n_items > 0 && !timed_out) timed_out |= !mbar_wait(done_bar, 0);
   timed_out = __syncthreads_or(timed_out) != 0;
+  {  // the two row halves of the bias sums meet in the ring, which is idle: every copy and every MMA has completed
+    float *xch = reinterpret_cast<float *>(sm.ring);
+    const int p = (warp & 3) * 32 + lane;
+    if (!timed_out && warp >= 4 && warp < kConsumerWarps) { xch[2 * p] = db0; xch[2 * p + 1] = db1; }
+    __syncthreads();
+    if (!timed_out && warp < 4) { db0 += xch[2 * p]; db1 += xch[2 * p + 1]; }
+  }
   if (!timed_out && my_tiles > 0 && warp < kConsumerWarps) {
     tc_fence_after();
     float *part = partial + static_cast<size_t>(blockIdx.x) * n_params;
@@ -595,7 +616,7 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
 #pragma unroll
           for (int c = 0; c < 16; ++c) dst[c] += v[c];
         }
-      part[net.b2 + tid] += db;
+      if (warp < 4) { part[net.b2 + 2 * tid] += db0; part[net.b2 + 2 * tid + 1] += db1; }
     } else {
       for (int c0 = 0; c0 < kK1; c0 += 16) {
         tmem_ld16(tmem + lane_off + static_cast<uint32_t>(a * kK1 + c0), v);
@@ -607,7 +628,7 @@ ppo_weights256_kernel(const unsigned char *__restrict__ staging, int n_tiles, in
         if (has_actor)
           for (int k = 0; k < kActions; ++k) part[net.Wa + static_cast<size_t>(k) * kH + unit] += v[k];
         if (has_value) part[net.Wv + unit] += v[kActions];
-        part[net.b1 + tid] += db;
+        if (warp < 4) { part[net.b1 + 2 * tid] += db0; part[net.b1 + 2 * tid + 1] += db1; }
       }
     }
   }
