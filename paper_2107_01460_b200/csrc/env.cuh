@@ -420,40 +420,75 @@ __device__ __forceinline__ void step_env_warp(EnvRegs<N, F> &s, const EnvParams 
     const bool inside = tr >= 0 && tr < G && tc >= 0 && tc < G;
     my_target = moving ? (inside ? (static_cast<uint32_t>(tr) | (static_cast<uint32_t>(tc) << 8)) : 0xFFFEu) : 0xFFFFu;
   }
-  // everybody's action and target, one shuffle per agent
-  int act[N];
-  uint32_t target[N];
-  const uint32_t mine_packed = my_target | (static_cast<uint32_t>(action) << 16);
-#pragma unroll
-  for (int m = 0; m < N; ++m) {
-    const uint32_t w = __shfl_sync(kFull, mine_packed, base + m);
-    act[m] = static_cast<int>(w >> 16);
-    target[m] = w & 0xFFFFu;
-  }
-  bool ok = my_target < 0xFFFEu;  // moving and inside the grid
-#pragma unroll
-  for (int f = 0; f < F; ++f) ok = ok && !((s.ent[N + f] >> 16) != 0 && (s.ent[N + f] & 0xFFFFu) == my_target);
-#pragma unroll
-  for (int m = 0; m < N; ++m)
-    ok = ok && (m == ag || ((s.ent[m] & 0xFFFFu) != my_target && target[m] != my_target));
-  const uint32_t my_new = ok ? my_target : my_pos;
-  // foods: lane `ag` decides foods ag, ag + N, ...
+  uint32_t my_new;
   uint32_t collected_mask = 0;  // bit f: food f collected
+  if constexpr (N >= 3) {
+    // Who tries to load, as one bit per agent of this environment; and whether another agent of this environment wants
+    // the same cell: lanes with equal (environment, target) keys.  A lane that stays, leaves the grid or has no
+    // environment gets a key of its own.
+    const uint32_t loaders = (__ballot_sync(kFull, action == 5) >> base) & ((1u << N) - 1u);
+    const uint32_t key = my_target < 0xFFFEu ? (my_target | (static_cast<uint32_t>(base) << 16)) : (0x80000000u | (threadIdx.x & 31u));
+    const uint32_t same = __match_any_sync(kFull, key);
+    bool ok = my_target < 0xFFFEu && (same & (same - 1u)) == 0u;  // moving, inside the grid, alone with this target
+    // ... and the cell holds neither food nor an agent at the start of the step (this lane's own agent is elsewhere)
 #pragma unroll
-  for (int round = 0; round * N < F; ++round) {
-    uint32_t fe = 0;  // level 0: nothing to decide
+    for (int f = 0; f < F; ++f) ok = ok && !((s.ent[N + f] >> 16) != 0 && (s.ent[N + f] & 0xFFFFu) == my_target);
 #pragma unroll
-    for (int j = 0; j < N; ++j)
-      if (round * N + j < F) fe = (ag == j) ? s.ent[N + round * N + j] : fe;
-    const int fr = fe & 0xFF, fc = (fe >> 8) & 0xFF, fl = static_cast<int>(fe >> 16);
-    int load = 0;
+    for (int m = 0; m < N; ++m) ok = ok && (s.ent[m] & 0xFFFFu) != my_target;
+    my_new = ok ? my_target : my_pos;
+    // foods: lane `ag` decides foods ag, ag + N, ...
+#pragma unroll
+    for (int round = 0; round * N < F; ++round) {
+      uint32_t fe = 0;  // level 0: nothing to decide
+#pragma unroll
+      for (int j = 0; j < N; ++j)
+        if (round * N + j < F) fe = (ag == j) ? s.ent[N + round * N + j] : fe;
+      const uint32_t fpos = fe & 0xFFFFu;
+      const int fl = static_cast<int>(fe >> 16);
+      int load = 0;
+#pragma unroll
+      for (int m = 0; m < N; ++m) {
+        const uint32_t dist = __vsadu4(s.ent[m] & 0xFFFFu, fpos);  // |row difference| + |column difference|
+        load += (((loaders >> m) & 1u) != 0u && dist == 1u) ? static_cast<int>(s.ent[m] >> 16) : 0;
+      }
+      const uint32_t bal = __ballot_sync(kFull, fl > 0 && load >= fl);
+      collected_mask |= ((bal >> base) & ((1u << N) - 1u)) << (round * N);
+    }
+  } else {  // two agents: two shuffles are cheaper than a match across the warp
+    // everybody's action and target, one shuffle per agent
+    int act[N];
+    uint32_t target[N];
+    const uint32_t mine_packed = my_target | (static_cast<uint32_t>(action) << 16);
 #pragma unroll
     for (int m = 0; m < N; ++m) {
-      const int dist = abs(static_cast<int>(s.ent[m] & 0xFF) - fr) + abs(static_cast<int>((s.ent[m] >> 8) & 0xFF) - fc);
-      load += (act[m] == 5 && dist == 1) ? static_cast<int>(s.ent[m] >> 16) : 0;
+      const uint32_t w = __shfl_sync(kFull, mine_packed, base + m);
+      act[m] = static_cast<int>(w >> 16);
+      target[m] = w & 0xFFFFu;
     }
-    const uint32_t bal = __ballot_sync(kFull, fl > 0 && load >= fl);
-    collected_mask |= ((bal >> base) & ((1u << N) - 1u)) << (round * N);
+    bool ok = my_target < 0xFFFEu;  // moving and inside the grid
+#pragma unroll
+    for (int f = 0; f < F; ++f) ok = ok && !((s.ent[N + f] >> 16) != 0 && (s.ent[N + f] & 0xFFFFu) == my_target);
+#pragma unroll
+    for (int m = 0; m < N; ++m)
+      ok = ok && (m == ag || ((s.ent[m] & 0xFFFFu) != my_target && target[m] != my_target));
+    my_new = ok ? my_target : my_pos;
+    // foods: lane `ag` decides foods ag, ag + N, ...
+#pragma unroll
+    for (int round = 0; round * N < F; ++round) {
+      uint32_t fe = 0;  // level 0: nothing to decide
+#pragma unroll
+      for (int j = 0; j < N; ++j)
+        if (round * N + j < F) fe = (ag == j) ? s.ent[N + round * N + j] : fe;
+      const int fr = fe & 0xFF, fc = (fe >> 8) & 0xFF, fl = static_cast<int>(fe >> 16);
+      int load = 0;
+#pragma unroll
+      for (int m = 0; m < N; ++m) {
+        const int dist = abs(static_cast<int>(s.ent[m] & 0xFF) - fr) + abs(static_cast<int>((s.ent[m] >> 8) & 0xFF) - fc);
+        load += (act[m] == 5 && dist == 1) ? static_cast<int>(s.ent[m] >> 16) : 0;
+      }
+      const uint32_t bal = __ballot_sync(kFull, fl > 0 && load >= fl);
+      collected_mask |= ((bal >> base) & ((1u << N) - 1u)) << (round * N);
+    }
   }
   // apply: every lane updates its copy identically
   int gained = 0, left = 0;

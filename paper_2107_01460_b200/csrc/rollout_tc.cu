@@ -491,7 +491,7 @@ rollout_tc_kernel(RolloutArgs a, const unsigned char *__restrict__ image, int ep
       const size_t row0 = static_cast<size_t>(t) * M + static_cast<size_t>(e0) * N;
       if (PP) {
         pair_sync(kBarTile + g, TP);  // the other group (and the helpers' copy of its rows) is done with the A tile
-        // one verdict for the whole group (its threads may see the flag at different times); the flag
+        // one decision for the whole group (its threads may see the flag at different times); the flag
         // is looked at every eighth step only: the load would queue behind the partner's copy-out
         idle = group_any(g, idle || ((t & 7) == 0 && lds_s32(abort_addr) != 0));
         if (idle) {  // keep the hand-over order of a working step: three acquisitions, then three releases
