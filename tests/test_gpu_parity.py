@@ -71,7 +71,10 @@ def test_reduced_configs_fp32(idx, n_envs, T):
 @pytest.mark.parametrize("idx,n_envs,T,mode", [(1, 333, 60, ""), (2, 300, 110, ""), (3, 200, 105, ""),
                                                (4, 150, 40, ""), (0, 16, 32, "tmem"), (1, 333, 60, "tmem"),
                                                (2, 300, 110, "tmem"), (1, 333, 60, "wide"), (2, 300, 110, "wide"),
-                                               (1, 1500, 40, ""), (2, 1000, 40, ""), (1, 1500, 40, "wide")])
+                                               (1, 1500, 40, ""), (2, 1000, 40, ""), (1, 1500, 40, "wide"),
+                                               # H = 256 with more tiles than one round holds and an odd count: a second
+                                               # round in which one thread group of a CTA has no tile (on 148 SMs)
+                                               (4, 4737, 12, ""), (3, 9473, 7, "")])
 def test_reduced_configs_bf16(idx, n_envs, T, mode):
     """mode "tmem" keeps the hidden activations in tensor memory (the layout H = 256 always uses);
     "wide" forces 128-row tiles where the batch is small enough for the few-rows form of the kernel
